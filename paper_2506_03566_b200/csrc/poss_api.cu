@@ -1,0 +1,616 @@
+// Host side of the PosS library: context, workspace layout, argument checks and the launch chains
+// of a draft round, the target pass and verification.  No device memory is allocated here; every
+// buffer is carved out of the caller's workspace.
+#include "poss_internal.cuh"
+#include "gemm_tc.cuh"
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+namespace {
+
+constexpr int R = POSS_MAX_ROWS;
+constexpr int KMAX = POSS_MAX_TOPK;
+constexpr int ATTN_MAX_SPLITS = 16;
+
+struct Bump {
+  size_t off = 0;
+  char* base = nullptr;
+  template <typename P> P* take(size_t count, size_t elem) {
+    size_t bytes = (count * elem + 255) / 256 * 256;
+    P* p = base ? reinterpret_cast<P*>(base + off) : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+struct Buffers {
+  void* X;            // [R][2H] act
+  float* h0;          // [R][H]
+  void* xn;           // [R][H] act
+  float* qkv;         // [R][(Hq+2Hkv)d]
+  void* q;            // [R][Hq d] act
+  float* attn_part;
+  void* o;            // [R][Hq d] act
+  float* h1;          // [R][H]
+  void* u;            // [R][H] act
+  float* gu;          // [R][2F]
+  void* act;          // [R][F] act
+  float* fout;        // [Lmax][KMAX][H] fp32 specialist features per level
+  void* fb;           // same, act dtype (layer input of the children, LM-head operand)
+  float* hx;          // [R][H] target residual stream
+  float* tfeat;       // [R][H] target features fp32
+  float* logits;      // [R][V]
+  float* pmax; float* psum; float* pval; int32_t* pidx;   // top-k partials
+  int32_t* top_ids;   // [R][KMAX]
+  float* top_logp;    // [R][KMAX]
+  uint64_t* chain_mask;  // [R][2]
+  int32_t* chain_depth;  // [R]
+  int32_t* argmax_tmp;   // [R]
+  unsigned long long* counters;  // [POSS_MAX_DEPTH + 2]
+  int32_t* status;       // [1]
+  void* tc_scratch;      // split-K partials + tile counters of the tensor-core GEMM
+  TreeState ts;
+};
+
+}  // namespace
+
+struct poss_ctx {
+  poss_config cfg;
+  poss_layer_w* spec;
+  poss_layer_w* tgt;
+  const void *embed, *lm_head, *final_norm;
+  Buffers b;
+  size_t esize;          // bytes of the context dtype
+  int n_chunks;          // vocabulary chunks of the top-k kernels
+  int n_cand_max;
+  int64_t launches;
+  int last_depth, last_topk, last_nodes;
+  TcGemmPlanCache* tc;
+};
+
+namespace {
+
+int n_cand_of(int depth, int topk) { return topk + (depth - 1) * topk * topk; }
+
+bool config_ok(const poss_config* c, int* why) {
+  *why = POSS_E_INVALID;
+  if (!c) return false;
+  if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->ffn <= 0 || c->vocab <= 0) return false;
+  if (c->dtype != POSS_FP32 && c->dtype != POSS_BF16) return false;
+  if (c->n_specialists < 1 || c->positions_per_specialist < 1) return false;
+  if (c->n_target_layers < 0 || c->draft_kv_slots < 1) return false;
+  if (c->n_target_layers > 0 && c->target_kv_slots < 1) return false;
+  *why = POSS_E_SHAPE;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  int g = c->n_q_heads / c->n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 3 || g == 4 || g == 8)) return false;
+  if (c->hidden % 8 || c->ffn % 8) return false;
+  *why = POSS_E_CAPACITY;
+  if (c->max_depth < 1 || c->max_depth > POSS_MAX_DEPTH) return false;
+  if (c->max_topk < 1 || c->max_topk > POSS_MAX_TOPK) return false;
+  if (c->max_total < 1 || c->max_total > 255) return false;
+  if ((c->max_depth - 1) * c->max_topk > 128) return false;   // tree-slot mask is two 64-bit words
+  if ((c->max_depth - 1) * c->max_topk + 1 > R) return false;
+  if (c->vocab < c->max_topk) return false;
+  *why = POSS_OK;
+  return true;
+}
+
+void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_cand_max) {
+  size_t es = c.dtype == POSS_BF16 ? 2 : 4;
+  size_t H = c.hidden, F = c.ffn, V = c.vocab;
+  size_t qd = (size_t)c.n_q_heads * c.head_dim, kd = (size_t)c.n_kv_heads * c.head_dim;
+  int L = c.max_depth;
+  *n_chunks = (int)((V + POSS_TOPK_CHUNK - 1) / POSS_TOPK_CHUNK);
+  *n_cand_max = n_cand_of(c.max_depth, c.max_topk);
+  b.X = bp.take<void>(R * 2 * H, es);
+  b.h0 = bp.take<float>(R * H, 4);
+  b.xn = bp.take<void>(R * H, es);
+  b.qkv = bp.take<float>(R * (qd + 2 * kd), 4);
+  b.q = bp.take<void>(R * qd, es);
+  b.attn_part = bp.take<float>(attn_partial_floats(R, c.n_q_heads, c.head_dim, ATTN_MAX_SPLITS), 4);
+  b.o = bp.take<void>(R * qd, es);
+  b.h1 = bp.take<float>(R * H, 4);
+  b.u = bp.take<void>(R * H, es);
+  b.gu = bp.take<float>(R * 2 * F, 4);
+  b.act = bp.take<void>(R * F, es);
+  b.fout = bp.take<float>((size_t)L * KMAX * H, 4);
+  b.fb = bp.take<void>((size_t)L * KMAX * H, es);
+  b.hx = bp.take<float>(R * H, 4);
+  b.tfeat = bp.take<float>(R * H, 4);
+  b.logits = bp.take<float>(R * V, 4);
+  b.pmax = bp.take<float>((size_t)R * *n_chunks, 4);
+  b.psum = bp.take<float>((size_t)R * *n_chunks, 4);
+  b.pval = bp.take<float>((size_t)R * *n_chunks * KMAX, 4);
+  b.pidx = bp.take<int32_t>((size_t)R * *n_chunks * KMAX, 4);
+  b.top_ids = bp.take<int32_t>(R * KMAX, 4);
+  b.top_logp = bp.take<float>(R * KMAX, 4);
+  b.chain_mask = bp.take<uint64_t>(R * 2, 8);
+  b.chain_depth = bp.take<int32_t>(R, 4);
+  b.argmax_tmp = bp.take<int32_t>(R, 4);
+  b.counters = bp.take<unsigned long long>(POSS_MAX_DEPTH + 2, 8);
+  b.status = bp.take<int32_t>(64, 4);
+  b.tc_scratch = bp.take<void>(tc_gemm_scratch_bytes(), 1);
+  b.ts.cand_tok = bp.take<int32_t>(*n_cand_max, 4);
+  b.ts.cand_parent = bp.take<int32_t>(*n_cand_max, 4);
+  b.ts.cand_score = bp.take<float>(*n_cand_max, 4);
+  b.ts.node_tok = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
+  b.ts.node_prow = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
+  b.ts.node_cand = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
+  b.ts.node_score = bp.take<float>((size_t)(L + 1) * KMAX, 4);
+  b.ts.node_mask = bp.take<uint64_t>((size_t)(L + 1) * KMAX * 2, 8);
+  b.ts.selected = bp.take<int32_t>(256, 4);
+}
+
+inline cudaStream_t S(poss_stream s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// ------------------------------------------------------------------ typed implementation
+template <typename T>
+struct Impl {
+  poss_ctx* c;
+  Launcher L;
+  Impl(poss_ctx* ctx, poss_stream s) : c(ctx) { L.stream = S(s); L.launches = &ctx->launches; L.err = POSS_OK; }
+
+  const T* W(const void* p) const { return reinterpret_cast<const T*>(p); }
+  T* A(void* p) const { return reinterpret_cast<T*>(p); }
+
+  // out[M][N] = x . segs^T (+bias) (+residual); picks the tensor-core kernel when it applies
+  void gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual, int ldr,
+            float* out, int ldo, int impl = 0);
+
+  void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out) {
+    const poss_config& g = c->cfg;
+    GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = g.vocab;
+    float* lg = logits_out ? logits_out : c->b.logits;
+    gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
+    launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
+    launch_topk_merge(L, rows, K, c->n_chunks, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp);
+  }
+
+  // fc + norm + K/V(+Q) projection + rotary + cache append for one batch of a specialist
+  void project_rows(const poss_layer_w& lw, const StepRows& s, const int32_t* new_tokens, const T* new_features,
+                    T* kcache, T* vcache, bool with_q) {
+    const poss_config& g = c->cfg;
+    Buffers& b = c->b;
+    int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
+    launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), W(c->embed), H, A(b.X));
+    GemmSegs fc; fc.n = 1; fc.w[0] = lw.fc_w; fc.rows[0] = H;
+    gemm(A(b.X), 2 * H, s.M, fc, 2 * H, W(lw.fc_b), nullptr, 0, b.h0, H);
+    launch_rmsnorm<T>(L, b.h0, s.M, H, W(lw.norm_in), g.rms_eps, A(b.xn));
+    GemmSegs qkv; qkv.n = 3;
+    qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
+    gemm(A(b.xn), H, s.M, qkv, H, nullptr, nullptr, 0, b.qkv, qd + 2 * kd);
+    RopeArgs ra;
+    ra.mode = 0; ra.s = s; ra.base = 0; ra.depth = nullptr; ra.rows = s.M; ra.q_rows = with_q ? s.Mc : 0;
+    ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.draft_kv_slots; ra.theta = g.rope_theta;
+    launch_rope_append<T>(L, ra, b.qkv, kcache, vcache, A(b.q));
+  }
+
+  // attention output -> O-proj + residual -> MLP + residual; x0 = layer input rows, result in `out`
+  void layer_tail(const poss_layer_w& lw, const float* x0, int rows, float* out) {
+    const poss_config& g = c->cfg;
+    Buffers& b = c->b;
+    int H = g.hidden, qd = g.n_q_heads * g.head_dim, F = g.ffn;
+    GemmSegs so; so.n = 1; so.w[0] = lw.wo; so.rows[0] = H;
+    gemm(A(b.o), qd, rows, so, qd, nullptr, x0, H, b.h1, H);
+    launch_rmsnorm<T>(L, b.h1, rows, H, W(lw.norm_post), g.rms_eps, A(b.u));
+    GemmSegs sg; sg.n = 2; sg.w[0] = lw.w_gate; sg.rows[0] = F; sg.w[1] = lw.w_up; sg.rows[1] = F;
+    gemm(A(b.u), H, rows, sg, H, nullptr, nullptr, 0, b.gu, 2 * F);
+    launch_silu_mul<T>(L, b.gu, rows, F, A(b.act));
+    GemmSegs sd; sd.n = 1; sd.w[0] = lw.w_down; sd.rows[0] = H;
+    gemm(A(b.act), F, rows, sd, F, nullptr, b.h1, H, out, H);
+  }
+
+  int draft_prefill(void* draft_kv, int start, const int32_t* tokens, const void* features, int n) {
+    const poss_config& g = c->cfg;
+    size_t per_spec = (size_t)2 * g.n_kv_heads * g.draft_kv_slots * g.head_dim;
+    size_t half = per_spec / 2;
+    for (int s = 0; s < g.n_specialists; ++s) {
+      T* kc = A(draft_kv) + s * per_spec;
+      for (int off = 0; off < n; off += R) {
+        int m = n - off < R ? n - off : R;
+        StepRows sr; sr.n_ver = m; sr.n_lvl = 0; sr.cur_level = 0; sr.K = 1; sr.n_new = m;
+        sr.prefix_len = start + off; sr.M = m; sr.Mc = 0;
+        project_rows(c->spec[s], sr, tokens + off, W(features) + (size_t)off * g.hidden, kc, kc + half, false);
+      }
+    }
+    return L.err;
+  }
+
+  int draft_round(void* draft_kv, int prefix_len, const int32_t* new_tokens, const void* new_features, int n_new,
+                  int depth, int K, int total, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
+                  int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
+    const poss_config& g = c->cfg;
+    Buffers& b = c->b;
+    int H = g.hidden, n = g.positions_per_specialist, Sn = g.n_specialists;
+    size_t per_spec = (size_t)2 * g.n_kv_heads * g.draft_kv_slots * g.head_dim;
+    size_t half = per_spec / 2;
+    bool used[64] = {false};
+    int cand_base = 0;
+    for (int i = 0; i < depth; ++i) {
+      int s = i / n < Sn - 1 ? i / n : Sn - 1;          // specialist ceil((i+1)/n), clamped, 0-based
+      bool first = !used[s < 64 ? s : 63];
+      used[s < 64 ? s : 63] = true;
+      StepRows sr;
+      sr.K = K; sr.n_new = n_new; sr.prefix_len = prefix_len; sr.cur_level = i;
+      sr.n_ver = first ? n_new : 0;
+      sr.n_lvl = first && i >= 1 ? (i - 1) * K : 0;
+      sr.Mc = i == 0 ? 1 : K;
+      sr.M = sr.n_ver + sr.n_lvl + (i == 0 ? 0 : K);
+      if (i == 0 && !first) { sr.n_ver = 1; sr.M = 1; }   // unreachable: step 0 is always a first use
+      T* kc = A(draft_kv) + s * per_spec;
+      T* vc = kc + half;
+      const poss_layer_w& lw = c->spec[s];
+      project_rows(lw, sr, new_tokens, W(new_features), kc, vc, true);
+      AttnArgs aa;
+      aa.rows = sr.Mc; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.draft_kv_slots;
+      aa.n_all = prefix_len + n_new; aa.n_tree = i * K;
+      aa.mask = b.ts.node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
+      aa.scale = 1.0f / sqrtf((float)g.head_dim);
+      plan_attention_splits(aa.rows, aa.Hkv, aa.n_all + aa.n_tree, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
+      launch_tree_attention<T>(L, aa, A(b.q), kc, vc, b.attn_part, A(b.o));
+      float* fo = b.fout + (size_t)i * KMAX * H;
+      T* fbi = A(b.fb) + (size_t)i * KMAX * H;
+      layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo);
+      launch_cast_rows<T>(L, fo, (size_t)sr.Mc * H, fbi);
+      lm_head_topk(fbi, sr.Mc, K, b.top_ids, b.top_logp, nullptr);
+      launch_expand(L, b.ts, KMAX, i, sr.Mc, K, cand_base, i == depth - 1, b.top_ids, b.top_logp);
+      cand_base += sr.Mc * K;
+    }
+    // specialists the round did not reach still cache the verified pairs
+    for (int s = 0; s < Sn && s < 64; ++s) {
+      if (used[s]) continue;
+      StepRows sr; sr.n_ver = n_new; sr.n_lvl = 0; sr.cur_level = 0; sr.K = K; sr.n_new = n_new;
+      sr.prefix_len = prefix_len; sr.M = n_new; sr.Mc = 0;
+      T* kc = A(draft_kv) + s * per_spec;
+      project_rows(c->spec[s], sr, new_tokens, W(new_features), kc, kc + half, false);
+    }
+    launch_rerank(L, b.ts, cand_base, K, total, n_new - 1, new_tokens, out_tokens, out_parents, out_scores, out_depth,
+                  out_mask, out_n_nodes);
+    c->last_depth = depth; c->last_topk = K;
+    c->last_nodes = 1 + (total < cand_base ? total : cand_base);
+    return L.err;
+  }
+
+  int tree_attention(const void* q, const void* kv, int kv_slots, int prefix_len, int rows, const uint64_t* mask,
+                     float scale, void* out) {
+    const poss_config& g = c->cfg;
+    AttnArgs aa;
+    aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = kv_slots;
+    aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = (rows + 63) / 64; aa.scale = scale;
+    plan_attention_splits(rows, aa.Hkv, prefix_len + rows, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
+    const T* kc = W(kv);
+    const T* vc = kc + (size_t)g.n_kv_heads * kv_slots * g.head_dim;
+    launch_tree_attention<T>(L, aa, W(q), kc, vc, c->b.attn_part, A(out));
+    return L.err;
+  }
+
+  int target_forward(void* target_kv, int prefix_len, const int32_t* tokens, const int32_t* depth,
+                     const uint64_t* mask, int mask_words, int rows, void* out_features, int32_t* out_argmax,
+                     float* out_logits) {
+    const poss_config& g = c->cfg;
+    Buffers& b = c->b;
+    int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
+    size_t per_layer = (size_t)2 * g.n_kv_heads * g.target_kv_slots * g.head_dim;
+    launch_embed_rows<T>(L, tokens, rows, W(c->embed), H, b.hx);
+    for (int li = 0; li < g.n_target_layers; ++li) {
+      const poss_layer_w& lw = c->tgt[li];
+      T* kc = A(target_kv) + li * per_layer;
+      T* vc = kc + per_layer / 2;
+      launch_rmsnorm<T>(L, b.hx, rows, H, W(lw.norm_in), g.rms_eps, A(b.xn));
+      GemmSegs qkv; qkv.n = 3;
+      qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
+      gemm(A(b.xn), H, rows, qkv, H, nullptr, nullptr, 0, b.qkv, qd + 2 * kd);
+      RopeArgs ra;
+      ra.mode = 1; ra.base = prefix_len; ra.depth = depth; ra.rows = rows; ra.q_rows = rows;
+      ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.target_kv_slots;
+      ra.theta = g.rope_theta; memset(&ra.s, 0, sizeof(ra.s));
+      launch_rope_append<T>(L, ra, b.qkv, kc, vc, A(b.q));
+      AttnArgs aa;
+      aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.target_kv_slots;
+      aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = mask_words;
+      aa.scale = 1.0f / sqrtf((float)g.head_dim);
+      plan_attention_splits(rows, aa.Hkv, prefix_len + rows, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
+      launch_tree_attention<T>(L, aa, A(b.q), kc, vc, b.attn_part, A(b.o));
+      layer_tail(lw, b.hx, rows, b.hx);
+    }
+    launch_rmsnorm<T>(L, b.hx, rows, H, W(c->final_norm), g.rms_eps, A(out_features));
+    if (out_argmax || out_logits)
+      lm_head_topk(A(out_features), rows, 1, out_argmax ? out_argmax : b.argmax_tmp, b.top_logp, out_logits);
+    return L.err;
+  }
+};
+
+template <typename T>
+void Impl<T>::gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual,
+                   int ldr, float* out, int ldo, int impl) {
+  launch_gemm_simt<T>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
+}
+template <>
+void Impl<bf16>::gemm(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, const bf16* bias,
+                      const float* residual, int ldr, float* out, int ldo, int impl) {
+  bool can_tc = tc_gemm_supported(segs, K, ldx, M);
+  if (impl == 2 && !can_tc) { L.err = POSS_E_SHAPE; return; }
+  if (impl != 1 && can_tc)
+    launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, bias, residual, ldr, out, ldo, c->b.tc_scratch, c->b.status);
+  else
+    launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
+}
+
+#define DISPATCH(ctx, stream, call)                         \
+  ((ctx)->cfg.dtype == POSS_BF16 ? Impl<bf16>(ctx, stream).call : Impl<float>(ctx, stream).call)
+
+}  // namespace
+
+// ====================================================================== C ABI
+extern "C" {
+
+size_t poss_workspace_bytes(const poss_config* cfg) {
+  int why;
+  if (!config_ok(cfg, &why)) return 0;
+  Bump bp;
+  Buffers b;
+  int nc, ncand;
+  layout(*cfg, bp, b, &nc, &ncand);
+  return bp.off;
+}
+
+int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, void* workspace, size_t workspace_bytes,
+              poss_stream stream) {
+  if (!out) return POSS_E_INVALID;
+  *out = nullptr;
+  int why;
+  if (!config_ok(cfg, &why)) return why;
+  if (!w || !w->embed || !w->lm_head || !w->h_specialist) return POSS_E_INVALID;
+  if (cfg->n_target_layers > 0 && (!w->h_target || !w->target_final_norm)) return POSS_E_INVALID;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return POSS_E_WORKSPACE;
+  if (workspace_bytes < poss_workspace_bytes(cfg)) return POSS_E_WORKSPACE;
+  for (int s = 0; s < cfg->n_specialists; ++s) {
+    const poss_layer_w& l = w->h_specialist[s];
+    if (!l.fc_w || !l.wq || !l.wk || !l.wv || !l.wo || !l.norm_post || !l.w_gate || !l.w_up || !l.w_down)
+      return POSS_E_INVALID;
+  }
+  for (int s = 0; s < cfg->n_target_layers; ++s) {
+    const poss_layer_w& l = w->h_target[s];
+    if (!l.wq || !l.wk || !l.wv || !l.wo || !l.norm_post || !l.w_gate || !l.w_up || !l.w_down) return POSS_E_INVALID;
+  }
+  poss_ctx* c = new (std::nothrow) poss_ctx();
+  if (!c) return POSS_E_INVALID;
+  c->cfg = *cfg;
+  c->spec = (poss_layer_w*)malloc(sizeof(poss_layer_w) * cfg->n_specialists);
+  c->tgt = cfg->n_target_layers ? (poss_layer_w*)malloc(sizeof(poss_layer_w) * cfg->n_target_layers) : nullptr;
+  memcpy(c->spec, w->h_specialist, sizeof(poss_layer_w) * cfg->n_specialists);
+  if (c->tgt) memcpy(c->tgt, w->h_target, sizeof(poss_layer_w) * cfg->n_target_layers);
+  c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->target_final_norm;
+  c->esize = cfg->dtype == POSS_BF16 ? 2 : 4;
+  c->launches = 0; c->last_depth = 0; c->last_topk = 0; c->last_nodes = 0;
+  Bump bp;
+  bp.base = reinterpret_cast<char*>(workspace);
+  layout(*cfg, bp, c->b, &c->n_chunks, &c->n_cand_max);
+  c->tc = tc_plan_cache_create();
+  cudaStream_t st = S(stream);
+  bool ok = cudaMemsetAsync(workspace, 0, bp.off, st) == cudaSuccess;
+  Launcher L; L.stream = st; L.launches = &c->launches; L.err = POSS_OK;
+  launch_chain_mask(L, c->b.chain_mask, c->b.chain_depth, R);
+  ok = ok && L.err == POSS_OK && cudaStreamSynchronize(st) == cudaSuccess;
+  if (!ok) { poss_destroy(c); return POSS_E_CUDA; }
+  *out = c;
+  return POSS_OK;
+}
+
+int poss_destroy(poss_ctx* c) {
+  if (!c) return POSS_E_INVALID;
+  tc_plan_cache_destroy(c->tc);
+  free(c->spec);
+  free(c->tgt);
+  delete c;
+  return POSS_OK;
+}
+
+int poss_reset(poss_ctx* c, poss_stream stream) {
+  if (!c) return POSS_E_INVALID;
+  if (cudaMemsetAsync(c->b.counters, 0, sizeof(unsigned long long) * (POSS_MAX_DEPTH + 2), S(stream)) != cudaSuccess)
+    return POSS_E_CUDA;
+  if (cudaMemsetAsync(c->b.status, 0, sizeof(int32_t) * 64, S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  return POSS_OK;
+}
+
+int poss_draft_prefill(poss_ctx* c, void* draft_kv, int start, const int32_t* tokens, const void* features, int n,
+                       poss_stream stream) {
+  if (!c || !draft_kv || n < 0 || start < 0) return POSS_E_INVALID;
+  if (n == 0) return POSS_OK;
+  if (!tokens || !features) return POSS_E_INVALID;
+  if (start + n > c->cfg.draft_kv_slots) return POSS_E_CAPACITY;
+  return DISPATCH(c, stream, draft_prefill(draft_kv, start, tokens, features, n));
+}
+
+int poss_draft_round(poss_ctx* c, void* draft_kv, int prefix_len, const int32_t* new_tokens, const void* new_features,
+                     int n_new, int depth, int topk, int total, int32_t* out_tokens, int32_t* out_parents,
+                     float* out_scores, int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes,
+                     poss_stream stream) {
+  if (!c || !draft_kv || !new_tokens || !new_features || !out_tokens || !out_parents || !out_scores || !out_depth ||
+      !out_mask || !out_n_nodes)
+    return POSS_E_INVALID;
+  if (prefix_len < 0 || n_new < 1 || depth < 1 || topk < 1 || total < 1) return POSS_E_INVALID;
+  const poss_config& g = c->cfg;
+  if (depth > g.max_depth || topk > g.max_topk || total > g.max_total) return POSS_E_CAPACITY;
+  if (n_new + (depth - 1) * topk > R) return POSS_E_CAPACITY;
+  if (prefix_len + n_new + (depth - 1) * topk > g.draft_kv_slots) return POSS_E_CAPACITY;
+  return DISPATCH(c, stream, draft_round(draft_kv, prefix_len, new_tokens, new_features, n_new, depth, topk, total,
+                                         out_tokens, out_parents, out_scores, out_depth, out_mask, out_n_nodes));
+}
+
+int poss_draft_trace(poss_ctx* c, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores, int32_t* frontier,
+                     float* step_features, int32_t* selected, poss_stream stream) {
+  if (!c || c->last_depth < 1) return POSS_E_INVALID;
+  cudaStream_t st = S(stream);
+  int K = c->last_topk, Ld = c->last_depth, H = c->cfg.hidden;
+  size_t nc = n_cand_of(Ld, K);
+  bool ok = true;
+  auto cp = [&](void* dst, const void* src, size_t bytes) {
+    if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  };
+  cp(cand_tokens, c->b.ts.cand_tok, nc * 4);
+  cp(cand_parents, c->b.ts.cand_parent, nc * 4);
+  cp(cand_scores, c->b.ts.cand_score, nc * 4);
+  cp(selected, c->b.ts.selected, (size_t)(c->last_nodes - 1) * 4);
+  for (int l = 1; l < Ld; ++l) {
+    if (frontier) cp(frontier + (size_t)(l - 1) * K, c->b.ts.node_cand + (size_t)l * KMAX, (size_t)K * 4);
+  }
+  for (int l = 0; l < Ld; ++l) {
+    if (step_features)
+      cp(step_features + (size_t)l * K * H, c->b.fout + (size_t)l * KMAX * H, (size_t)(l == 0 ? 1 : K) * H * 4);
+  }
+  return ok ? POSS_OK : POSS_E_CUDA;
+}
+
+int poss_tree_attention(poss_ctx* c, const void* q, const void* kv, int kv_slots, int prefix_len, int rows,
+                        const uint64_t* anc_mask, float scale, void* out, poss_stream stream) {
+  if (!c || !q || !kv || !anc_mask || !out || prefix_len < 0 || rows < 0 || kv_slots < 1) return POSS_E_INVALID;
+  if (rows == 0) return POSS_OK;
+  if (rows > R) return POSS_E_CAPACITY;
+  if (prefix_len + rows > kv_slots) return POSS_E_CAPACITY;
+  return DISPATCH(c, stream, tree_attention(q, kv, kv_slots, prefix_len, rows, anc_mask, scale, out));
+}
+
+int poss_verify_accept(poss_ctx* c, const void* target_logits, const int32_t* target_argmax,
+                       const void* target_features, const int32_t* tokens, const int32_t* parents, int rows,
+                       int32_t* out_path, int32_t* out_n_accepted, int32_t* out_bonus, int32_t* out_new_tokens,
+                       void* out_new_features, poss_stream stream) {
+  if (!c || !target_features || !tokens || !parents || !out_path || !out_n_accepted || !out_bonus ||
+      !out_new_tokens || !out_new_features)
+    return POSS_E_INVALID;
+  if ((target_logits == nullptr) == (target_argmax == nullptr)) return POSS_E_INVALID;
+  if (rows < 1) return POSS_E_INVALID;
+  if (rows > 256) return POSS_E_CAPACITY;
+  Launcher L; L.stream = S(stream); L.launches = &c->launches; L.err = POSS_OK;
+  const int32_t* g = target_argmax;
+  const poss_config& cf = c->cfg;
+  if (target_logits) {
+    if (rows > R) return POSS_E_CAPACITY;
+    // row argmax over the vocabulary with the same chunked top-1 kernels (ties -> lowest id)
+    const float* lg;
+    if (cf.dtype == POSS_BF16) {
+      launch_widen_bf16(L, reinterpret_cast<const bf16*>(target_logits), (size_t)rows * cf.vocab, c->b.logits);
+      lg = c->b.logits;
+    } else {
+      lg = reinterpret_cast<const float*>(target_logits);
+    }
+    launch_topk_partial(L, lg, rows, cf.vocab, 1, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
+    launch_topk_merge(L, rows, 1, c->n_chunks, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->b.argmax_tmp,
+                      c->b.top_logp);
+    g = c->b.argmax_tmp;
+  }
+  if (cf.dtype == POSS_BF16)
+    launch_accept_walk<bf16>(L, g, reinterpret_cast<const bf16*>(target_features), cf.hidden, tokens, parents, rows,
+                             POSS_MAX_DEPTH, out_path, out_n_accepted, out_bonus, out_new_tokens,
+                             reinterpret_cast<bf16*>(out_new_features), c->b.counters);
+  else
+    launch_accept_walk<float>(L, g, reinterpret_cast<const float*>(target_features), cf.hidden, tokens, parents, rows,
+                              POSS_MAX_DEPTH, out_path, out_n_accepted, out_bonus, out_new_tokens,
+                              reinterpret_cast<float*>(out_new_features), c->b.counters);
+  return L.err;
+}
+
+int poss_target_forward(poss_ctx* c, void* target_kv, int prefix_len, const int32_t* tokens, const int32_t* depth,
+                        const uint64_t* anc_mask, int rows, void* out_features, int32_t* out_argmax,
+                        float* out_logits, poss_stream stream) {
+  if (!c || !target_kv || !tokens || !depth || !anc_mask || !out_features || prefix_len < 0 || rows < 1)
+    return POSS_E_INVALID;
+  if (c->cfg.n_target_layers < 1) return POSS_E_INVALID;
+  if (rows > R) return POSS_E_CAPACITY;
+  if (prefix_len + rows > c->cfg.target_kv_slots) return POSS_E_CAPACITY;
+  return DISPATCH(c, stream, target_forward(target_kv, prefix_len, tokens, depth, anc_mask, (rows + 63) / 64, rows,
+                                            out_features, out_argmax, out_logits));
+}
+
+int poss_target_prefill(poss_ctx* c, void* target_kv, int start, const int32_t* tokens, int n, void* out_features,
+                        int32_t* out_argmax, poss_stream stream) {
+  if (!c || !target_kv || !tokens || !out_features || start < 0 || n < 0) return POSS_E_INVALID;
+  if (c->cfg.n_target_layers < 1) return POSS_E_INVALID;
+  if (start + n > c->cfg.target_kv_slots) return POSS_E_CAPACITY;
+  int rc = POSS_OK;
+  for (int off = 0; off < n && rc == POSS_OK; off += R) {
+    int m = n - off < R ? n - off : R;
+    char* of = reinterpret_cast<char*>(out_features) + (size_t)off * c->cfg.hidden * c->esize;
+    rc = DISPATCH(c, stream, target_forward(target_kv, start + off, tokens + off, c->b.chain_depth, c->b.chain_mask, 2,
+                                            m, of, out_argmax ? out_argmax + off : nullptr, nullptr));
+  }
+  return rc;
+}
+
+int poss_kv_compact(poss_ctx* c, void* target_kv, int prefix_len, const int32_t* path, const int32_t* n_accepted,
+                    poss_stream stream) {
+  if (!c || !target_kv || !path || !n_accepted || prefix_len < 0) return POSS_E_INVALID;
+  if (c->cfg.n_target_layers < 1) return POSS_E_INVALID;
+  Launcher L; L.stream = S(stream); L.launches = &c->launches; L.err = POSS_OK;
+  const poss_config& g = c->cfg;
+  if (g.dtype == POSS_BF16)
+    launch_kv_compact<bf16>(L, reinterpret_cast<bf16*>(target_kv), g.n_target_layers, g.n_kv_heads, g.target_kv_slots,
+                            g.head_dim, prefix_len, path, n_accepted);
+  else
+    launch_kv_compact<float>(L, reinterpret_cast<float*>(target_kv), g.n_target_layers, g.n_kv_heads,
+                             g.target_kv_slots, g.head_dim, prefix_len, path, n_accepted);
+  return L.err;
+}
+
+int poss_get_counters(poss_ctx* c, int64_t* h_rounds, int64_t* h_accepted_at, poss_stream stream) {
+  if (!c || !h_rounds || !h_accepted_at) return POSS_E_INVALID;
+  unsigned long long tmp[POSS_MAX_DEPTH + 2];
+  if (cudaMemcpyAsync(tmp, c->b.counters, sizeof(tmp), cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess)
+    return POSS_E_CUDA;
+  if (cudaStreamSynchronize(S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  *h_rounds = (int64_t)tmp[0];
+  h_accepted_at[0] = 0;
+  for (int i = 1; i <= c->cfg.max_depth; ++i) h_accepted_at[i] = (int64_t)tmp[i];
+  return POSS_OK;
+}
+
+int poss_last_status(poss_ctx* c, poss_stream stream) {
+  if (!c) return POSS_E_INVALID;
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, c->b.status, 4, cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  if (cudaStreamSynchronize(S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  return v;
+}
+
+int poss_linear(poss_ctx* c, const void* x, int M, const void* w, int N, int K, const void* bias,
+                const float* residual, float* out, int impl, poss_stream stream) {
+  if (!c || !x || !w || !out || M < 0 || N < 1 || K < 1 || impl < 0 || impl > 2) return POSS_E_INVALID;
+  if (M == 0) return POSS_OK;
+  if (M > R) return POSS_E_CAPACITY;
+  if (K % 8) return POSS_E_SHAPE;
+  GemmSegs sg; sg.n = 1; sg.w[0] = w; sg.rows[0] = N;
+  if (c->cfg.dtype == POSS_BF16) {
+    Impl<bf16> im(c, stream);
+    im.gemm(reinterpret_cast<const bf16*>(x), K, M, sg, K, reinterpret_cast<const bf16*>(bias), residual, N, out, N,
+            impl);
+    return im.L.err;
+  }
+  if (impl == 2) return POSS_E_SHAPE;
+  Impl<float> im(c, stream);
+  im.gemm(reinterpret_cast<const float*>(x), K, M, sg, K, reinterpret_cast<const float*>(bias), residual, N, out, N,
+          impl);
+  return im.L.err;
+}
+
+int poss_lm_head_topk(poss_ctx* c, const void* features, int rows, int topk, int32_t* out_ids, float* out_logp,
+                      float* out_logits, poss_stream stream) {
+  if (!c || !features || !out_ids || !out_logp || rows < 0 || topk < 1) return POSS_E_INVALID;
+  if (rows == 0) return POSS_OK;
+  if (rows > R || topk > POSS_MAX_TOPK || topk > c->cfg.vocab) return POSS_E_CAPACITY;
+  if (c->cfg.dtype == POSS_BF16) {
+    Impl<bf16> im(c, stream);
+    im.lm_head_topk(reinterpret_cast<const bf16*>(features), rows, topk, out_ids, out_logp, out_logits);
+    return im.L.err;
+  }
+  Impl<float> im(c, stream);
+  im.lm_head_topk(reinterpret_cast<const float*>(features), rows, topk, out_ids, out_logp, out_logits);
+  return im.L.err;
+}
+
+int64_t poss_launch_count(const poss_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"
