@@ -286,9 +286,12 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
     every specialist; slots from prefix_len on are written here.  new_tokens/new_features are the
     verified pairs not yet in any cache; the last one is the root pair [x_t ; f_{t-1}].
 
-    follow: optional list (one entry per step >= 1) of frontier flat-candidate indices, and
-    follow["top_ids"][i] the [Mc][K] token ids to use for step i's candidates; used to replay
-    another implementation's decisions while computing every value here.
+    follow: replay of another implementation's decisions, every value still computed here:
+    follow["top_ids"][i] the [Mc][K] token ids of step i's candidates, follow["frontier"][i] the flat
+    candidate indices expanded at step i+1, follow["selected"] the rerank's choice.  Optional teacher
+    forcing of values, so that a comparison is per step and rounding noise does not pile up over
+    the depth: follow["features"][i] ([Mc][H]) replaces this step's output features as the input of
+    the children, and follow["cand_scores"] (flat) replaces the parents' cumulative scores.
     """
     S, n, K = cfg.S, cfg.n, topk
     H = cfg.hidden
@@ -354,8 +357,9 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
                 o[r] = masked_attention(q[r:r + 1], Kseq, Vseq, vis1, scale, num)[0]
 
         fout = layer_tail(h0c, num.r(o), lw, cfg, num)
+        forced_f = None if follow is None or "features" not in follow else np.asarray(follow["features"][i], dtype=num.dtype)
         for r, nd in enumerate(current):
-            nd.fout = fout[r]
+            nd.fout = fout[r] if forced_f is None else forced_f[r]
         logits = linear(fout, w["lm_head"], num)
         logp = log_softmax_rows(logits)
         own_ids = topk_rows(logits, K)
@@ -386,8 +390,11 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
             nxt = []
             for jj, c in enumerate(pick):
                 par = cand_node_parent[base + c]
+                sc = cand_score[base + c]
+                if follow is not None and "cand_scores" in follow:
+                    sc = float(follow["cand_scores"][base + int(c)])
                 nxt.append(Node(cand_tok[base + c], par.fout, i + 1, tree_base + i * K + jj,
-                                root_pos + i + 1, par, base + int(c), cand_score[base + c]))
+                                root_pos + i + 1, par, base + int(c), sc))
             levels.append(nxt)
         steps.append(st)
 

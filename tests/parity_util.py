@@ -4,9 +4,12 @@ the same seeded inputs, and compare under the stated rules.
 Rules (written here, used by every parity test):
   * check mode (fp32): structure, tokens and paths bit-exact; features/logits within 1e-4.
   * bf16: features/logits/log-probs within 2e-2; structure bit-exact unless the oracle's margin at the
-    deciding comparison is below 1e-2.  When the free-running oracle and the GPU differ, the oracle is
-    re-run FOLLOWING the GPU's decisions (its own arithmetic on the GPU's tree) and every GPU decision
-    must be valid up to that margin; such decisions are counted and reported.
+    deciding comparison is below 1e-2.  bf16 results of two correct implementations agree only to
+    about one bf16 unit per rounding boundary, and that noise grows with the draft depth, so the
+    numeric comparison is PER STEP WITH TEACHER FORCING: the oracle is re-run following the GPU's
+    decisions and taking the GPU's previous-step features and parent scores as inputs (all arithmetic
+    of the step is the oracle's own).  Every GPU decision must be valid up to the margin under the
+    oracle's values; decisions that differ from the oracle's own choice are counted and reported.
 """
 from __future__ import annotations
 
@@ -89,11 +92,11 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
     free = po.draft_round(cfg, w, kv_o, prefix_len, new_tok, new_feat, depth, K, T, num)
     n = free.n_nodes
     check_structure_self_consistent(g, trace, depth, K, T)
-    exact = (np.array_equal(free.tokens, g["tokens"][:n]) and np.array_equal(free.parents, g["parents"][:n])
+    exact = (len(free.tokens) == n and np.array_equal(free.tokens, g["tokens"][:n]) and np.array_equal(free.parents, g["parents"][:n])
              and np.array_equal(free.depth, g["depth"][:n]) and np.array_equal(free.anc_mask, g["anc_mask"][:n])
              and np.array_equal(free.cand_tok, trace["cand_tokens"]))
     report = {"exact": bool(exact), "inexact_decisions": 0, "min_margin_seen": float("inf")}
-    if exact:
+    if exact and cfg.dtype == "fp32":
         assert np.abs(free.scores - g["scores"][:n]).max() <= tol * max(depth, 1)
         assert np.abs(free.cand_score - trace["cand_scores"]).max() <= tol * max(depth, 1)
         for i, st in enumerate(free.steps):
@@ -114,7 +117,9 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
             base += mc * K
             if i < depth - 1:
                 frontier.append(trace["frontier"][i])
-        follow = {"top_ids": top_ids, "frontier": frontier, "selected": trace["selected"][: n - 1]}
+        follow = {"top_ids": top_ids, "frontier": frontier, "selected": trace["selected"][: n - 1],
+                  "features": [trace["step_features"][i, : (1 if i == 0 else K)] for i in range(depth)],
+                  "cand_scores": trace["cand_scores"]}
         kv_o = po.widen(kv_np, num.dtype).copy()
         fol = po.draft_round(cfg, w, kv_o, prefix_len, new_tok, new_feat, depth, K, T, num, keep_logits=True,
                              follow=follow)
@@ -138,7 +143,9 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
             n_step = mc * K
             sc_o = fol.cand_score[base: base + n_step]
             sc_g = trace["cand_scores"][base: base + n_step]
-            assert np.abs(sc_o - sc_g).max() <= tol * (i + 1), f"step {i} candidate scores"
+            assert np.abs(sc_o - sc_g).max() <= tol, f"step {i} candidate scores (teacher-forced log-probs)"
+            report["max_logp_err"] = max(report.get("max_logp_err", 0.0), float(np.abs(sc_o - sc_g).max()))
+            report["max_feature_err"] = max(report.get("max_feature_err", 0.0), float(err))
             if i < depth - 1:
                 pick = np.asarray(st.next_frontier) - base
                 rest = np.setdiff1d(np.arange(n_step), pick)
@@ -159,7 +166,7 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
             inexact += 1
             report["min_margin_seen"] = min(report["min_margin_seen"], float(own.rerank_margin))
         assert np.array_equal(fol.tokens, g["tokens"][:n]) and np.array_equal(fol.parents, g["parents"][:n])
-        assert np.abs(fol.scores - g["scores"][:n]).max() <= tol * depth
+        assert np.abs(fol.scores - g["scores"][:n]).max() <= tol
         report["inexact_decisions"] = inexact
         assert report["min_margin_seen"] < MARGIN or inexact == 0, \
             f"GPU decision differs although the oracle margin is {report['min_margin_seen']}"

@@ -48,6 +48,34 @@ def test_linear_matches_oracle(name, M, N, K, impl):
         assert np.array_equal(one[0], got2[M - 1])
 
 
+@pytest.mark.parametrize("M,N,K", [
+    (1, 128, 64), (10, 256, 512), (16, 5000, 512), (17, 777, 1024), (57, 4096, 1024), (64, 1408, 2048),
+    (100, 384, 4096), (128, 130, 8192), (3, 640, 328),
+])
+def test_tensor_core_linear_matches_oracle_and_simt(M, N, K):
+    """tcgen05 GEMM: several tiles, ragged N, K tails, split-K, every row-count padding."""
+    cfg = ps.CONFIGS["t_bf16"]
+    w = ps.make_weights(cfg, 1)
+    P = make_poss(cfg, w, 512)
+    num = pu.oracle_num(cfg)
+    x = ps.normal(5, "x", (M, K), 1.0, "bf16")
+    W = ps.normal(5, "w", (N, K), 0.02, "bf16")
+    b = ps.normal(5, "b", (N,), 0.02, "bf16")
+    res = ps.normal(5, "r", (M, N), 1.0, "fp32")
+    got = P.poss_linear(dev(x), dev(W), dev(b), dev(res), impl=2).cpu().numpy()
+    assert P.poss_last_status() == 0
+    want = po.linear(po.widen(x, num.dtype), W, num, b) + res
+    assert np.abs(got - want).max() <= 1e-4
+    simt = P.poss_linear(dev(x), dev(W), dev(b), dev(res), impl=1).cpu().numpy()
+    assert np.abs(got - simt).max() <= 1e-4
+    # deterministic, and a row's value does not depend on the batch around it
+    again = P.poss_linear(dev(x), dev(W), dev(b), dev(res), impl=2).cpu().numpy()
+    assert np.array_equal(got, again)
+    plain = P.poss_linear(dev(x), dev(W), impl=2).cpu().numpy()
+    one = P.poss_linear(dev(x[M - 1:M]), dev(W), impl=2).cpu().numpy()
+    assert np.array_equal(one[0], plain[M - 1])
+
+
 @pytest.mark.parametrize("name,rows,P_len,Hq,Hkv,d", [
     ("t_fp32", 14, 37, 6, 2, 32), ("t_fp32", 1, 0, 4, 4, 64), ("t_fp32", 61, 300, 8, 1, 32),
     ("t_bf16", 25, 300, 8, 2, 64), ("t_bf16", 61, 1024, 32, 8, 128), ("t_bf16", 81, 2100, 8, 8, 128),
