@@ -1,0 +1,276 @@
+"""Benchmark of one PosS speculative round on the Llama-3-8B-shaped drafter workload (config c2).
+
+A step = the whole hot path once: poss_draft_round (6 specialist steps, width 10, 60 kept tokens,
+prefix 1024) + tree-masked verification attention over the 61 tree rows at the target's geometry
++ argmax over target logits and the greedy accept walk.  Weights are random-init, inputs seeded
+and synthetic (poss_synth).  One JSON line on stdout.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c2]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "poss_draft_round_us_60tok_depth6"
+
+
+def algorithmic_bytes(cfg):
+    """Bytes one draft round must move (bf16 weights of every matrix product + the active prefix KV)."""
+    H, F, V = cfg.hidden, cfg.ffn, cfg.vocab
+    qd, kd = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+    per_step = 2 * (2 * H * H + H * (qd + 2 * kd) + qd * H + 3 * H * F + V * H) + 2 * 2 * kd * cfg.prefix
+    return per_step * cfg.depth, 2 * V * H
+
+
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.rows, self.stop, self.index = [], False, index
+        self.t = threading.Thread(target=self.run, daemon=True)
+
+    def run(self):
+        while not self.stop:
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                self.rows.append([c.strip() for c in out.strip().split(",")])
+            except Exception:
+                pass
+            time.sleep(0.1)
+
+    def __enter__(self):
+        self.t.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop = True
+        self.t.join(timeout=6)
+
+    def summary(self):
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        reasons = []
+        for name, col in (("hw_slowdown", 3), ("hw_thermal_slowdown", 4), ("sw_thermal_slowdown", 5), ("sw_power_cap", 6)):
+            if any(len(r) >= 7 and r[col].lower().startswith("active") for r in self.rows):
+                reasons.append(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def run_reference(args, cfg):
+    """The oracle, as it stands, on the host cores: one full draft round per step."""
+    import poss_synth as ps
+    from oracle import poss_oracle as po
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = ps.make_weights(cfg, 1)
+    cap = cfg.prefix + 1 + cfg.tree_slots
+    kv = ps.make_draft_kv(cfg, 1, cap)
+    tok, feat = ps.make_round_inputs(cfg, 1, 1)
+    num = po.Num(np.float32, "bf16")
+    kvw = po.widen(kv, num.dtype)
+    steps, warm = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    for _ in range(warm):
+        po.draft_round(cfg, w, kvw.copy(), cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, num)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        po.draft_round(cfg, w, kvw.copy(), cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, num)
+    dt = (time.perf_counter() - t0) / steps
+    us = dt * 1e6
+    cores = len(os.sched_getaffinity(0))
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: Llama-3-8B-shaped drafter, 6 specialists, depth 6, top-k 10, 60 tokens, prefix 1024"},
+            "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
+                             "sample": "one full draft round (numpy fp32, bf16 rounding contract); verify stages not included"},
+            "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--config", default="c2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    import poss_synth as ps
+    cfg = ps.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2506_03566_b200 import Poss, make_config, to_device
+    from paper_2506_03566_b200 import build as pbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        pbuild.build()
+    if world > 1:
+        dist.barrier()
+    warmup = max(args.warmup, 3)
+
+    # ---------------- inputs: seeded, host-generated, resident in HBM before timing
+    seed = 1 + rank          # replicas only: every rank runs an independent request
+    w = ps.make_weights(cfg, seed)
+    rows = cfg.total + 1
+    cap = cfg.prefix + 8 + cfg.tree_slots
+    P = Poss(make_config(cfg, cap), w)
+    dkv = to_device(ps.make_draft_kv(cfg, seed, cap))
+    tok_h, feat_h = ps.make_round_inputs(cfg, seed, 1)
+    tok_pin = torch.from_numpy(tok_h).pin_memory()
+    feat_pin = torch.from_numpy(feat_h.view(np.int16)).pin_memory()
+    tok_d = tok_pin.cuda()
+    feat_d = feat_pin.cuda().view(torch.bfloat16)
+    # verification side: target-geometry KV with the tree rows' keys behind the prefix, queries, logits
+    tcap = cfg.prefix + rows
+    q_h, tkv_h = ps.make_attention_case(seed, rows, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.prefix, tcap, "bf16")
+    q_d, tkv_d = to_device(q_h), to_device(tkv_h)
+    logits_d = to_device(ps.normal(seed, "target_logits", (rows, cfg.vocab), 1.0, "bf16"))
+    tfeat_d = to_device(ps.normal(seed, "target_features", (rows, cfg.hidden), 1.0, "bf16"))
+    scale = 1.0 / float(np.sqrt(cfg.head_dim))
+    out = P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total)
+    attn_out = torch.empty_like(q_d)
+    del w
+
+    def step(tok, feat):
+        tree = P.poss_draft_round(dkv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, out=out)
+        P.poss_tree_attention(q_d, tkv_d, cfg.prefix, tree["anc_mask"], scale, out=attn_out)
+        return P.poss_verify_accept(logits_d, None, tfeat_d, tree["tokens"], tree["parents"], rows)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step(tok_d, feat_d)
+    sync_all()
+    assert P.poss_last_status() == 0
+
+    # ---------------- timed region 1: inputs resident in HBM
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    P.poss_profile(True)
+    launches0 = P.poss_launch_count()
+    with ClockSampler(local) as clocks:
+        sync_all()
+        ev[0].record()
+        for _ in range(args.steps):
+            step(tok_d, feat_d)
+        ev[1].record()
+        sync_all()
+    ms = ev[0].elapsed_time(ev[1]) / args.steps
+    launches = (P.poss_launch_count() - launches0) // args.steps
+    n_lm, lm_ms = P.poss_profile_read()
+    P.poss_profile(False)
+
+    # draft round alone (the metric's own quantity)
+    sync_all()
+    ev[2].record()
+    for _ in range(args.steps):
+        P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total, out=out)
+    ev[3].record()
+    sync_all()
+    draft_ms = ev[2].elapsed_time(ev[3]) / args.steps
+
+    # ---------------- timed region 2: end to end through the C ABI with host buffers
+    res_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items() if k != "anc_mask"}
+    acc_host = torch.empty(2, dtype=torch.int32).pin_memory()
+    h2d = tok_pin.numel() * 4 + feat_pin.numel() * 2
+    d2h = sum(v.numel() * v.element_size() for v in res_host.values()) + 8
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        tok = tok_pin.cuda(non_blocking=True)
+        feat = feat_pin.cuda(non_blocking=True).view(torch.bfloat16)
+        va = step(tok, feat)
+        for k, v in res_host.items():
+            v.copy_(out[k], non_blocking=True)
+        acc_host[0:1].copy_(va["n_accepted"], non_blocking=True)
+        acc_host[1:2].copy_(va["bonus"], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    sync_all()
+
+    stats = torch.tensor([ms, draft_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+    ms, draft_ms, e2e_ms = [float(x) for x in stats.tolist()]
+
+    if rank == 0:
+        peaks, which = None, "fallback"
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+            which = "measured"
+        except Exception:
+            pass
+        hbm_peak = float(peaks["hbm_gbs"]) if peaks else 6650.0
+        round_bytes, lm_bytes = algorithmic_bytes(cfg)
+        lm_dur = lm_ms / max(n_lm, 1)
+        achieved = lm_bytes / (lm_dur * 1e-3) / 1e9 if n_lm else None
+        line = {
+            "metric": METRIC, "value": draft_ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: Llama-3-8B-shaped drafter, 6 specialists, depth 6, top-k 10, "
+                                   "60 tokens, prefix 1024; step = draft round + 61-row verification attention + accept walk",
+                       "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "stages_us": {"draft_round": draft_ms * 1e3, "whole_step": ms * 1e3,
+                          "verify_attention_plus_accept": max(ms - draft_ms, 0.0) * 1e3},
+            "rounds_per_s": world * 1e3 / ms,
+            "draft_round_gbs": round_bytes / (draft_ms * 1e-3) / 1e9,
+            "draft_round_frac_of_hbm_peak": round_bytes / (draft_ms * 1e-3) / 1e9 / hbm_peak,
+            "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "what": "whole step incl. pinned-host input copy and result read-back, host-timed"},
+            "gpu_launches": int(launches),
+            "clocks": clocks.summary(),
+            "roofline": {"bound": "hbm", "kernel": "k_gemm_tc on the LM head (V x H bf16)", "achieved": achieved,
+                         "peak": hbm_peak, "peak_source": which, "unit": "GB/s",
+                         "frac": achieved / hbm_peak if achieved else None, "traffic": None,
+                         "launches_timed": n_lm, "avg_launch_us": lm_dur * 1e3,
+                         "algorithmic_bytes_per_launch": lm_bytes},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            from oracle import poss_oracle as po
+            wr = ps.make_weights(cfg, seed)
+            kvw = po.widen(ps.make_draft_kv(cfg, seed, cap), np.float32)
+            num = po.Num(np.float32, "bf16")
+            t0 = time.perf_counter()
+            po.draft_round(cfg, wr, kvw, cfg.prefix, tok_h, feat_h, cfg.depth, cfg.topk, cfg.total, num)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": dt * 1e6, "unit": "us", "cores": len(os.sched_getaffinity(0)),
+                                    "kind": "oracle", "sample": "one full draft round of the same workload"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -70,6 +70,8 @@ EXPORTS = {
                               C.c_void_p, C.c_int, C.c_void_p]),
     "poss_lm_head_topk": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]),
+    "poss_profile": (C.c_int, [C.c_void_p, C.c_int]),
+    "poss_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_float)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
 }
 
@@ -301,6 +303,14 @@ class Poss:
         _check(self.lib.poss_lm_head_topk(self.ctx, _ptr(features), rows, topk, _ptr(ids), _ptr(logp), _ptr(logits),
                                           _stream()), "poss_lm_head_topk")
         return ids, logp, logits
+
+    def poss_profile(self, enable: bool):
+        _check(self.lib.poss_profile(self.ctx, int(enable)), "poss_profile")
+
+    def poss_profile_read(self):
+        n, ms = C.c_int(), C.c_float()
+        _check(self.lib.poss_profile_read(self.ctx, C.byref(n), C.byref(ms)), "poss_profile_read")
+        return n.value, ms.value
 
     def poss_launch_count(self) -> int:
         return int(self.lib.poss_launch_count(self.ctx))

@@ -67,7 +67,11 @@ struct poss_ctx {
   int64_t launches;
   int last_depth, last_topk, last_nodes;
   TcGemmPlanCache* tc;
+  bool prof_on;
+  int prof_n;
+  cudaEvent_t* prof_ev;   // 2 * PROF_MAX events, created on first enable
 };
+constexpr int PROF_MAX = 1024;
 
 namespace {
 
@@ -164,7 +168,10 @@ struct Impl {
     const poss_config& g = c->cfg;
     GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = g.vocab;
     float* lg = logits_out ? logits_out : c->b.logits;
+    bool prof = c->prof_on && c->prof_n < PROF_MAX;
+    if (prof) cudaEventRecord(c->prof_ev[2 * c->prof_n], L.stream);
     gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
+    if (prof) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], L.stream); ++c->prof_n; }
     launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
     launch_topk_merge(L, rows, K, c->n_chunks, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp);
   }
@@ -385,6 +392,7 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   if (c->tgt) memcpy(c->tgt, w->h_target, sizeof(poss_layer_w) * cfg->n_target_layers);
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->target_final_norm;
   c->esize = cfg->dtype == POSS_BF16 ? 2 : 4;
+  c->prof_on = false; c->prof_n = 0; c->prof_ev = nullptr;
   c->launches = 0; c->last_depth = 0; c->last_topk = 0; c->last_nodes = 0;
   Bump bp;
   bp.base = reinterpret_cast<char*>(workspace);
@@ -403,6 +411,10 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
 int poss_destroy(poss_ctx* c) {
   if (!c) return POSS_E_INVALID;
   tc_plan_cache_destroy(c->tc);
+  if (c->prof_ev) {
+    for (int i = 0; i < 2 * PROF_MAX; ++i) cudaEventDestroy(c->prof_ev[i]);
+    free(c->prof_ev);
+  }
   free(c->spec);
   free(c->tgt);
   delete c;
@@ -609,6 +621,37 @@ int poss_lm_head_topk(poss_ctx* c, const void* features, int rows, int topk, int
   Impl<float> im(c, stream);
   im.lm_head_topk(reinterpret_cast<const float*>(features), rows, topk, out_ids, out_logp, out_logits);
   return im.L.err;
+}
+
+int poss_profile(poss_ctx* c, int enable) {
+  if (!c) return POSS_E_INVALID;
+  if (enable && !c->prof_ev) {
+    c->prof_ev = (cudaEvent_t*)malloc(sizeof(cudaEvent_t) * 2 * PROF_MAX);
+    if (!c->prof_ev) return POSS_E_INVALID;
+    for (int i = 0; i < 2 * PROF_MAX; ++i)
+      if (cudaEventCreate(&c->prof_ev[i]) != cudaSuccess) return POSS_E_CUDA;
+  }
+  c->prof_on = enable != 0;
+  c->prof_n = 0;
+  return POSS_OK;
+}
+
+int poss_profile_read(poss_ctx* c, int* h_launches, float* h_total_ms) {
+  if (!c || !h_launches || !h_total_ms) return POSS_E_INVALID;
+  *h_launches = 0;
+  *h_total_ms = 0.f;
+  if (!c->prof_ev || c->prof_n == 0) return POSS_OK;
+  if (cudaEventSynchronize(c->prof_ev[2 * c->prof_n - 1]) != cudaSuccess) return POSS_E_CUDA;
+  float total = 0.f;
+  for (int i = 0; i < c->prof_n; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) return POSS_E_CUDA;
+    total += ms;
+  }
+  *h_launches = c->prof_n;
+  *h_total_ms = total;
+  c->prof_n = 0;
+  return POSS_OK;
 }
 
 int64_t poss_launch_count(const poss_ctx* c) { return c ? c->launches : 0; }
