@@ -205,6 +205,26 @@ POSS_API int poss_lm_head_topk(poss_ctx* ctx, const void* features, int rows, in
 POSS_API int poss_profile(poss_ctx* ctx, int enable);
 POSS_API int poss_profile_read(poss_ctx* ctx, int* h_launches, float* h_total_ms);
 
+/* Tree-masked attention for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of poss_tree_attention).
+ * Who needs it: code that is handed device pointers but may not call cudaMalloc -- an engine whose
+ * memory pools were sized once at start-up, a latency-critical stream where an allocation would
+ * force a device-wide synchronisation, a plugin without access to the host application's allocator.
+ * Such callers cannot create the workspace a poss_ctx needs, so this entry takes no context: the
+ * geometry comes as arguments and the split-KV partial results go to a fixed 8 MiB array inside the
+ * library image (resident on every GPU that loads the library until the process exits).
+ * Same semantics and layouts as poss_tree_attention; dtype is POSS_FP32 or POSS_BF16.
+ * Limit: rows * n_q_heads * (head_dim + 2) floats must fit the 8 MiB array (2,097,152 floats),
+ * otherwise POSS_E_CAPACITY; with less room the key range is split fewer ways (never wrongly).
+ * The call allocates nothing and calls no allocating routine.  Its first call on a device looks up
+ * the array's device address (once per device, that device current); make that first call outside
+ * any stream capture.  All calls share the one array and it keeps the previous call's contents:
+ * nothing in it has to start at zero (every value read was written by the same call), but two calls
+ * that overlap on the GPU -- different streams, no ordering -- race on it.  Serialise them. */
+POSS_API int poss_tree_attention_noalloc(const void* q, const void* kv, int kv_slots, int prefix_len,
+                                         int rows, int n_q_heads, int n_kv_heads, int head_dim, int dtype,
+                                         const uint64_t* anc_mask, float scale, void* out, poss_stream stream);
+
 /* Number of kernels this context has launched so far (host counter). */
 POSS_API int64_t poss_launch_count(const poss_ctx* ctx);
 

@@ -73,6 +73,8 @@ EXPORTS = {
     "poss_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_float)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
+    "poss_tree_attention_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                              C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
 }
 
 _lib = None
@@ -314,3 +316,16 @@ class Poss:
 
     def poss_launch_count(self) -> int:
         return int(self.lib.poss_launch_count(self.ctx))
+
+
+def poss_tree_attention_noalloc(q, kv, prefix_len, anc_mask, scale, out):
+    """Context-free tree attention for callers that may not allocate device memory: the caller passes
+    every buffer, `out` included, and the library keeps its partial results in a fixed internal array.
+    q, out [rows][Hq][d]; kv [2][Hkv][slots][d]; anc_mask int64/uint64 [rows][ceil(rows/64)]."""
+    lib = load_library()
+    rows, hq, d = q.shape
+    dtype = POSS_BF16 if q.dtype == torch.bfloat16 else POSS_FP32
+    _check(lib.poss_tree_attention_noalloc(_ptr(q), _ptr(kv), kv.shape[2], prefix_len, rows, hq, kv.shape[1], d,
+                                           dtype, _ptr(anc_mask), float(scale), _ptr(out), _stream()),
+           "poss_tree_attention_noalloc")
+    return out
