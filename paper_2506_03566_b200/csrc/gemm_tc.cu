@@ -1,18 +1,32 @@
 // Skinny bf16 GEMM on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM, operands
-// staged by TMA).
+// staged by TMA): a persistent, warp-specialised, stream-K kernel with fused epilogues.
 //
 // out[m][n] = sum_k X[m][k] * W[n][k]  with M <= 128 activation rows and N large.  The product is
 // evaluated "swapped": a tile of 128 weight rows is the MMA's M dimension (TMEM lane = weight row n),
 // the activation rows are the MMA's N dimension (TMEM column = row m, padded to a multiple of 16).
-// So the weights, which are all of the traffic, stream through shared memory exactly once in 16 KB
-// TMA boxes [128 rows x 64 k] (128-byte swizzle), and the small activation tile rides along.
+// The weights, which are all of the traffic, stream through shared memory exactly once in 16 KB TMA
+// boxes [128 rows x 64 k] (128-byte swizzle); the small activation tile rides along from L2.
 //
-// Grid = (weight-row tiles, K splits).  Roles inside a CTA of 128 threads: warp 0 lane 0 issues TMA
-// into a ring of stages; warp 1 lane 0 issues the MMAs and releases stages with tcgen05.commit; all
-// four warps run the epilogue (tcgen05.ld, 32 TMEM lanes per warp).  With K splits every CTA writes
-// its fp32 partial tile to scratch, and the CTA that arrives last at the tile's counter adds the
-// partials in split order (never in arrival order) and applies bias / residual: the result is
-// deterministic and a row's value does not depend on M.  No CTA ever waits for another CTA.
+// Work split.  The (tile, k-block) pairs of a product form one linear sequence; a fixed grid of CTAs
+// cuts it into equal contiguous ranges ("stream-K"), so every SM streams the same number of bytes
+// whatever the shape.  A range may start or end inside a tile.  A CTA that holds only part of a tile's
+// K range writes its fp32 partial to scratch and bumps the tile's counter; the CTA that arrives last
+// adds the partials in range order (never in arrival order) and runs the epilogue.  No CTA waits for
+// another one, the result is deterministic, and a row's value depends on the weight shape and the
+// grid only, never on M or on the row's place in the batch.
+//
+// Roles inside a CTA of 192 threads: warp 0 lane 0 issues TMA into a ring of stages; warp 1 lane 0
+// issues the MMAs into one of two TMEM accumulators and releases stages with tcgen05.commit; warps
+// 2..5 drain the other accumulator (tcgen05.ld, 32 TMEM lanes per warp) and run the epilogue, so the
+// epilogue of one tile overlaps the weight stream of the next.
+//
+// Epilogues: (0) fp32 store with bias / residual and an optional bf16 copy; (1) SwiGLU: the tile holds
+// 64 gate rows and 64 up rows of the same ffn columns and the epilogue writes bf16(silu(g) * u);
+// (2) LM head: running max / sum-exp / top-k per activation row over the CTA's vocabulary tiles, one
+// partial list per CTA, the logits never reach memory.
+//
+// Programmatic dependent launch: the kernel lets its successor start early and itself prefetches
+// weight tiles (which no kernel writes) before it waits for its predecessor's results.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA raises POSS_E_TIMEOUT in the status word,
 // stops issuing work, drains its own copies (bounded), frees its TMEM and returns.
@@ -21,6 +35,8 @@
 #include <unordered_map>
 #include <string>
 #include <string.h>
+#include <stdlib.h>
+#include <math.h>
 
 #define LAUNCH_CHECK(L)                                         \
   do {                                                          \
@@ -33,23 +49,30 @@ namespace {
 constexpr int TILE_N = 128;          // weight rows per tile (UMMA M)
 constexpr int TILE_K = 64;           // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
-constexpr int MAX_STAGES = 8;
+constexpr int MAX_STAGES = 10;
+constexpr int N_THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr size_t SCRATCH_PARTIAL_BYTES = 96ull << 20;
 constexpr int N_COUNTERS = 8192;
+constexpr int XCH_STRIDE = 17;
 
 struct TcArgs {
-  int M, Npad, n_stages;
+  int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
-  int kb_total, kb_per_split, n_splits;
+  int n_tiles, kb_total, gran;
   const bf16* bias;
   const float* residual;
   int ldr;
   float* out;
   int ldo;
+  bf16* out_bf;
+  int ldo_bf;
   float* scratch;
   int* counters;
   int32_t* status;
+  // LM-head mode
+  int topk, V;
+  float* pmax; float* psum; float* pval; int32_t* pidx;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -60,6 +83,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -84,12 +110,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
                : "memory");
@@ -124,6 +167,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// barrier among the four epilogue warps only
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major tile whose rows are 128 bytes (64 bf16), 128-byte swizzle,
 // 8-row groups 1024 bytes apart; descriptor version 1 (Blackwell), swizzle code 2 in bits 61..63.
@@ -140,18 +185,41 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// ------------------------------------------------------------------ the stream-K range arithmetic
+// Units are k-blocks in (tile, k-block) order.  CTA c owns [range_begin(c), range_begin(c+1)).
+__host__ __device__ __forceinline__ long long range_begin(long long c, long long groups, int G, int gran) {
+  return (c * groups / G) * gran;
+}
+// the CTA whose range contains unit u
+__host__ __device__ __forceinline__ int cta_of_unit(long long u, long long groups, int G, int gran) {
+  long long g = u / gran;                       // group of the unit
+  // largest c with floor(c * groups / G) <= g  <=>  c * groups < (g + 1) * G
+  long long c = ((g + 1) * G + groups - 1) / groups - 1;
+  if (c > G - 1) c = G - 1;
+  return (int)c;
+}
+
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
+
+struct Segment {
+  int tile, kb_begin, kb_end;
+};
+
 // ------------------------------------------------------------------ the kernel
-__global__ void __launch_bounds__(128) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
-                                                 const __grid_constant__ CUtensorMap map_w0,
-                                                 const __grid_constant__ CUtensorMap map_w1,
-                                                 const __grid_constant__ CUtensorMap map_w2, const TcArgs a) {
+__global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
+                                                       const __grid_constant__ CUtensorMap map_w0,
+                                                       const __grid_constant__ CUtensorMap map_w1,
+                                                       const __grid_constant__ CUtensorMap map_w2, const TcArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 1];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
   __shared__ uint32_t tmem_slot;
-  __shared__ int s_abort, s_last;
+  __shared__ int s_abort, s_last, s_epi_ok;
+
+  pdl_launch_dependents();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
   const uint32_t x_tile_bytes = (uint32_t)a.Npad * 128u;
   const uint32_t stage_bytes = W_TILE_BYTES + x_tile_bytes;
   const int S = a.n_stages;
@@ -159,26 +227,29 @@ __global__ void __launch_bounds__(128) k_gemm_tc(const __grid_constant__ CUtenso
   auto x_tile = [&](int s) { return tiles_base + (uint32_t)s * stage_bytes + W_TILE_BYTES; };
   auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
   auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
-  const uint32_t accum_bar = smem_u32(&bars[2 * MAX_STAGES]);
+  auto acc_full = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
+  auto acc_empty = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + 2 + b]); };
+  float* extra = reinterpret_cast<float*>(tiles_ptr + (size_t)S * stage_bytes);   // mode-specific scratch
 
-  // which weight tile
-  int tile = blockIdx.x, seg = 0, ltile = tile;
-  while (seg < a.n_segs - 1 && ltile >= a.seg_tiles[seg]) { ltile -= a.seg_tiles[seg]; ++seg; }
-  const CUtensorMap* map_w = seg == 0 ? &map_w0 : (seg == 1 ? &map_w1 : &map_w2);
-  const int n0 = ltile * TILE_N;
-  const int split = blockIdx.y;
-  const int kb0 = split * a.kb_per_split;
-  const int nkb = min(a.kb_total, kb0 + a.kb_per_split) - kb0;
+  const int G = gridDim.x;
+  const long long groups = (long long)a.n_tiles * a.kb_total / a.gran;
+  const long long u0 = range_begin(blockIdx.x, groups, G, a.gran);
+  const long long u1 = range_begin(blockIdx.x + 1, groups, G, a.gran);
+  const int n_kb = (int)(u1 - u0);
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < a.Npad) tmem_cols <<= 1;
+  while ((int)tmem_cols < 2 * a.Npad) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
     s_last = 0;
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(accum_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    prefetch_tensormap(&map_x);
+    prefetch_tensormap(&map_w0);
+    if (a.n_segs > 1) prefetch_tensormap(&map_w1);
+    if (a.n_segs > 2) prefetch_tensormap(&map_w2);
   }
   if (warp == 1) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
   tc_fence_before();
@@ -187,111 +258,359 @@ __global__ void __launch_bounds__(128) k_gemm_tc(const __grid_constant__ CUtenso
   const uint32_t tmem_base = tmem_slot;
   volatile int* abort_flag = &s_abort;
 
-  if (warp == 0 && lane == 0) {
-    // ---------------- TMA producer
-    int issued = 0;
-    for (int i = 0; i < nkb; ++i) {
-      int s = i % S;
-      if (i >= S && !mbar_wait(empty_bar(s), (uint32_t)((i / S - 1) & 1), abort_flag)) break;
-      mbar_expect_tx(full_bar(s), stage_bytes);
-      int kcoord = (kb0 + i) * TILE_K;
-      tma_load_2d(w_tile(s), map_w, full_bar(s), kcoord, n0);
-      tma_load_2d(x_tile(s), &map_x, full_bar(s), kcoord, 0);
-      issued = i + 1;
-    }
-    if (*abort_flag) {
-      // drain: every copy this thread started must land before the CTA's shared memory goes away
-      for (int i = max(0, issued - S); i < issued; ++i) {
-        uint32_t bar = full_bar(i % S), par = (uint32_t)((i / S) & 1);
-        for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try_wait(bar, par); ++it) __nanosleep(64);
+  // which weight map / first row a tile starts at
+  auto tile_seg = [&](int tile, int* ltile) {
+    int seg = 0, lt = tile;
+    while (seg < a.n_segs - 1 && lt >= a.seg_tiles[seg]) { lt -= a.seg_tiles[seg]; ++seg; }
+    *ltile = lt;
+    return seg;
+  };
+
+  if (warp == 0) {
+    if (lane == 0 && n_kb > 0) {
+      // ---------------- TMA producer
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      // position of the next k-block to load, advanced without divisions
+      struct Cursor { int tile, kb, seg, lt; };
+      auto cursor_at = [&](long long u) {
+        Cursor c;
+        c.tile = (int)(u / a.kb_total);
+        c.kb = (int)(u - (long long)c.tile * a.kb_total);
+        c.seg = tile_seg(c.tile, &c.lt);
+        return c;
+      };
+      auto advance = [&](Cursor& c) {
+        if (++c.kb == a.kb_total) {
+          c.kb = 0;
+          ++c.tile;
+          if (++c.lt == a.seg_tiles[c.seg] && c.seg < a.n_segs - 1) { c.lt = 0; ++c.seg; }
+        }
+      };
+      auto load_w = [&](const Cursor& c, int s) {
+        int kcoord = c.kb * TILE_K;
+        if (a.mode == 1) {           // 64 gate rows + 64 up rows of the same ffn columns
+          tma_load_2d(w_tile(s), &map_w0, full_bar(s), kcoord, c.tile * 64, pol_w);
+          tma_load_2d(w_tile(s) + W_TILE_BYTES / 2, &map_w1, full_bar(s), kcoord, c.tile * 64, pol_w);
+        } else {
+          const CUtensorMap* mw = c.seg == 0 ? &map_w0 : (c.seg == 1 ? &map_w1 : &map_w2);
+          tma_load_2d(w_tile(s), mw, full_bar(s), kcoord, c.lt * TILE_N, pol_w);
+        }
+      };
+      auto load_x = [&](const Cursor& c, int s) {
+        tma_load_2d(x_tile(s), &map_x, full_bar(s), c.kb * TILE_K, 0, pol_x);
+      };
+      // weights are never written by a kernel: fill the ring with them before waiting for the
+      // predecessor, whose results are the activations
+      const int pre = n_kb < S ? n_kb : S;
+      Cursor cw = cursor_at(u0), cx = cw;
+      for (int it = 0; it < pre; ++it) {
+        mbar_expect_tx(full_bar(it), stage_bytes);
+        load_w(cw, it);
+        advance(cw);
+      }
+      pdl_wait();
+      for (int it = 0; it < pre; ++it) { load_x(cx, it); advance(cx); }
+      int issued = pre, s = 0;
+      uint32_t phase = 0;                     // parity of the "empty" completion that frees stage s next
+      for (int it = pre; it < n_kb; ++it) {
+        if (!mbar_wait(empty_bar(s), phase, abort_flag)) break;
+        mbar_expect_tx(full_bar(s), stage_bytes);
+        load_w(cw, s);
+        load_x(cw, s);
+        advance(cw);
+        issued = it + 1;
+        if (++s == S) { s = 0; phase ^= 1u; }
+      }
+      if (*abort_flag) {
+        // drain: every copy this thread started must land before the CTA's shared memory goes away
+        for (int it = max(0, issued - S); it < issued; ++it) {
+          uint32_t bar = full_bar(it % S), par = (uint32_t)((it / S) & 1);
+          for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(bar, par); ++w) __nanosleep(64);
+        }
       }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ---------------- MMA issuer
-    const uint32_t idesc = instr_desc_bf16(TILE_N, a.Npad);
+  } else if (warp == 1) {
+    if (lane == 0 && n_kb > 0) {
+      // ---------------- MMA issuer
+      const uint32_t idesc = instr_desc_bf16(TILE_N, a.Npad);
+      bool ok = true;
+      int it = 0, seg_i = 0, s = 0;
+      uint32_t phase = 0;
+      int kb_begin = (int)(u0 % a.kb_total);
+      while (it < n_kb && ok) {
+        int len = min(a.kb_total - kb_begin, n_kb - it);
+        kb_begin = 0;                          // every later segment starts a tile
+        int buf = seg_i & 1, use = seg_i >> 1;
+        if (use > 0) ok = mbar_wait(acc_empty(buf), (uint32_t)((use - 1) & 1), abort_flag);
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * a.Npad);
+        for (int i = 0; i < len && ok; ++i, ++it) {
+          ok = mbar_wait(full_bar(s), phase, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          uint64_t ad = smem_desc_sw128(w_tile(s)), bd = smem_desc_sw128(x_tile(s));
+#pragma unroll
+          for (int kk = 0; kk < TILE_K / 16; ++kk)      // 16 bf16 = 32 bytes = 2 descriptor address units
+            umma_bf16(tmem_d, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(empty_bar(s));
+          if (++s == S) { s = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(acc_full(buf));     // arrives once every MMA of this segment has finished
+        ++seg_i;
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: TMEM lane = weight row
+    pdl_wait();
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int t = q * 32 + lane;                  // row inside the tile
+    const int K = a.topk;
+    // LM-head running state of this warp: max, sum-exp and a best-first list per activation row
+    float* st_max = extra + (size_t)q * a.M;
+    float* st_sum = extra + (size_t)(4 + q) * a.M;
+    float* lst_val = extra + (size_t)8 * a.M + (size_t)q * a.M * K;
+    int* lst_idx = reinterpret_cast<int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K) + (size_t)q * a.M * K;
+    if (a.mode == 2) {
+      for (int m = lane; m < a.M; m += 32) { st_max[m] = -INFINITY; st_sum[m] = 0.f; }
+      for (int i = lane; i < a.M * K; i += 32) { lst_val[i] = -INFINITY; lst_idx[i] = 0x7fffffff; }
+      __syncwarp();
+    }
     bool ok = true;
-    for (int i = 0; i < nkb && ok; ++i) {
-      int s = i % S;
-      ok = mbar_wait(full_bar(s), (uint32_t)((i / S) & 1), abort_flag);
+    int it = 0, seg_i = 0;
+    while (it < n_kb && ok) {
+      long long u = u0 + it;
+      const int tile = (int)(u / a.kb_total);
+      const int kb_begin = (int)(u % a.kb_total);
+      const int len = min(a.kb_total - kb_begin, n_kb - it);
+      const bool whole = len == a.kb_total;
+      const int buf = seg_i & 1, use = seg_i >> 1;
+      mbar_wait(acc_full(buf), (uint32_t)(use & 1), abort_flag);
+      // one verdict for all four warps (their barriers below must stay matched)
+      epi_sync();
+      if (threadIdx.x == 64) s_epi_ok = *abort_flag == 0;
+      epi_sync();
+      ok = s_epi_ok != 0;
       if (!ok) break;
       tc_fence_after();
-      uint64_t ad = smem_desc_sw128(w_tile(s)), bd = smem_desc_sw128(x_tile(s));
-#pragma unroll
-      for (int kk = 0; kk < TILE_K / 16; ++kk)      // 16 bf16 = 32 bytes = 2 descriptor address units
-        umma_bf16(tmem_base, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (i > 0 || kk > 0) ? 1u : 0u);
-      umma_commit(empty_bar(s));
-    }
-    umma_commit(accum_bar);        // arrives once every MMA issued above has finished
-  }
-  __syncwarp();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.Npad);
 
-  // ---------------- epilogue: all four warps, TMEM lane = weight row
-  bool have = mbar_wait(accum_bar, 0u, abort_flag);
-  have = have && !*abort_flag;
-  tc_fence_after();
-  const int t = threadIdx.x;
-  const int n_local = n0 + t;
-  const bool n_ok = n_local < a.seg_rows[seg];
-  const int col = a.seg_col[seg] + n_local;
-  const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
-  if (have) {
-    if (a.n_splits == 1) {
-      float bv = (a.bias && n_ok) ? __bfloat162float(a.bias[col]) : 0.f;
-      for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
-        float v[16];
-        tmem_ld16(taddr + (uint32_t)c0, v);
+      // where this thread's row lands
+      int lt, seg = 0, col, n_local;
+      bool n_ok;
+      if (a.mode == 1) {
+        n_local = tile * 64 + (t & 63);
+        n_ok = n_local < a.seg_rows[0];
+        col = n_local;
+        lt = tile;
+      } else {
+        seg = tile_seg(tile, &lt);
+        n_local = lt * TILE_N + t;
+        n_ok = n_local < a.seg_rows[seg];
+        col = a.seg_col[seg] + n_local;
+      }
+
+      // ---- epilogue of one 16-column chunk held in v[]
+      auto epilogue_chunk = [&](int c0, float* v) {
+        if (a.mode == 0) {
+          float bv = (a.bias && n_ok) ? __bfloat162float(a.bias[col]) : 0.f;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          int m = c0 + j;
-          if (m < a.M && n_ok) {
-            float r = v[j] + bv;
-            if (a.residual) r += a.residual[(size_t)m * a.ldr + col];
-            a.out[(size_t)m * a.ldo + col] = r;
+          for (int j = 0; j < 16; ++j) {
+            int m = c0 + j;
+            if (m < a.M && n_ok) {
+              float r = v[j] + bv;
+              if (a.residual) r += a.residual[(size_t)m * a.ldr + col];
+              if (a.out) a.out[(size_t)m * a.ldo + col] = r;
+              if (a.out_bf) a.out_bf[(size_t)m * a.ldo_bf + col] = __float2bfloat16_rn(r);
+            }
+          }
+        } else if (a.mode == 1) {
+          float* xch = extra;                     // [64][XCH_STRIDE]
+          if (t >= 64) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) xch[(t - 64) * XCH_STRIDE + j] = v[j];
+          }
+          epi_sync();
+          if (t < 64) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              int m = c0 + j;
+              if (m < a.M && n_ok) {
+                float g = v[j], up = xch[t * XCH_STRIDE + j];
+                float s = g / (1.f + expf(-g));
+                a.out_bf[(size_t)m * a.ldo_bf + col] = __float2bfloat16_rn(s * up);
+              }
+            }
+          }
+          epi_sync();
+        } else {
+          const int n_glob = n_local;             // vocabulary id of this lane's row
+          for (int j = 0; j < 16; ++j) {
+            int m = c0 + j;
+            if (m >= a.M) break;
+            float val = n_ok ? v[j] : -INFINITY;
+            // running log-sum-exp
+            float tmax = val;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+            float omax = st_max[m];
+            float nmax = fmaxf(omax, tmax);
+            float p = n_ok ? expf(val - nmax) : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
+            // running top-k: lanes 0..K-1 hold the list, best first
+            float lv = lane < K ? lst_val[m * K + lane] : -INFINITY;
+            int li = lane < K ? lst_idx[m * K + lane] : 0x7fffffff;
+            float thr = __shfl_sync(0xffffffffu, lv, K - 1);
+            unsigned cand = __ballot_sync(0xffffffffu, val > thr);
+            bool changed = false;
+            while (cand) {
+              int src = __ffs(cand) - 1;
+              cand &= cand - 1;
+              float x = __shfl_sync(0xffffffffu, val, src);
+              int xi = n_glob - lane + src;
+              if (!(x > thr)) continue;
+              unsigned ahead = __ballot_sync(0xffffffffu, lane < K && better(lv, li, x, xi));
+              int pos = __popc(ahead);
+              float pv = __shfl_up_sync(0xffffffffu, lv, 1);
+              int pi = __shfl_up_sync(0xffffffffu, li, 1);
+              if (lane == pos) { lv = x; li = xi; }
+              else if (lane > pos) { lv = pv; li = pi; }
+              thr = __shfl_sync(0xffffffffu, lv, K - 1);
+              changed = true;
+            }
+            __syncwarp();
+            if (lane == 0 && tmax > -INFINITY) {
+              st_sum[m] = st_sum[m] * expf(omax - nmax) + p;
+              st_max[m] = nmax;
+            }
+            if (changed && lane < K) { lst_val[m * K + lane] = lv; lst_idx[m * K + lane] = li; }
+            __syncwarp();
           }
         }
-      }
-    } else {
-      float* part = a.scratch + ((size_t)tile * a.n_splits + split) * (size_t)a.Npad * TILE_N;
-      for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
-        float v[16];
-        tmem_ld16(taddr + (uint32_t)c0, v);
+      };
+
+      if (whole) {
+        for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + (uint32_t)c0, v);
+          if (c0 + 16 >= a.Npad || c0 + 16 >= a.M) {    // last read of this accumulator: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(buf));
+          }
+          epilogue_chunk(c0, v);
+        }
+      } else {
+        // partial K range: park the fp32 partial, the last arriver of the tile finishes it
+        const long long tile_u0 = (long long)tile * a.kb_total;
+        const int c_first = cta_of_unit(tile_u0, groups, G, a.gran);
+        const int c_last = cta_of_unit(tile_u0 + a.kb_total - 1, groups, G, a.gran);
+        const int slot = (u == u0) ? 0 : 1;       // a range's first segment, or its trailing one
+        const size_t part_elems = (size_t)a.Npad * TILE_N;
+        float* part = a.scratch + ((size_t)blockIdx.x * 2 + slot) * part_elems;
+        for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + (uint32_t)c0, v);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          int m = c0 + j;
-          if (m < a.M) part[(size_t)m * TILE_N + t] = v[j];
+          for (int j = 0; j < 16; ++j) {
+            int m = c0 + j;
+            if (m < a.M) part[(size_t)m * TILE_N + t] = v[j];
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty(buf));
+        __threadfence();
+        epi_sync();
+        if (threadIdx.x == 64) {
+          int prev = atomicAdd(&a.counters[tile], 1);
+          s_last = prev == (c_last - c_first);
+        }
+        epi_sync();
+        const bool last = s_last != 0;
+        epi_sync();                                // s_last is rewritten by the next partial segment
+        if (last) {
+          __threadfence();
+          for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = 0.f;
+            for (int c = c_first; c <= c_last; c += 2) {
+              // contributor c: its range begins inside this tile (slot 0) unless it is the first
+              // contributor and began earlier (then this tile is its trailing segment, slot 1)
+              const bool two = c + 1 <= c_last;
+              long long b0 = range_begin(c, groups, G, a.gran);
+              int s0 = (b0 >= tile_u0) ? 0 : 1;
+              const float* p0 = a.scratch + ((size_t)c * 2 + s0) * part_elems + t;
+              const float* p1 = a.scratch + ((size_t)(c + 1) * 2) * part_elems + t;   // a later contributor: slot 0
+              float x0[16], x1[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                int m = c0 + j;
+                x0[j] = m < a.M ? __ldcg(p0 + (size_t)m * TILE_N) : 0.f;
+                x1[j] = (two && m < a.M) ? __ldcg(p1 + (size_t)m * TILE_N) : 0.f;
+              }
+#pragma unroll
+              for (int j = 0; j < 16; ++j) { v[j] += x0[j]; if (two) v[j] += x1[j]; }
+            }
+            epilogue_chunk(c0, v);
+          }
+          if (threadIdx.x == 64) a.counters[tile] = 0;     // ready for the next launch on this stream
         }
       }
-      __threadfence();
+      it += len;
+      ++seg_i;
+    }
+
+    if (a.mode == 2) {
+      // ---- merge the four warps' running states into this CTA's list (columns dealt round-robin)
+      epi_sync();
+      const float* all_max = extra;
+      const float* all_sum = extra + (size_t)4 * a.M;
+      const float* all_val = extra + (size_t)8 * a.M;
+      const int* all_idx = reinterpret_cast<const int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K);
+      for (int m = q; m < a.M; m += 4) {
+        float mx = -INFINITY;
+        for (int w = 0; w < 4; ++w) mx = fmaxf(mx, all_max[w * a.M + m]);
+        float sm = 0.f;
+        for (int w = 0; w < 4; ++w) {
+          float wm = all_max[w * a.M + m];
+          if (wm > -INFINITY) sm += all_sum[w * a.M + m] * expf(wm - mx);
+        }
+        // K rounds: take the best head among the four best-first lists
+        int head = 0;                              // lane w < 4 tracks list w's head
+        size_t o = ((size_t)m * gridDim.x + blockIdx.x);
+        for (int k = 0; k < K; ++k) {
+          float hv = -INFINITY;
+          int hi = 0x7fffffff;
+          if (lane < 4 && head < K) {
+            hv = all_val[((size_t)lane * a.M + m) * K + head];
+            hi = all_idx[((size_t)lane * a.M + m) * K + head];
+          }
+          float bv = hv;
+          int bi = hi, bw = lane;
+#pragma unroll
+          for (int off = 2; off > 0; off >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            int ow = __shfl_xor_sync(0xffffffffu, bw, off);
+            if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bw = ow; }
+          }
+          bv = __shfl_sync(0xffffffffu, bv, 0);
+          bi = __shfl_sync(0xffffffffu, bi, 0);
+          bw = __shfl_sync(0xffffffffu, bw, 0);
+          if (lane == bw && bi != 0x7fffffff) ++head;
+          if (lane == 0) { a.pval[o * K + k] = bv; a.pidx[o * K + k] = bi; }
+        }
+        if (lane == 0) { a.pmax[o] = mx; a.psum[o] = sm; }
+      }
     }
   }
+
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
   if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, (int)POSS_E_TIMEOUT);
-
-  if (a.n_splits > 1 && !*abort_flag) {
-    if (threadIdx.x == 0) {
-      int prev = atomicAdd(&a.counters[tile], 1);
-      s_last = prev == a.n_splits - 1;
-    }
-    __syncthreads();
-    if (s_last) {
-      __threadfence();
-      const float* p0 = a.scratch + (size_t)tile * a.n_splits * (size_t)a.Npad * TILE_N;
-      float bv = (a.bias && n_ok) ? __bfloat162float(a.bias[col]) : 0.f;
-      for (int m = 0; m < a.M; ++m) {
-        float acc = 0.f;
-        for (int sp = 0; sp < a.n_splits; ++sp)
-          acc += __ldcg(p0 + ((size_t)sp * a.Npad + m) * TILE_N + t);
-        if (n_ok) {
-          float r = acc + bv;
-          if (a.residual) r += a.residual[(size_t)m * a.ldr + col];
-          a.out[(size_t)m * a.ldo + col] = r;
-        }
-      }
-      if (threadIdx.x == 0) a.counters[tile] = 0;     // ready for the next launch on this stream
-    }
-  }
 }
 
 // ------------------------------------------------------------------ host side
@@ -319,10 +638,25 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
+  int grid = 0, stages = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
-TcGemmPlanCache* tc_plan_cache_create() { return new TcGemmPlanCache(); }
+TcGemmPlanCache* tc_plan_cache_create() {
+  TcGemmPlanCache* c = new TcGemmPlanCache();
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (sms < 1) sms = 148;
+  // The grid is a property of the device, not of a call: the work split (and with it the order in
+  // which a tile's partial sums are added) must not change from call to call.
+  int per_sm = 1;
+  if (const char* e = getenv("POSS_TC_CTAS_PER_SM")) { int v = atoi(e); if (v >= 1 && v <= 2) per_sm = v; }
+  c->grid = sms * per_sm;
+  if (c->grid > TC_MAX_GRID) c->grid = TC_MAX_GRID;
+  c->stages = 0;
+  if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
+  return c;
+}
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
 size_t tc_gemm_scratch_bytes() { return SCRATCH_PARTIAL_BYTES + N_COUNTERS * sizeof(int); }
 
@@ -367,68 +701,76 @@ bool get_map(TcGemmPlanCache* c, const void* p, int rows, int cols, int ld, int 
 
 }  // namespace
 
-// Split factor and stage count depend on the weight shape only, never on M.
-void tc_plan_splits(int n_tiles, int kb_total, int* n_splits, int* kb_per_split) {
-  int target = 2 * 148;
-  int want = (target + n_tiles - 1) / n_tiles;
-  int max_by_k = kb_total / 4;
-  if (max_by_k < 1) max_by_k = 1;
-  if (want > max_by_k) want = max_by_k;
-  if (want < 1) want = 1;
-  int per = (kb_total + want - 1) / want;
-  *kb_per_split = per;
-  *n_splits = (kb_total + per - 1) / per;
-}
-
 void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx, int M, const GemmSegs& segs, int K,
-                    const bf16* bias, const float* residual, int ldr, float* out, int ldo, void* scratch,
-                    int32_t* status) {
+                    const TcEpilogue& ep, void* scratch, int32_t* status) {
   TcArgs a;
   memset(&a, 0, sizeof(a));
   a.M = M;
   a.Npad = (M + 15) / 16 * 16;
+  a.mode = ep.mode;
   a.n_segs = segs.n;
+  const int tile_rows = ep.mode == TC_EPI_SWIGLU ? 64 : TILE_N;
   int n_tiles = 0, col = 0;
   for (int i = 0; i < segs.n; ++i) {
-    a.seg_tiles[i] = (segs.rows[i] + TILE_N - 1) / TILE_N;
+    a.seg_tiles[i] = (segs.rows[i] + tile_rows - 1) / tile_rows;
     a.seg_rows[i] = segs.rows[i];
     a.seg_col[i] = col;
     col += segs.rows[i];
     n_tiles += a.seg_tiles[i];
   }
+  if (ep.mode == TC_EPI_SWIGLU) n_tiles = a.seg_tiles[0];   // one tile = 64 gate + 64 up rows
+  a.n_tiles = n_tiles;
   a.kb_total = (K + TILE_K - 1) / TILE_K;
-  tc_plan_splits(n_tiles, a.kb_total, &a.n_splits, &a.kb_per_split);
-  size_t part_bytes = (size_t)n_tiles * a.n_splits * a.Npad * TILE_N * sizeof(float);
-  if (a.n_splits > 1 && (part_bytes > SCRATCH_PARTIAL_BYTES || n_tiles > N_COUNTERS)) {
-    a.n_splits = 1;
-    a.kb_per_split = a.kb_total;
-  }
+  // whole tiles per CTA for the LM head (its epilogue keeps running state across tiles), and whenever
+  // the partial buffers or the tile counters could not hold the split
+  size_t part_bytes = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
+  bool no_split = ep.mode == TC_EPI_TOPK || part_bytes > SCRATCH_PARTIAL_BYTES || n_tiles > N_COUNTERS;
+  a.gran = no_split ? a.kb_total : 1;
+  // never more CTAs than ranges to hand out: every CTA of the grid owns at least one k-block
+  long long groups = (long long)n_tiles * a.kb_total / a.gran;
+  const int G = (long long)cache->grid < groups ? cache->grid : (int)groups;
+  if (ep.n_lists) *ep.n_lists = G;
   uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
-  int stages = (int)((100u * 1024u) / stage_bytes);
+  size_t extra = 0;
+  if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
+  if (ep.mode == TC_EPI_TOPK) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
+  int stages = cache->stages ? cache->stages : (int)((108u * 1024u - extra) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
-  if (stages > a.kb_per_split) stages = a.kb_per_split;
-  if (stages < 2) stages = a.kb_per_split < 2 ? 1 : 2;
+  if (stages < 2) stages = 2;
   a.n_stages = stages;
-  a.bias = bias; a.residual = residual; a.ldr = ldr; a.out = out; a.ldo = ldo;
+  a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
+  a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);
   a.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + SCRATCH_PARTIAL_BYTES);
   a.status = status;
+  a.topk = ep.topk; a.V = segs.rows[0];
+  a.pmax = ep.pmax; a.psum = ep.psum; a.pval = ep.pval; a.pidx = ep.pidx;
 
   CUtensorMap mx, mw[3];
   if (!get_map(cache, X, M, K, ldx, a.Npad, false, &mx)) { L.err = POSS_E_CUDA; return; }
   for (int i = 0; i < 3; ++i) {
     int j = i < segs.n ? i : 0;
-    if (!get_map(cache, segs.w[j], segs.rows[j], K, K, TILE_N, true, &mw[i])) { L.err = POSS_E_CUDA; return; }
+    if (!get_map(cache, segs.w[j], segs.rows[j], K, K, tile_rows, true, &mw[i])) { L.err = POSS_E_CUDA; return; }
   }
-  size_t smem = (size_t)stages * stage_bytes + 1024;
+  size_t smem = (size_t)stages * stage_bytes + extra + 1024;
   if (!cache->attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
     cache->attr_set = true;
   }
-  dim3 grid(n_tiles, a.n_splits);
-  k_gemm_tc<<<grid, 128, smem, L.stream>>>(mx, mw[0], mw[1], mw[2], a);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(G);
+  cfg.blockDim = dim3(N_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, mx, mw[0], mw[1], mw[2], a) != cudaSuccess) L.err = POSS_E_CUDA;
   LAUNCH_CHECK(L);
 }

@@ -6,8 +6,36 @@ struct TcGemmPlanCache;
 TcGemmPlanCache* tc_plan_cache_create();
 void tc_plan_cache_destroy(TcGemmPlanCache*);
 size_t tc_gemm_scratch_bytes();
-// true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 64, ...)
+// true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 8, ...)
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);
+
+constexpr int TC_MAX_GRID = 512;     // upper bound of the persistent grid = of the LM-head partial lists per row
+
+enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_TOPK = 2 };
+
+// What happens to the accumulators.
+//   TC_EPI_STORE : out[m][n] (fp32, may be NULL) = acc + bias[n] + residual[m][n]; out_bf (may be NULL) gets the
+//                  same value rounded to bf16.
+//   TC_EPI_SWIGLU: segs = {gate, up} with equal row counts F; out_bf[m][f] = bf16(silu(gate_f . x_m) * (up_f . x_m)).
+//   TC_EPI_TOPK  : segs = {lm_head}; every CTA leaves, per activation row, the max, the sum of exp(logit - max) and
+//                  the topk best (logit, id) pairs of its vocabulary tiles, best first:
+//                  pmax/psum [M][n_lists], pval/pidx [M][n_lists][topk]; *n_lists receives the list count.
+struct TcEpilogue {
+  int mode = TC_EPI_STORE;
+  const bf16* bias = nullptr;
+  const float* residual = nullptr;
+  int ldr = 0;
+  float* out = nullptr;
+  int ldo = 0;
+  bf16* out_bf = nullptr;
+  int ldo_bf = 0;
+  int topk = 0;
+  float* pmax = nullptr;
+  float* psum = nullptr;
+  float* pval = nullptr;
+  int32_t* pidx = nullptr;
+  int* n_lists = nullptr;
+};
+
 void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx, int M, const GemmSegs& segs, int K,
-                    const bf16* bias, const float* residual, int ldr, float* out, int ldo, void* scratch,
-                    int32_t* status);
+                    const TcEpilogue& ep, void* scratch, int32_t* status);

@@ -53,7 +53,7 @@ extern "C" POSS_API int poss_tree_attention_noalloc(const void* q, const void* k
   size_t per_split = attn_partial_floats(rows, n_q_heads, head_dim, 1);
   if (per_split > NOALLOC_SCRATCH_FLOATS) return POSS_E_CAPACITY;
   int max_splits = (int)(NOALLOC_SCRATCH_FLOATS / per_split);
-  if (max_splits > 16) max_splits = 16;
+  if (max_splits > 32) max_splits = 32;
 
   float* scratch = nullptr;
   int rc = scratch_for_current_device(&scratch);
@@ -62,7 +62,6 @@ extern "C" POSS_API int poss_tree_attention_noalloc(const void* q, const void* k
   AttnArgs a;
   a.rows = rows; a.Hq = n_q_heads; a.Hkv = n_kv_heads; a.d = head_dim; a.cap = kv_slots;
   a.n_all = prefix_len; a.n_tree = rows; a.mask = anc_mask; a.mask_words = (rows + 63) / 64; a.scale = scale;
-  plan_attention_splits(rows, n_kv_heads, prefix_len + rows, max_splits, &a.n_splits, &a.keys_per_split);
   Launcher L;
   L.stream = reinterpret_cast<cudaStream_t>(stream);
   L.launches = &g_launches;
@@ -72,12 +71,12 @@ extern "C" POSS_API int poss_tree_attention_noalloc(const void* q, const void* k
   // written by this call's first kernel, so the previous call's leftovers are never seen.
   if (dtype == POSS_BF16) {
     const bf16* kc = reinterpret_cast<const bf16*>(kv);
-    launch_tree_attention<bf16>(L, a, reinterpret_cast<const bf16*>(q), kc, kc + half, scratch,
-                                reinterpret_cast<bf16*>(out));
+    run_tree_attention<bf16>(L, a, max_splits, reinterpret_cast<const bf16*>(q), kc, kc + half, scratch,
+                             reinterpret_cast<bf16*>(out));
   } else {
     const float* kc = reinterpret_cast<const float*>(kv);
-    launch_tree_attention<float>(L, a, reinterpret_cast<const float*>(q), kc, kc + half, scratch,
-                                 reinterpret_cast<float*>(out));
+    run_tree_attention<float>(L, a, max_splits, reinterpret_cast<const float*>(q), kc, kc + half, scratch,
+                              reinterpret_cast<float*>(out));
   }
   return L.err;
 }

@@ -11,7 +11,7 @@ namespace {
 
 constexpr int R = POSS_MAX_ROWS;
 constexpr int KMAX = POSS_MAX_TOPK;
-constexpr int ATTN_MAX_SPLITS = 16;
+constexpr int ATTN_MAX_SPLITS = 32;
 
 struct Bump {
   size_t off = 0;
@@ -125,10 +125,11 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.hx = bp.take<float>(R * H, 4);
   b.tfeat = bp.take<float>(R * H, 4);
   b.logits = bp.take<float>(R * V, 4);
-  b.pmax = bp.take<float>((size_t)R * *n_chunks, 4);
-  b.psum = bp.take<float>((size_t)R * *n_chunks, 4);
-  b.pval = bp.take<float>((size_t)R * *n_chunks * KMAX, 4);
-  b.pidx = bp.take<int32_t>((size_t)R * *n_chunks * KMAX, 4);
+  size_t n_lists = *n_chunks > TC_MAX_GRID ? *n_chunks : TC_MAX_GRID;   // chunk lists or one list per GEMM CTA
+  b.pmax = bp.take<float>((size_t)R * n_lists, 4);
+  b.psum = bp.take<float>((size_t)R * n_lists, 4);
+  b.pval = bp.take<float>((size_t)R * n_lists * KMAX, 4);
+  b.pidx = bp.take<int32_t>((size_t)R * n_lists * KMAX, 4);
   b.top_ids = bp.take<int32_t>(R * KMAX, 4);
   b.top_logp = bp.take<float>(R * KMAX, 4);
   b.chain_mask = bp.take<uint64_t>(R * 2, 8);
@@ -161,8 +162,13 @@ struct Impl {
   T* A(void* p) const { return reinterpret_cast<T*>(p); }
 
   // out[M][N] = x . segs^T (+bias) (+residual); picks the tensor-core kernel when it applies
+  // out_act (optional, [M][ldo]) receives the same values in the context dtype
   void gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual, int ldr,
-            float* out, int ldo, int impl = 0);
+            float* out, int ldo, int impl = 0, T* out_act = nullptr);
+  // act[M][F] = T(silu(x . gate^T) * (x . up^T))
+  void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
+  // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
+  bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists);
 
   void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out) {
     const poss_config& g = c->cfg;
@@ -170,10 +176,15 @@ struct Impl {
     float* lg = logits_out ? logits_out : c->b.logits;
     bool prof = c->prof_on && c->prof_n < PROF_MAX;
     if (prof) cudaEventRecord(c->prof_ev[2 * c->prof_n], L.stream);
-    gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
+    int n_lists = 0;
+    bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists);
+    if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
     if (prof) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], L.stream); ++c->prof_n; }
-    launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
-    launch_topk_merge(L, rows, K, c->n_chunks, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp);
+    if (!fused) {
+      launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
+      n_lists = c->n_chunks;
+    }
+    launch_topk_merge(L, rows, K, n_lists, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp);
   }
 
   // fc + norm + K/V(+Q) projection + rotary + cache append for one batch of a specialist
@@ -196,18 +207,16 @@ struct Impl {
   }
 
   // attention output -> O-proj + residual -> MLP + residual; x0 = layer input rows, result in `out`
-  void layer_tail(const poss_layer_w& lw, const float* x0, int rows, float* out) {
+  void layer_tail(const poss_layer_w& lw, const float* x0, int rows, float* out, T* out_act = nullptr) {
     const poss_config& g = c->cfg;
     Buffers& b = c->b;
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, F = g.ffn;
     GemmSegs so; so.n = 1; so.w[0] = lw.wo; so.rows[0] = H;
     gemm(A(b.o), qd, rows, so, qd, nullptr, x0, H, b.h1, H);
     launch_rmsnorm<T>(L, b.h1, rows, H, W(lw.norm_post), g.rms_eps, A(b.u));
-    GemmSegs sg; sg.n = 2; sg.w[0] = lw.w_gate; sg.rows[0] = F; sg.w[1] = lw.w_up; sg.rows[1] = F;
-    gemm(A(b.u), H, rows, sg, H, nullptr, nullptr, 0, b.gu, 2 * F);
-    launch_silu_mul<T>(L, b.gu, rows, F, A(b.act));
+    gemm_swiglu(A(b.u), rows, lw.w_gate, lw.w_up, F, H, A(b.act));
     GemmSegs sd; sd.n = 1; sd.w[0] = lw.w_down; sd.rows[0] = H;
-    gemm(A(b.act), F, rows, sd, F, nullptr, b.h1, H, out, H);
+    gemm(A(b.act), F, rows, sd, F, nullptr, b.h1, H, out, H, 0, out_act);
   }
 
   int draft_prefill(void* draft_kv, int start, const int32_t* tokens, const void* features, int n) {
@@ -256,12 +265,10 @@ struct Impl {
       aa.n_all = prefix_len + n_new; aa.n_tree = i * K;
       aa.mask = b.ts.node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
-      plan_attention_splits(aa.rows, aa.Hkv, aa.n_all + aa.n_tree, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
-      launch_tree_attention<T>(L, aa, A(b.q), kc, vc, b.attn_part, A(b.o));
+      run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
       float* fo = b.fout + (size_t)i * KMAX * H;
       T* fbi = A(b.fb) + (size_t)i * KMAX * H;
-      layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo);
-      launch_cast_rows<T>(L, fo, (size_t)sr.Mc * H, fbi);
+      layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo, fbi);
       lm_head_topk(fbi, sr.Mc, K, b.top_ids, b.top_logp, nullptr);
       launch_expand(L, b.ts, KMAX, i, sr.Mc, K, cand_base, i == depth - 1, b.top_ids, b.top_logp);
       cand_base += sr.Mc * K;
@@ -287,10 +294,9 @@ struct Impl {
     AttnArgs aa;
     aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = kv_slots;
     aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = (rows + 63) / 64; aa.scale = scale;
-    plan_attention_splits(rows, aa.Hkv, prefix_len + rows, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
     const T* kc = W(kv);
     const T* vc = kc + (size_t)g.n_kv_heads * kv_slots * g.head_dim;
-    launch_tree_attention<T>(L, aa, W(q), kc, vc, c->b.attn_part, A(out));
+    run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, W(q), kc, vc, c->b.attn_part, A(out));
     return L.err;
   }
 
@@ -319,8 +325,7 @@ struct Impl {
       aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.target_kv_slots;
       aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = mask_words;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
-      plan_attention_splits(rows, aa.Hkv, prefix_len + rows, ATTN_MAX_SPLITS, &aa.n_splits, &aa.keys_per_split);
-      launch_tree_attention<T>(L, aa, A(b.q), kc, vc, b.attn_part, A(b.o));
+      run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
       layer_tail(lw, b.hx, rows, b.hx);
     }
     launch_rmsnorm<T>(L, b.hx, rows, H, W(c->final_norm), g.rms_eps, A(out_features));
@@ -332,18 +337,56 @@ struct Impl {
 
 template <typename T>
 void Impl<T>::gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual,
-                   int ldr, float* out, int ldo, int impl) {
+                   int ldr, float* out, int ldo, int impl, T* out_act) {
   launch_gemm_simt<T>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
+  if (out_act) launch_cast_rows<T>(L, out, (size_t)M * ldo, out_act);
 }
 template <>
 void Impl<bf16>::gemm(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, const bf16* bias,
-                      const float* residual, int ldr, float* out, int ldo, int impl) {
+                      const float* residual, int ldr, float* out, int ldo, int impl, bf16* out_act) {
   bool can_tc = tc_gemm_supported(segs, K, ldx, M);
   if (impl == 2 && !can_tc) { L.err = POSS_E_SHAPE; return; }
-  if (impl != 1 && can_tc)
-    launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, bias, residual, ldr, out, ldo, c->b.tc_scratch, c->b.status);
-  else
+  if (impl != 1 && can_tc) {
+    TcEpilogue ep;
+    ep.mode = TC_EPI_STORE; ep.bias = bias; ep.residual = residual; ep.ldr = ldr; ep.out = out; ep.ldo = ldo;
+    ep.out_bf = out_act; ep.ldo_bf = ldo;
+    launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, ep, c->b.tc_scratch, c->b.status);
+  } else {
     launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
+    if (out_act) launch_cast_rows<bf16>(L, out, (size_t)M * ldo, out_act);
+  }
+}
+
+template <typename T>
+void Impl<T>::gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act) {
+  GemmSegs sg; sg.n = 2; sg.w[0] = w_gate; sg.rows[0] = F; sg.w[1] = w_up; sg.rows[1] = F;
+  gemm(x, K, M, sg, K, nullptr, nullptr, 0, c->b.gu, 2 * F);
+  launch_silu_mul<T>(L, c->b.gu, M, F, act);
+}
+template <>
+void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const void* w_up, int F, int K, bf16* act) {
+  GemmSegs sg; sg.n = 2; sg.w[0] = w_gate; sg.rows[0] = F; sg.w[1] = w_up; sg.rows[1] = F;
+  if (tc_gemm_supported(sg, K, K, M)) {
+    TcEpilogue ep;
+    ep.mode = TC_EPI_SWIGLU; ep.out_bf = act; ep.ldo_bf = F;
+    launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
+    return;
+  }
+  gemm(x, K, M, sg, K, nullptr, nullptr, 0, c->b.gu, 2 * F);
+  launch_silu_mul<bf16>(L, c->b.gu, M, F, act);
+}
+
+template <typename T>
+bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*) { return false; }
+template <>
+bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists) {
+  GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = c->cfg.vocab;
+  if (!tc_gemm_supported(sg, K, K, M)) return false;
+  TcEpilogue ep;
+  ep.mode = TC_EPI_TOPK; ep.topk = topk;
+  ep.pmax = c->b.pmax; ep.psum = c->b.psum; ep.pval = c->b.pval; ep.pidx = c->b.pidx; ep.n_lists = n_lists;
+  launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
+  return true;
 }
 
 #define DISPATCH(ctx, stream, call)                         \

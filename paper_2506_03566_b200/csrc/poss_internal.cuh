@@ -114,6 +114,17 @@ void launch_tree_attention(Launcher& L, const AttnArgs& a, const T* q, const T* 
                            float* part, T* out);
 size_t attn_partial_floats(int rows, int Hq, int d, int n_splits);
 void plan_attention_splits(int rows, int Hkv, int total_keys, int max_splits, int* n_splits, int* keys_per_split);
+// Plans the key split (at most max_splits ranges; `part` holds attn_partial_floats(rows, Hq, d, max_splits)
+// floats) and runs the attention: the tensor-core kernel for bf16 shapes it covers, else the SIMT kernel.
+// a.n_splits / a.keys_per_split are filled in here.
+template <typename T>
+void run_tree_attention(Launcher& L, AttnArgs a, int max_splits, const T* q, const T* kcache, const T* vcache,
+                        float* part, T* out);
+bool tree_attention_mma_supported(const AttnArgs& a);
+void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int max_splits, int* n_splits,
+                               int* keys_per_split);
+void launch_tree_attention_mma(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc,
+                               float* part, bf16* out);
 
 #define POSS_TOPK_CHUNK 2048
 void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int K, float* pmax, float* psum,
