@@ -59,7 +59,7 @@ constexpr int XCH_STRIDE = 17;
 struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
-  int n_tiles, kb_total, gran;
+  int n_tiles, kb_total, gran, l2_ahead;
   const bf16* bias;
   const float* residual;
   int ldr;
@@ -128,6 +128,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
 }
+// brings a box into L2 only (no shared-memory destination, no barrier)
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -185,20 +189,6 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// ------------------------------------------------------------------ the stream-K range arithmetic
-// Units are k-blocks in (tile, k-block) order.  CTA c owns [range_begin(c), range_begin(c+1)).
-__host__ __device__ __forceinline__ long long range_begin(long long c, long long groups, int G, int gran) {
-  return (c * groups / G) * gran;
-}
-// the CTA whose range contains unit u
-__host__ __device__ __forceinline__ int cta_of_unit(long long u, long long groups, int G, int gran) {
-  long long g = u / gran;                       // group of the unit
-  // largest c with floor(c * groups / G) <= g  <=>  c * groups < (g + 1) * G
-  long long c = ((g + 1) * G + groups - 1) / groups - 1;
-  if (c > G - 1) c = G - 1;
-  return (int)c;
-}
-
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
 struct Segment {
@@ -233,8 +223,8 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
 
   const int G = gridDim.x;
   const long long groups = (long long)a.n_tiles * a.kb_total / a.gran;
-  const long long u0 = range_begin(blockIdx.x, groups, G, a.gran);
-  const long long u1 = range_begin(blockIdx.x + 1, groups, G, a.gran);
+  const long long u0 = splitk_range_begin(blockIdx.x, groups, G, a.gran);
+  const long long u1 = splitk_range_begin(blockIdx.x + 1, groups, G, a.gran);
   const int n_kb = (int)(u1 - u0);
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < 2 * a.Npad) tmem_cols <<= 1;
@@ -296,18 +286,33 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
           tma_load_2d(w_tile(s), mw, full_bar(s), kcoord, c.lt * TILE_N, pol_w);
         }
       };
+      auto prefetch_w = [&](const Cursor& c) {
+        int kcoord = c.kb * TILE_K;
+        if (a.mode == 1) {
+          tma_prefetch_l2_2d(&map_w0, kcoord, c.tile * 64);
+          tma_prefetch_l2_2d(&map_w1, kcoord, c.tile * 64);
+        } else {
+          const CUtensorMap* mw = c.seg == 0 ? &map_w0 : (c.seg == 1 ? &map_w1 : &map_w2);
+          tma_prefetch_l2_2d(mw, kcoord, c.lt * TILE_N);
+        }
+      };
       auto load_x = [&](const Cursor& c, int s) {
         tma_load_2d(x_tile(s), &map_x, full_bar(s), c.kb * TILE_K, 0, pol_x);
       };
-      // weights are never written by a kernel: fill the ring with them before waiting for the
-      // predecessor, whose results are the activations
+      // Weights are never written by a kernel: before waiting for the predecessor (whose results are
+      // the activations) fill the ring with them and ask L2 for the next k-blocks behind the ring, so
+      // the memory system keeps streaming through the predecessor's tail.
       const int pre = n_kb < S ? n_kb : S;
+      const int ahead = a.l2_ahead;
       Cursor cw = cursor_at(u0), cx = cw;
       for (int it = 0; it < pre; ++it) {
         mbar_expect_tx(full_bar(it), stage_bytes);
         load_w(cw, it);
         advance(cw);
       }
+      Cursor cp = cw;                          // next k-block to prefetch into L2
+      int n_pf = pre;
+      for (; n_pf < n_kb && n_pf < pre + ahead; ++n_pf) { prefetch_w(cp); advance(cp); }
       pdl_wait();
       for (int it = 0; it < pre; ++it) { load_x(cx, it); advance(cx); }
       int issued = pre, s = 0;
@@ -489,7 +494,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         }
       };
 
-      if (whole) {
+      if (whole && a.mode != 3) {
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
           float v[16];
           tmem_ld16(taddr + (uint32_t)c0, v);
@@ -501,10 +506,8 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
           epilogue_chunk(c0, v);
         }
       } else {
-        // partial K range: park the fp32 partial, the last arriver of the tile finishes it
-        const long long tile_u0 = (long long)tile * a.kb_total;
-        const int c_first = cta_of_unit(tile_u0, groups, G, a.gran);
-        const int c_last = cta_of_unit(tile_u0 + a.kb_total - 1, groups, G, a.gran);
+        // partial K range (or a product whose reduction is left to the consumer): park the fp32 partial;
+        // unless deferred, the last arriver of the tile finishes it
         const int slot = (u == u0) ? 0 : 1;       // a range's first segment, or its trailing one
         const size_t part_elems = (size_t)a.Npad * TILE_N;
         float* part = a.scratch + ((size_t)blockIdx.x * 2 + slot) * part_elems;
@@ -520,17 +523,22 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acc_empty(buf));
-        __threadfence();
+        if (a.mode == 3) { it += len; ++seg_i; continue; }   // the consumer kernel adds the partials
+        const long long tile_u0 = (long long)tile * a.kb_total;
+        const int c_first = splitk_cta_of_unit(tile_u0, groups, G, a.gran);
+        const int c_last = splitk_cta_of_unit(tile_u0 + a.kb_total - 1, groups, G, a.gran);
         epi_sync();
         if (threadIdx.x == 64) {
-          int prev = atomicAdd(&a.counters[tile], 1);
+          // release: the four warps' partial stores (ordered before this by the barrier) become visible
+          // before the count; acquire: the last arriver sees every earlier contributor's partial
+          int prev;
+          asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(prev) : "l"(&a.counters[tile]) : "memory");
           s_last = prev == (c_last - c_first);
         }
         epi_sync();
         const bool last = s_last != 0;
         epi_sync();                                // s_last is rewritten by the next partial segment
         if (last) {
-          __threadfence();
           for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
             float v[16];
 #pragma unroll
@@ -539,7 +547,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
               // contributor c: its range begins inside this tile (slot 0) unless it is the first
               // contributor and began earlier (then this tile is its trailing segment, slot 1)
               const bool two = c + 1 <= c_last;
-              long long b0 = range_begin(c, groups, G, a.gran);
+              long long b0 = splitk_range_begin(c, groups, G, a.gran);
               int s0 = (b0 >= tile_u0) ? 0 : 1;
               const float* p0 = a.scratch + ((size_t)c * 2 + s0) * part_elems + t;
               const float* p1 = a.scratch + ((size_t)(c + 1) * 2) * part_elems + t;   // a later contributor: slot 0
@@ -638,7 +646,7 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
-  int grid = 0, stages = 0;
+  int grid = 0, stages = 0, l2_ahead = 16;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -655,6 +663,7 @@ TcGemmPlanCache* tc_plan_cache_create() {
   if (c->grid > TC_MAX_GRID) c->grid = TC_MAX_GRID;
   c->stages = 0;
   if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
+  if (const char* e = getenv("POSS_TC_L2_AHEAD")) { int v = atoi(e); if (v >= 0 && v <= 4096) c->l2_ahead = v; }
   return c;
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
@@ -721,15 +730,38 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (ep.mode == TC_EPI_SWIGLU) n_tiles = a.seg_tiles[0];   // one tile = 64 gate + 64 up rows
   a.n_tiles = n_tiles;
   a.kb_total = (K + TILE_K - 1) / TILE_K;
+  // Leave the reduction to the consumer when the caller can take a view, every range is at most one
+  // tile long (so a CTA parks at most two segments) and groups of four columns never straddle a tile.
+  if (ep.view) {
+    bool ok4 = true;
+    for (int i = 0; i < segs.n; ++i) ok4 = ok4 && (segs.rows[i] % 4 == 0);
+    size_t need = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
+    bool defer = ep.mode == TC_EPI_STORE && ok4 && n_tiles <= cache->grid && need <= SCRATCH_PARTIAL_BYTES;
+    memset(ep.view, 0, sizeof(*ep.view));
+    if (defer) {
+      a.mode = TC_EPI_PARTIAL;
+    } else {
+      ep.view->deferred = 0;
+      ep.view->direct = ep.out;
+      ep.view->ld = ep.ldo;
+    }
+  }
   // whole tiles per CTA for the LM head (its epilogue keeps running state across tiles), and whenever
   // the partial buffers or the tile counters could not hold the split
   size_t part_bytes = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
-  bool no_split = ep.mode == TC_EPI_TOPK || part_bytes > SCRATCH_PARTIAL_BYTES || n_tiles > N_COUNTERS;
+  bool no_split = a.mode == TC_EPI_TOPK || part_bytes > SCRATCH_PARTIAL_BYTES || n_tiles > N_COUNTERS;
   a.gran = no_split ? a.kb_total : 1;
   // never more CTAs than ranges to hand out: every CTA of the grid owns at least one k-block
   long long groups = (long long)n_tiles * a.kb_total / a.gran;
   const int G = (long long)cache->grid < groups ? cache->grid : (int)groups;
   if (ep.n_lists) *ep.n_lists = G;
+  if (a.mode == TC_EPI_PARTIAL) {
+    SplitKView* v = ep.view;
+    v->deferred = 1;
+    v->scratch = reinterpret_cast<const float*>(scratch);
+    v->Npad = a.Npad; v->G = G; v->kb_total = a.kb_total; v->n_tiles = n_tiles; v->n_segs = segs.n;
+    for (int i = 0; i < segs.n; ++i) { v->seg_tiles[i] = a.seg_tiles[i]; v->seg_rows[i] = a.seg_rows[i]; }
+  }
   uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
@@ -738,6 +770,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
+  a.l2_ahead = cache->l2_ahead;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);

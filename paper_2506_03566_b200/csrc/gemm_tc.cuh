@@ -11,7 +11,7 @@ bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);
 
 constexpr int TC_MAX_GRID = 512;     // upper bound of the persistent grid = of the LM-head partial lists per row
 
-enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_TOPK = 2 };
+enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_TOPK = 2, TC_EPI_PARTIAL = 3 };
 
 // What happens to the accumulators.
 //   TC_EPI_STORE : out[m][n] (fp32, may be NULL) = acc + bias[n] + residual[m][n]; out_bf (may be NULL) gets the
@@ -20,6 +20,9 @@ enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_TOPK = 2 };
 //   TC_EPI_TOPK  : segs = {lm_head}; every CTA leaves, per activation row, the max, the sum of exp(logit - max) and
 //                  the topk best (logit, id) pairs of its vocabulary tiles, best first:
 //                  pmax/psum [M][n_lists], pval/pidx [M][n_lists][topk]; *n_lists receives the list count.
+//   TC_EPI_PARTIAL: nothing is reduced or stored: *view describes the parked partials for the consumer kernel
+//                  (see SplitKView).  Only chosen by the launcher when `view` is given and the shape allows it;
+//                  otherwise the launcher falls back to TC_EPI_STORE into `out` and *view describes that matrix.
 struct TcEpilogue {
   int mode = TC_EPI_STORE;
   const bf16* bias = nullptr;
@@ -35,6 +38,7 @@ struct TcEpilogue {
   float* pval = nullptr;
   int32_t* pidx = nullptr;
   int* n_lists = nullptr;
+  SplitKView* view = nullptr;
 };
 
 void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx, int M, const GemmSegs& segs, int K,

@@ -21,7 +21,7 @@ template <typename T, int D> struct KeyLoad;
 template <int D> struct KeyLoad<bf16, D> {
   // dot products of one key (D bf16, 16-byte loads) with G query vectors held in shared memory
   template <int G>
-  static __device__ __forceinline__ void dots(const bf16* __restrict__ k, const float* __restrict__ qs, float* s) {
+  static __device__ __forceinline__ void dots(const bf16* k, const float* qs, float* s) {
 #pragma unroll
     for (int c = 0; c < D / 8; ++c) {
       uint4 raw = *reinterpret_cast<const uint4*>(k + c * 8);
@@ -39,7 +39,7 @@ template <int D> struct KeyLoad<bf16, D> {
 };
 template <int D> struct KeyLoad<float, D> {
   template <int G>
-  static __device__ __forceinline__ void dots(const float* __restrict__ k, const float* __restrict__ qs, float* s) {
+  static __device__ __forceinline__ void dots(const float* k, const float* qs, float* s) {
 #pragma unroll
     for (int c = 0; c < D / 4; ++c) {
       float4 raw = *reinterpret_cast<const float4*>(k + c * 4);
@@ -54,13 +54,14 @@ template <int D> struct KeyLoad<float, D> {
 };
 
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(128) k_attn_partial(AttnArgs a, const T* __restrict__ q,
-                                                      const T* __restrict__ kcache, const T* __restrict__ vcache,
-                                                      float* __restrict__ part) {
+__global__ void __launch_bounds__(128) k_attn_partial(AttnArgs a, const T* q,
+                                                      const T* kcache, const T* vcache,
+                                                      float* part) {
   constexpr int PER = D / 32;                 // head-dim elements owned by a lane in the PV phase
   __shared__ float qs[G * D];
   __shared__ float sm_m[4][G], sm_l[4][G];
   __shared__ float sm_o[4][G][D];
+  pdl_enter();
   int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < G * D; i += 128)
@@ -152,7 +153,8 @@ __global__ void __launch_bounds__(128) k_attn_partial(AttnArgs a, const T* __res
 }
 
 template <typename T, int D>
-__global__ void k_attn_combine(int n_splits, const float* __restrict__ part, T* __restrict__ out) {
+__global__ void k_attn_combine(int n_splits, const float* part, T* out) {
+  pdl_enter();
   int rh = blockIdx.x;       // row * Hq + head
   int e = threadIdx.x;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);
@@ -190,10 +192,8 @@ void plan_attention_splits(int rows, int Hkv, int total_keys, int max_splits, in
 template <typename T, int D, int G>
 static void launch_attn_g(Launcher& L, const AttnArgs& a, const T* q, const T* kc, const T* vc, float* part, T* out) {
   dim3 grid(a.n_splits, a.Hkv, a.rows);
-  k_attn_partial<T, D, G><<<grid, 128, 0, L.stream>>>(a, q, kc, vc, part);
-  LAUNCH_CHECK(L);
-  k_attn_combine<T, D><<<a.rows * a.Hq, D, 0, L.stream>>>(a.n_splits, part, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_attn_partial<T, D, G>, grid, dim3(128), 0, a, q, kc, vc, part);
+  launch_pdl(L, k_attn_combine<T, D>, dim3(a.rows * a.Hq), dim3(D), 0, a.n_splits, (const float*)part, out);
 }
 template <typename T, int D>
 static void launch_attn_d(Launcher& L, const AttnArgs& a, const T* q, const T* kc, const T* vc, float* part, T* out) {

@@ -64,9 +64,9 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
 }
 
 template <int D>
-__global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* __restrict__ q,
-                                                  const bf16* __restrict__ kcache, const bf16* __restrict__ vcache,
-                                                  float* __restrict__ part, bf16* __restrict__ out) {
+__global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
+                                                  const bf16* kcache, const bf16* vcache,
+                                                  float* part, bf16* out) {
   constexpr int LD = D + 8;                       // padded shared-memory row, elements
   constexpr int KSTEPS = D / 16;                  // k-steps of Q K^T
   constexpr int NT_D = D / 8;                     // n-tiles of the output
@@ -74,8 +74,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* __rest
   bf16* Ks = reinterpret_cast<bf16*>(smem_attn);  // [2][CHUNK][LD]
   bf16* Vs = Ks + 2 * CHUNK * LD;                 // [2][CHUNK][LD]
 
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  pdl_enter();
 
   const int split = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -263,9 +262,8 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* __rest
 }
 
 template <int D>
-__global__ void k_attn_combine_bf16(int n_splits, const float* __restrict__ part, bf16* __restrict__ out) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+__global__ void k_attn_combine_bf16(int n_splits, const float* part, bf16* out) {
+  pdl_enter();
   int rh = blockIdx.x;       // row * Hq + head
   int e = threadIdx.x;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);
@@ -293,27 +291,9 @@ void launch_d(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, con
   }
   int G = a.Hq / a.Hkv;
   int q_tiles = (a.rows * G + QROWS - 1) / QROWS;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(a.n_splits, a.Hkv, q_tiles);
-  cfg.blockDim = dim3(128);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = L.stream;
-  cfg.attrs = at;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, k_attn_mma<D>, a, q, kc, vc, part, out) != cudaSuccess) L.err = POSS_E_CUDA;
-  LAUNCH_CHECK(L);
-  if (a.n_splits > 1) {
-    cfg.gridDim = dim3(a.rows * a.Hq);
-    cfg.blockDim = dim3(D);
-    cfg.dynamicSmemBytes = 0;
-    if (cudaLaunchKernelEx(&cfg, k_attn_combine_bf16<D>, a.n_splits, (const float*)part, out) != cudaSuccess)
-      L.err = POSS_E_CUDA;
-    LAUNCH_CHECK(L);
-  }
+  launch_pdl(L, k_attn_mma<D>, dim3(a.n_splits, a.Hkv, q_tiles), dim3(128), smem, a, q, kc, vc, part, out);
+  if (a.n_splits > 1)
+    launch_pdl(L, k_attn_combine_bf16<D>, dim3(a.rows * a.Hq), dim3(D), 0, a.n_splits, (const float*)part, out);
 }
 
 }  // namespace

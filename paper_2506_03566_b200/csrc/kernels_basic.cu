@@ -30,10 +30,11 @@ template <> struct Vec8<bf16> {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(256) k_gemm_simt(const T* __restrict__ X, int ldx, int M, GemmSegs segs, int N,
-                                                   int K, const T* __restrict__ bias,
-                                                   const float* __restrict__ residual, int ldr,
-                                                   float* __restrict__ out, int ldo) {
+__global__ void __launch_bounds__(256) k_gemm_simt(const T* X, int ldx, int M, GemmSegs segs, int N,
+                                                   int K, const T* bias,
+                                                   const float* residual, int ldr,
+                                                   float* out, int ldo) {
+  pdl_enter();
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int n = blockIdx.x * 8 + warp;
   if (n >= N) return;
@@ -80,8 +81,7 @@ void launch_gemm_simt(Launcher& L, const T* X, int ldx, int M, const GemmSegs& s
   int N = 0;
   for (int i = 0; i < segs.n; ++i) N += segs.rows[i];
   if (M <= 0 || N <= 0) return;
-  k_gemm_simt<T><<<(N + 7) / 8, 256, 0, L.stream>>>(X, ldx, M, segs, N, K, bias, residual, ldr, out, ldo);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_gemm_simt<T>, dim3((N + 7) / 8), dim3(256), 0, X, ldx, M, segs, N, K, bias, residual, ldr, out, ldo);
 }
 template void launch_gemm_simt<float>(Launcher&, const float*, int, int, const GemmSegs&, int, const float*,
                                       const float*, int, float*, int);
@@ -90,9 +90,13 @@ template void launch_gemm_simt<bf16>(Launcher&, const bf16*, int, int, const Gem
 
 // ------------------------------------------------------------------ layer-input pairs [E[tok] ; feature]
 template <typename T>
-__global__ void k_gather_x(StepRows s, const int32_t* __restrict__ new_tokens, const T* __restrict__ new_features,
-                           const int32_t* __restrict__ node_tok, const int32_t* __restrict__ node_prow, int Kmax,
-                           const T* __restrict__ fb, const T* __restrict__ embed, int H, T* __restrict__ X) {
+__global__ void __launch_bounds__(256) k_gather_x(StepRows s, const int32_t* new_tokens,
+                                                  const T* new_features,
+                                                  const int32_t* node_tok,
+                                                  const int32_t* node_prow, int Kmax,
+                                                  const T* fb, const T* embed, int H,
+                                                  T* X) {
+  pdl_enter();
   int m = blockIdx.x;
   RowInfo r = row_info(s, m);
   int tok;
@@ -107,18 +111,31 @@ __global__ void k_gather_x(StepRows s, const int32_t* __restrict__ new_tokens, c
   }
   const T* e = embed + (size_t)tok * H;
   T* x = X + (size_t)m * 2 * H;
-  for (int i = threadIdx.x; i < H; i += blockDim.x) {
-    x[i] = e[i];
-    x[H + i] = feat[i];
+  constexpr int PER = 16 / sizeof(T);                        // elements per 16-byte piece
+  bool vec = (H % PER) == 0 &&
+             ((reinterpret_cast<uintptr_t>(e) | reinterpret_cast<uintptr_t>(feat) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
+  if (vec) {
+    int n = H / PER;
+    const uint4* e4 = reinterpret_cast<const uint4*>(e);
+    const uint4* f4 = reinterpret_cast<const uint4*>(feat);
+    uint4* x4 = reinterpret_cast<uint4*>(x);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      x4[i] = e4[i];
+      x4[n + i] = f4[i];
+    }
+  } else {
+    for (int i = threadIdx.x; i < H; i += blockDim.x) {
+      x[i] = e[i];
+      x[H + i] = feat[i];
+    }
   }
 }
 template <typename T>
 void launch_gather_x(Launcher& L, StepRows s, const int32_t* new_tokens, const T* new_features,
                      const TreeState& ts, int Kmax, const T* fb, const T* embed, int H, T* X) {
   if (s.M <= 0) return;
-  k_gather_x<T><<<s.M, 256, 0, L.stream>>>(s, new_tokens, new_features, ts.node_tok, ts.node_prow, Kmax, fb, embed,
-                                           H, X);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_gather_x<T>, dim3(s.M), dim3(256), 0, s, new_tokens, new_features, ts.node_tok, ts.node_prow, Kmax,
+             fb, embed, H, X);
 }
 template void launch_gather_x<float>(Launcher&, StepRows, const int32_t*, const float*, const TreeState&, int,
                                      const float*, const float*, int, float*);
@@ -126,8 +143,9 @@ template void launch_gather_x<bf16>(Launcher&, StepRows, const int32_t*, const b
                                     const bf16*, const bf16*, int, bf16*);
 
 template <typename T>
-__global__ void k_embed_rows(const int32_t* __restrict__ tokens, const T* __restrict__ embed, int H,
-                             float* __restrict__ out) {
+__global__ void k_embed_rows(const int32_t* tokens, const T* embed, int H,
+                             float* out) {
+  pdl_enter();
   int m = blockIdx.x;
   const T* e = embed + (size_t)tokens[m] * H;
   for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)m * H + i] = to_f(e[i]);
@@ -135,26 +153,36 @@ __global__ void k_embed_rows(const int32_t* __restrict__ tokens, const T* __rest
 template <typename T>
 void launch_embed_rows(Launcher& L, const int32_t* tokens, int rows, const T* embed, int H, float* out) {
   if (rows <= 0) return;
-  k_embed_rows<T><<<rows, 256, 0, L.stream>>>(tokens, embed, H, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_embed_rows<T>, dim3(rows), dim3(256), 0, tokens, embed, H, out);
 }
 template void launch_embed_rows<float>(Launcher&, const int32_t*, int, const float*, int, float*);
 template void launch_embed_rows<bf16>(Launcher&, const int32_t*, int, const bf16*, int, float*);
 
 // ------------------------------------------------------------------ RMSNorm: out = T(gain * x / sqrt(mean x^2 + eps))
 template <typename T>
-__global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, int H, const T* __restrict__ gain,
-                                                 float eps, T* __restrict__ out) {
+__global__ void __launch_bounds__(256) k_rmsnorm(const float* x, int H, const T* gain,
+                                                 float eps, T* out) {
   __shared__ float red[8];
   __shared__ float inv_s;
+  pdl_enter();
   const float* xr = x + (size_t)blockIdx.x * H;
   T* o = out + (size_t)blockIdx.x * H;
   if (gain == nullptr) {
     for (int i = threadIdx.x; i < H; i += 256) o[i] = from_f<T>(xr[i]);
     return;
   }
+  // the row is summed in a fixed order: thread-strided partial sums, warp tree, then the eight warps
+  const bool vec = (H & 3) == 0 && (reinterpret_cast<uintptr_t>(xr) & 15) == 0;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < H; i += 256) { float v = xr[i]; ss = fmaf(v, v, ss); }
+  if (vec) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    for (int i = threadIdx.x; i < H / 4; i += 256) {
+      float4 v = x4[i];
+      ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+    }
+  } else {
+    for (int i = threadIdx.x; i < H; i += 256) { float v = xr[i]; ss = fmaf(v, v, ss); }
+  }
   for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
@@ -165,44 +193,55 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, in
   }
   __syncthreads();
   float inv = inv_s;
-  for (int i = threadIdx.x; i < H; i += 256) o[i] = from_f<T>(xr[i] * inv * to_f(gain[i]));
+  if (vec) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    for (int i = threadIdx.x; i < H / 4; i += 256) {
+      float4 v = x4[i];
+      o[4 * i] = from_f<T>(v.x * inv * to_f(gain[4 * i]));
+      o[4 * i + 1] = from_f<T>(v.y * inv * to_f(gain[4 * i + 1]));
+      o[4 * i + 2] = from_f<T>(v.z * inv * to_f(gain[4 * i + 2]));
+      o[4 * i + 3] = from_f<T>(v.w * inv * to_f(gain[4 * i + 3]));
+    }
+  } else {
+    for (int i = threadIdx.x; i < H; i += 256) o[i] = from_f<T>(xr[i] * inv * to_f(gain[i]));
+  }
 }
 template <typename T>
 void launch_rmsnorm(Launcher& L, const float* x, int rows, int H, const T* gain, float eps, T* out) {
   if (rows <= 0) return;
-  k_rmsnorm<T><<<rows, 256, 0, L.stream>>>(x, H, gain, eps, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_rmsnorm<T>, dim3(rows), dim3(256), 0, x, H, gain, eps, out);
 }
 template void launch_rmsnorm<float>(Launcher&, const float*, int, int, const float*, float, float*);
 template void launch_rmsnorm<bf16>(Launcher&, const float*, int, int, const bf16*, float, bf16*);
 
 template <typename T>
-__global__ void k_cast(const float* __restrict__ x, size_t n, T* __restrict__ out) {
+__global__ void k_cast(const float* x, size_t n, T* out) {
+  pdl_enter();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = from_f<T>(x[i]);
 }
 template <typename T>
 void launch_cast_rows(Launcher& L, const float* x, size_t n, T* out) {
   if (n == 0) return;
-  k_cast<T><<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(x, n, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_cast<T>, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, x, n, out);
 }
 template void launch_cast_rows<float>(Launcher&, const float*, size_t, float*);
 template void launch_cast_rows<bf16>(Launcher&, const float*, size_t, bf16*);
 
-__global__ void k_widen_bf16(const bf16* __restrict__ x, size_t n, float* __restrict__ out) {
+__global__ void k_widen_bf16(const bf16* x, size_t n, float* out) {
+  pdl_enter();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = __bfloat162float(x[i]);
 }
 void launch_widen_bf16(Launcher& L, const bf16* x, size_t n, float* out) {
   if (n == 0) return;
-  k_widen_bf16<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(x, n, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_widen_bf16, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, x, n, out);
 }
 
 // act = T(silu(gate) * up), gate/up stored side by side: gu[row][0..F) gate, [F..2F) up
 template <typename T>
-__global__ void k_silu_mul(const float* __restrict__ gu, int F, T* __restrict__ out) {
+__global__ void k_silu_mul(const float* gu, int F, T* out) {
+  pdl_enter();
   int row = blockIdx.y;
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= F) return;
@@ -214,21 +253,175 @@ template <typename T>
 void launch_silu_mul(Launcher& L, const float* gu, int rows, int F, T* out) {
   if (rows <= 0) return;
   dim3 grid((F + 255) / 256, rows);
-  k_silu_mul<T><<<grid, 256, 0, L.stream>>>(gu, F, out);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_silu_mul<T>, grid, dim3(256), 0, gu, F, out);
 }
 template void launch_silu_mul<float>(Launcher&, const float*, int, int, float*);
 template void launch_silu_mul<bf16>(Launcher&, const float*, int, int, bf16*);
 
-// ------------------------------------------------------------------ rotary embedding + KV append + q
-// qkv row layout: [Hq*d q | Hkv*d k | Hkv*d v] fp32.  Rotate-half pairing (j, j + d/2), angle
-// pos * theta^(-2j/d) evaluated in double so that long positions lose nothing.
+// ------------------------------------------------------------------ consumers of a (possibly split-K) product
+// Contributors of every tile, computed once per block.
+__device__ __forceinline__ void fill_tile_table(const SplitKView& v, TileContrib* tab) {
+  if (v.deferred)
+    for (int t = threadIdx.x; t < v.n_tiles; t += blockDim.x) tab[t] = splitk_tile_contrib(v, t);
+}
+// four consecutive columns of row m starting at n (a multiple of 4); N = row length
+__device__ __forceinline__ float4 product4(const SplitKView& v, const TileContrib* tab, int m, int n, int N) {
+  if (v.deferred) {
+    int tile, t;
+    splitk_locate(v, n, &tile, &t);
+    return splitk_load4(v, m, n, tab[tile], t);
+  }
+  const float* p = v.direct + (size_t)m * v.ld + n;
+  if ((v.ld & 3) == 0 && n + 3 < N && (reinterpret_cast<uintptr_t>(v.direct) & 15) == 0)
+    return *reinterpret_cast<const float4*>(p);
+  float4 r;
+  r.x = p[0];
+  r.y = n + 1 < N ? p[1] : 0.f;
+  r.z = n + 2 < N ? p[2] : 0.f;
+  r.w = n + 3 < N ? p[3] : 0.f;
+  return r;
+}
+
+// ---- h = product + bias + residual (fp32, stored);  xn = T(gain * h / rms(h))
+// One block per row.  The sum of squares is formed in a fixed order (per-thread partial sums over the
+// thread's column groups, a warp tree, then the warps in order), so a row's result does not depend on
+// the batch around it.
+#define NORM_THREADS 512
+#define NORM_KEEP 4
 template <typename T>
-__global__ void __launch_bounds__(128) k_rope_append(RopeArgs a, const float* __restrict__ qkv,
-                                                     T* __restrict__ kcache, T* __restrict__ vcache,
-                                                     T* __restrict__ qout) {
+__global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, int H, const T* bias,
+                                                               const float* residual, const T* gain, float eps,
+                                                               float* h, T* xn) {
+  __shared__ TileContrib tab[512];
+  __shared__ float red[NORM_THREADS / 32];
+  __shared__ float inv_s;
+  pdl_enter();
+  fill_tile_table(prod, tab);
+  __syncthreads();
+  const int m = blockIdx.x;
+  const int n_groups = (H + 3) / 4;
+  float ss = 0.f;
+  // value of one group of four columns: product + bias + residual, stored to h, squares added to ss
+  auto group_value = [&](int g) {
+    const int n = g * 4;
+    float4 v = product4(prod, tab, m, n, H);
+    float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (n + q < H) {
+        if (bias) e[q] += to_f(bias[n + q]);
+        if (residual) e[q] += residual[(size_t)m * H + n + q];
+        h[(size_t)m * H + n + q] = e[q];
+        ss = fmaf(e[q], e[q], ss);
+      } else {
+        e[q] = 0.f;
+      }
+    }
+    return make_float4(e[0], e[1], e[2], e[3]);
+  };
+  auto group_store = [&](int g, float4 v, float inv) {
+    const int n = g * 4;
+    float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (n + q < H) xn[(size_t)m * H + n + q] = gain ? from_f<T>(e[q] * inv * to_f(gain[n + q])) : from_f<T>(e[q]);
+  };
+  float4 keep[NORM_KEEP];
+#pragma unroll
+  for (int k = 0; k < NORM_KEEP; ++k) {
+    int g = threadIdx.x + k * NORM_THREADS;
+    keep[k] = g < n_groups ? group_value(g) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) group_value(g);
+  for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < NORM_THREADS / 32; ++w) t += red[w];
+    inv_s = gain ? rsqrtf(t / (float)H + eps) : 1.f;
+  }
+  __syncthreads();
+  const float inv = inv_s;
+#pragma unroll
+  for (int k = 0; k < NORM_KEEP; ++k) {
+    int g = threadIdx.x + k * NORM_THREADS;
+    if (g < n_groups) group_store(g, keep[k], inv);
+  }
+  for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) {
+    const int n = g * 4;                                    // wider rows: re-read this thread's own stores
+    float4 v;
+    v.x = h[(size_t)m * H + n];
+    v.y = n + 1 < H ? h[(size_t)m * H + n + 1] : 0.f;
+    v.z = n + 2 < H ? h[(size_t)m * H + n + 2] : 0.f;
+    v.w = n + 3 < H ? h[(size_t)m * H + n + 3] : 0.f;
+    group_store(g, v, inv);
+  }
+}
+template <typename T>
+void launch_reduce_norm(Launcher& L, const SplitKView& prod, int rows, int H, const T* bias, const float* residual,
+                        const T* gain, float eps, float* h, T* xn) {
+  if (rows <= 0) return;
+  launch_pdl(L, k_reduce_norm<T>, dim3(rows), dim3(NORM_THREADS), 0, prod, H, bias, residual, gain, eps, h, xn);
+}
+template void launch_reduce_norm<float>(Launcher&, const SplitKView&, int, int, const float*, const float*,
+                                        const float*, float, float*, float*);
+template void launch_reduce_norm<bf16>(Launcher&, const SplitKView&, int, int, const bf16*, const float*, const bf16*,
+                                       float, float*, bf16*);
+
+// ---- out = product + bias + residual, optionally also in the activation dtype
+template <typename T>
+__global__ void __launch_bounds__(256) k_splitk_reduce(SplitKView prod, int N, const T* bias, const float* residual,
+                                                       int ldr, float* out, int ldo, T* out_act) {
+  pdl_enter();
+  const int m = blockIdx.y;
+  const int n = (blockIdx.x * 256 + threadIdx.x) * 4;
+  if (n >= N) return;
+  float4 v;
+  if (prod.deferred) {
+    int tile, t;
+    splitk_locate(prod, n, &tile, &t);
+    TileContrib tc = splitk_tile_contrib(prod, tile);
+    v = splitk_load4(prod, m, n, tc, t);
+  } else {
+    v = product4(prod, nullptr, m, n, N);
+  }
+  float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (n + q < N) {
+      if (bias) e[q] += to_f(bias[n + q]);
+      if (residual) e[q] += residual[(size_t)m * ldr + n + q];
+      if (out) out[(size_t)m * ldo + n + q] = e[q];
+      if (out_act) out_act[(size_t)m * ldo + n + q] = from_f<T>(e[q]);
+    }
+  }
+}
+template <typename T>
+void launch_splitk_reduce(Launcher& L, const SplitKView& prod, int rows, int N, const T* bias, const float* residual,
+                          int ldr, float* out, int ldo, T* out_act) {
+  if (rows <= 0) return;
+  launch_pdl(L, k_splitk_reduce<T>, dim3((N + 1023) / 1024, rows), dim3(256), 0, prod, N, bias, residual, ldr, out, ldo,
+             out_act);
+}
+template void launch_splitk_reduce<float>(Launcher&, const SplitKView&, int, int, const float*, const float*, int,
+                                          float*, int, float*);
+template void launch_splitk_reduce<bf16>(Launcher&, const SplitKView&, int, int, const bf16*, const float*, int, float*,
+                                         int, bf16*);
+
+// ------------------------------------------------------------------ rotary embedding + KV append + q
+// The product's row layout is [Hq*d q | Hkv*d k | Hkv*d v] fp32.  Rotate-half pairing (j, j + d/2).
+// The angle pos * theta^(-2j/d) is formed in double from a table of the d/2 inverse frequencies and
+// reduced to [-pi, pi] in double (2 pi split in two terms), so long positions lose nothing; sine and
+// cosine of the reduced angle are then taken in fp32.  One block per row; a work item is four
+// neighbouring pairs of one head (two 16-byte loads) or four values.
+template <typename T>
+__global__ void __launch_bounds__(256) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache, T* qout) {
+  __shared__ TileContrib tab[512];
   __shared__ float cs[64], sn[64];
-  int m = blockIdx.x;
+  pdl_enter();
+  fill_tile_table(qkv, tab);
+  const int m = blockIdx.x;
   int slot, pos;
   if (a.mode == 0) {
     RowInfo r = row_info(a.s, m);
@@ -238,53 +431,60 @@ __global__ void __launch_bounds__(128) k_rope_append(RopeArgs a, const float* __
     slot = a.base + m;
     pos = a.base + a.depth[m];
   }
-  int half = a.d / 2;
+  const int half = a.d / 2;
   if ((int)threadIdx.x < half) {
-    double inv = exp2(-2.0 * (double)threadIdx.x / (double)a.d * log2((double)a.theta));
-    double s, c;
-    sincos((double)pos * inv, &s, &c);
-    cs[threadIdx.x] = (float)c;
-    sn[threadIdx.x] = (float)s;
+    const double two_pi_hi = 6.283185307179586, two_pi_lo = 2.4492935982947064e-16;
+    double x = (double)pos * a.inv_freq[threadIdx.x];
+    double k = rint(x * 0.15915494309189535);
+    double r = fma(-k, two_pi_hi, x);
+    r = fma(-k, two_pi_lo, r);
+    float s, c;
+    sincosf((float)r, &s, &c);
+    cs[threadIdx.x] = c;
+    sn[threadIdx.x] = s;
   }
   __syncthreads();
-  int qd = a.Hq * a.d, kd = a.Hkv * a.d;
-  const float* row = qkv + (size_t)m * (qd + 2 * kd);
-  // keys
-  for (int i = threadIdx.x; i < a.Hkv * half; i += blockDim.x) {
-    int h = i / half, j = i % half;
-    float x0 = row[qd + h * a.d + j], x1 = row[qd + h * a.d + j + half];
-    T* dst = kcache + ((size_t)h * a.cap + slot) * a.d;
-    dst[j] = from_f<T>(x0 * cs[j] - x1 * sn[j]);
-    dst[j + half] = from_f<T>(x1 * cs[j] + x0 * sn[j]);
-  }
-  // values
-  for (int i = threadIdx.x; i < kd; i += blockDim.x) {
-    int h = i / a.d, j = i % a.d;
-    vcache[((size_t)h * a.cap + slot) * a.d + j] = from_f<T>(row[qd + kd + i]);
-  }
-  // queries of the current rows
-  int q0 = a.rows - a.q_rows;
-  if (m >= q0) {
-    T* qo = qout + (size_t)(m - q0) * qd;
-    for (int i = threadIdx.x; i < a.Hq * half; i += blockDim.x) {
-      int h = i / half, j = i % half;
-      float x0 = row[h * a.d + j], x1 = row[h * a.d + j + half];
-      qo[h * a.d + j] = from_f<T>(x0 * cs[j] - x1 * sn[j]);
-      qo[h * a.d + j + half] = from_f<T>(x1 * cs[j] + x0 * sn[j]);
+  const int qd = a.Hq * a.d, kd = a.Hkv * a.d, N = qd + 2 * kd;
+  const int q0 = a.rows - a.q_rows;
+  const bool with_q = m >= q0;
+  const int per_head = half / 4;                         // items per rotated head (d is a multiple of 8)
+  const int n_qitems = with_q ? a.Hq * per_head : 0;
+  const int n_kitems = a.Hkv * per_head;
+  const int n_vitems = kd / 4;
+  for (int i = threadIdx.x; i < n_qitems + n_kitems + n_vitems; i += blockDim.x) {
+    if (i < n_qitems + n_kitems) {
+      const bool is_q = i < n_qitems;
+      const int ii = is_q ? i : i - n_qitems;
+      const int hh = ii / per_head, j = (ii % per_head) * 4;
+      const int col = (is_q ? 0 : qd) + hh * a.d + j;
+      float4 lo = product4(qkv, tab, m, col, N), hi = product4(qkv, tab, m, col + half, N);
+      float x0[4] = {lo.x, lo.y, lo.z, lo.w}, x1[4] = {hi.x, hi.y, hi.z, hi.w};
+      T* dst = is_q ? qout + (size_t)(m - q0) * qd + hh * a.d : kcache + ((size_t)hh * a.cap + slot) * a.d;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        dst[j + e] = from_f<T>(x0[e] * cs[j + e] - x1[e] * sn[j + e]);
+        dst[j + e + half] = from_f<T>(x1[e] * cs[j + e] + x0[e] * sn[j + e]);
+      }
+    } else {
+      const int ii = (i - n_qitems - n_kitems) * 4;
+      const int hh = ii / a.d, j = ii % a.d;
+      float4 v = product4(qkv, tab, m, qd + kd + ii, N);
+      T* dst = vcache + ((size_t)hh * a.cap + slot) * a.d + j;
+      dst[0] = from_f<T>(v.x); dst[1] = from_f<T>(v.y); dst[2] = from_f<T>(v.z); dst[3] = from_f<T>(v.w);
     }
   }
 }
 template <typename T>
-void launch_rope_append(Launcher& L, const RopeArgs& a, const float* qkv, T* kcache, T* vcache, T* qout) {
+void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {
   if (a.rows <= 0) return;
-  k_rope_append<T><<<a.rows, 128, 0, L.stream>>>(a, qkv, kcache, vcache, qout);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_rope_append<T>, dim3(a.rows), dim3(256), 0, a, qkv, kcache, vcache, qout);
 }
-template void launch_rope_append<float>(Launcher&, const RopeArgs&, const float*, float*, float*, float*);
-template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const float*, bf16*, bf16*, bf16*);
+template void launch_rope_append<float>(Launcher&, const RopeArgs&, const SplitKView&, float*, float*, float*);
+template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKView&, bf16*, bf16*, bf16*);
 
 // chain mask / depth for causal prefill chunks: row r sees rows 0..r of its chunk
 __global__ void k_chain_mask(uint64_t* mask, int32_t* depth, int rows) {
+  pdl_enter();
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= rows) return;
   depth[r] = r;
@@ -296,6 +496,5 @@ __global__ void k_chain_mask(uint64_t* mask, int32_t* depth, int rows) {
   mask[2 * r + 1] = hi;
 }
 void launch_chain_mask(Launcher& L, uint64_t* mask, int32_t* depth, int rows) {
-  k_chain_mask<<<(rows + 127) / 128, 128, 0, L.stream>>>(mask, depth, rows);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_chain_mask, dim3((rows + 127) / 128), dim3(128), 0, mask, depth, rows);
 }

@@ -2,6 +2,7 @@
 // Every ordering rule is (value descending, index ascending), so results are unique.
 #include "poss_internal.cuh"
 #include <math.h>
+#include <string.h>
 
 #define LAUNCH_CHECK(L)                                         \
   do {                                                          \
@@ -23,14 +24,15 @@ __device__ __forceinline__ void warp_best(float& v, int& i) {
 }
 
 // ------------------------------------------------------------------ per-chunk max / sum-exp / top-k of fp32 logits
-__global__ void __launch_bounds__(256) k_topk_partial(const float* __restrict__ logits, int V, int K,
-                                                      float* __restrict__ pmax, float* __restrict__ psum,
-                                                      float* __restrict__ pval, int32_t* __restrict__ pidx,
+__global__ void __launch_bounds__(256) k_topk_partial(const float* logits, int V, int K,
+                                                      float* pmax, float* psum,
+                                                      float* pval, int32_t* pidx,
                                                       int n_chunks) {
   __shared__ float vals[POSS_TOPK_CHUNK];
   __shared__ float wv[8];
   __shared__ int wi[8];
   __shared__ float s_max;
+  pdl_enter();
   int chunk = blockIdx.x, row = blockIdx.y;
   int lo = chunk * POSS_TOPK_CHUNK;
   int n = min(POSS_TOPK_CHUNK, V - lo);
@@ -96,87 +98,30 @@ void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int 
                          float* pval, int32_t* pidx, int n_chunks) {
   if (rows <= 0) return;
   dim3 grid(n_chunks, rows);
-  k_topk_partial<<<grid, 256, 0, L.stream>>>(logits, V, K, pmax, psum, pval, pidx, n_chunks);
-  LAUNCH_CHECK(L);
-}
-
-// ------------------------------------------------------------------ merge chunk partials: one warp per row
-// Each chunk's list is already ordered best first, so the merge repeatedly takes the best chunk head.
-// -inf entries (a chunk shorter than K) never win against a real value.
-__global__ void __launch_bounds__(32) k_topk_merge(int K, int n_chunks, const float* __restrict__ pmax,
-                                                   const float* __restrict__ psum, const float* __restrict__ pval,
-                                                   const int32_t* __restrict__ pidx, int32_t* __restrict__ out_ids,
-                                                   float* __restrict__ out_logp) {
-  extern __shared__ int heads[];     // [n_chunks]
-  int row = blockIdx.x, lane = threadIdx.x;
-  const float* rmax = pmax + (size_t)row * n_chunks;
-  const float* rsum = psum + (size_t)row * n_chunks;
-  float gm = NEG_INF;
-  for (int c = lane; c < n_chunks; c += 32) { gm = fmaxf(gm, rmax[c]); heads[c] = 0; }
-  for (int off = 16; off > 0; off >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, off));
-  float se = 0.f;
-  for (int c = lane; c < n_chunks; c += 32) se += rsum[c] * expf(rmax[c] - gm);
-  for (int off = 16; off > 0; off >>= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
-  float lse = gm + logf(se);
-  __syncwarp();
-  for (int k = 0; k < K; ++k) {
-    float bv = NEG_INF;
-    int bi = 0x7fffffff, bc = -1;
-    for (int c = lane; c < n_chunks; c += 32) {
-      int h = heads[c];
-      if (h < K) {
-        size_t p = ((size_t)row * n_chunks + c) * K + h;
-        float v = pval[p];
-        int i = pidx[p];
-        if (better(v, i, bv, bi)) { bv = v; bi = i; bc = c; }
-      }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-      int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-      int oc = __shfl_xor_sync(0xffffffffu, bc, off);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bc = oc; }
-    }
-    if (lane == 0) {
-      out_ids[(size_t)row * K + k] = bi;
-      out_logp[(size_t)row * K + k] = bv - lse;
-      if (bc >= 0) heads[bc] += 1;
-    }
-    __syncwarp();
-  }
-}
-
-void launch_topk_merge(Launcher& L, int rows, int K, int n_chunks, const float* pmax, const float* psum,
-                       const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp) {
-  if (rows <= 0) return;
-  k_topk_merge<<<rows, 32, n_chunks * sizeof(int), L.stream>>>(K, n_chunks, pmax, psum, pval, pidx, out_ids,
-                                                               out_logp);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_topk_partial, grid, dim3(256), 0, logits, V, K, pmax, psum, pval, pidx, n_chunks);
 }
 
 // ------------------------------------------------------------------ tree expansion after draft step `step`
 // Rows r = 0..Mc-1 are the level-`step` frontier.  Appends Mc*K level-(step+1) candidates in
 // (row, rank) order with score = row score + logp, then (unless last) picks the K best of them as the
 // next frontier, best first, and records for each its token, parent row, score, flat index and the
-// tree-slot mask (parent's mask plus its own slot step*K + rank).
-__global__ void __launch_bounds__(256) k_expand(TreeState ts, int Kmax, int step, int Mc, int K, int cand_base,
-                                                int last, const int32_t* __restrict__ top_ids,
-                                                const float* __restrict__ top_logp) {
-  __shared__ float sc[POSS_MAX_TOPK * POSS_MAX_TOPK];
-  int n = Mc * K;
+// tree-slot mask (parent's mask plus its own slot step*K + rank).  Runs inside one block.
+__device__ void expand_block(const TreeState& ts, const ExpandArgs& x, const int32_t* top_ids, const float* top_logp,
+                             float* sc) {
+  const int K = x.K, Kmax = x.Kmax, step = x.step;
+  int n = x.Mc * K;
   for (int c = threadIdx.x; c < n; c += blockDim.x) {
     int r = c / K;
     float ps = step == 0 ? 0.f : ts.node_score[step * Kmax + r];
     int pc = step == 0 ? -1 : ts.node_cand[step * Kmax + r];
-    float s = ps + top_logp[c];
+    float s = ps + __ldcg(top_logp + c);
     sc[c] = s;
-    ts.cand_tok[cand_base + c] = top_ids[c];
-    ts.cand_parent[cand_base + c] = pc;
-    ts.cand_score[cand_base + c] = s;
+    ts.cand_tok[x.cand_base + c] = __ldcg(top_ids + c);
+    ts.cand_parent[x.cand_base + c] = pc;
+    ts.cand_score[x.cand_base + c] = s;
   }
   __syncthreads();
-  if (last) return;
+  if (x.last) return;
   int lvl = step + 1;
   for (int c = threadIdx.x; c < n; c += blockDim.x) {
     float s = sc[c];
@@ -185,9 +130,9 @@ __global__ void __launch_bounds__(256) k_expand(TreeState ts, int Kmax, int step
     if (rank < K) {
       int r = c / K;
       int at = lvl * Kmax + rank;
-      ts.node_tok[at] = top_ids[c];
+      ts.node_tok[at] = __ldcg(top_ids + c);
       ts.node_prow[at] = r;
-      ts.node_cand[at] = cand_base + c;
+      ts.node_cand[at] = x.cand_base + c;
       ts.node_score[at] = s;
       uint64_t m0 = 0, m1 = 0;
       if (step > 0) { m0 = ts.node_mask[(step * Kmax + r) * 2]; m1 = ts.node_mask[(step * Kmax + r) * 2 + 1]; }
@@ -199,10 +144,115 @@ __global__ void __launch_bounds__(256) k_expand(TreeState ts, int Kmax, int step
   }
 }
 
-void launch_expand(Launcher& L, const TreeState& ts, int Kmax, int step, int Mc, int K, int cand_base, int last,
-                   const int32_t* top_ids, const float* top_logp) {
-  k_expand<<<1, 256, 0, L.stream>>>(ts, Kmax, step, Mc, K, cand_base, last, top_ids, top_logp);
-  LAUNCH_CHECK(L);
+// ------------------------------------------------------------------ merge the partial lists of a row, finish log-softmax
+// One block per activation row.  Every list is ordered best first, so the merge repeatedly takes the
+// best list head; -inf entries (a list shorter than K) never win against a real value.  The block that
+// finishes last (a counter, nobody waits) also runs the tree expansion when the caller asks for it.
+__global__ void __launch_bounds__(128) k_topk_merge(int K, int n_lists, const float* pmax,
+                                                    const float* psum, const float* pval,
+                                                    const int32_t* pidx, int32_t* out_ids,
+                                                    float* out_logp, TreeState ts, ExpandArgs x,
+                                                    int* done) {
+  extern __shared__ unsigned char merge_smem[];
+  float* vals = reinterpret_cast<float*>(merge_smem);                 // [n_lists][K]
+  int* idxs = reinterpret_cast<int*>(vals + (size_t)n_lists * K);     // [n_lists][K]
+  int* heads = idxs + (size_t)n_lists * K;                            // [n_lists]
+  __shared__ float red[4];
+  __shared__ float s_gm, s_lse;
+  __shared__ int s_is_last;
+  pdl_enter();
+  const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float* rmax = pmax + (size_t)row * n_lists;
+  const float* rsum = psum + (size_t)row * n_lists;
+  for (int i = threadIdx.x; i < n_lists * K; i += 128) {
+    vals[i] = pval[(size_t)row * n_lists * K + i];
+    idxs[i] = pidx[(size_t)row * n_lists * K + i];
+  }
+  float gm = NEG_INF;
+  for (int c = threadIdx.x; c < n_lists; c += 128) { gm = fmaxf(gm, rmax[c]); heads[c] = 0; }
+  for (int off = 16; off > 0; off >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, off));
+  if (lane == 0) red[warp] = gm;
+  __syncthreads();
+  if (threadIdx.x == 0) s_gm = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  __syncthreads();
+  gm = s_gm;
+  float se = 0.f;
+  for (int c = threadIdx.x; c < n_lists; c += 128) {
+    float m = rmax[c];
+    if (m > NEG_INF) se += rsum[c] * expf(m - gm);
+  }
+  for (int off = 16; off > 0; off >>= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
+  __syncthreads();
+  if (lane == 0) red[warp] = se;
+  __syncthreads();
+  if (threadIdx.x == 0) s_lse = gm + logf(((red[0] + red[1]) + red[2]) + red[3]);
+  __syncthreads();
+  if (warp == 0) {
+    const float lse = s_lse;
+    for (int k = 0; k < K; ++k) {
+      float bv = NEG_INF;
+      int bi = 0x7fffffff, bc = -1;
+      for (int c = lane; c < n_lists; c += 32) {
+        int h = heads[c];
+        if (h < K) {
+          float v = vals[c * K + h];
+          int i = idxs[c * K + h];
+          if (better(v, i, bv, bi)) { bv = v; bi = i; bc = c; }
+        }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+        int oc = __shfl_xor_sync(0xffffffffu, bc, off);
+        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bc = oc; }
+      }
+      if (lane == 0) {
+        out_ids[(size_t)row * K + k] = bi;
+        out_logp[(size_t)row * K + k] = bv - lse;
+        if (bc >= 0) heads[bc] += 1;
+      }
+      __syncwarp();
+    }
+  }
+  if (!x.enabled) return;
+  // ---- the last block to finish expands the tree
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    int prev = atomicAdd(done, 1);
+    s_is_last = prev == (int)gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_is_last) return;
+  __threadfence();
+  expand_block(ts, x, out_ids, out_logp, vals);      // vals is free now: K*K <= its size is checked by the host
+  if (threadIdx.x == 0) *done = 0;
+}
+
+void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* pmax, const float* psum,
+                       const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp,
+                       const TreeState* ts, const ExpandArgs* x, int* done) {
+  if (rows <= 0) return;
+  ExpandArgs xa;
+  memset(&xa, 0, sizeof(xa));
+  TreeState t;
+  memset(&t, 0, sizeof(t));
+  if (x && ts && x->enabled) { xa = *x; t = *ts; }
+  size_t elems = (size_t)n_lists * K;
+  if (xa.enabled && elems < (size_t)xa.Mc * K) elems = (size_t)xa.Mc * K;      // room for the expansion's scores
+  size_t smem = elems * 8 + (size_t)n_lists * 4;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(k_topk_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess) {
+      L.err = POSS_E_CUDA;
+      return;
+    }
+    attr_done = true;
+  }
+  if (smem > 100 * 1024) { L.err = POSS_E_CAPACITY; return; }
+  launch_pdl(L, k_topk_merge, dim3(rows), dim3(128), smem, K, n_lists, pmax, psum, pval, pidx, out_ids, out_logp, t, xa,
+             done);
 }
 
 // ------------------------------------------------------------------ rerank: keep the `total` best candidates
@@ -210,11 +260,12 @@ void launch_expand(Launcher& L, const TreeState& ts, int Kmax, int step, int Mc,
 // candidates are listed in flat (creation) order behind the root, so a parent always precedes its
 // children; level of flat index c is 1 for c < K, else 2 + (c - K) / K^2.
 __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K, int total,
-                                                 const int32_t* __restrict__ root_tok,
-                                                 int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_parents,
-                                                 float* __restrict__ out_scores, int32_t* __restrict__ out_depth,
-                                                 uint64_t* __restrict__ out_mask, int32_t* __restrict__ out_n_nodes) {
+                                                 const int32_t* root_tok,
+                                                 int32_t* out_tokens, int32_t* out_parents,
+                                                 float* out_scores, int32_t* out_depth,
+                                                 uint64_t* out_mask, int32_t* out_n_nodes) {
   extern __shared__ unsigned char smem_raw[];
+  pdl_enter();
   float* sc = reinterpret_cast<float*>(smem_raw);               // [n_cand]
   int* newidx = reinterpret_cast<int*>(sc + n_cand);            // [n_cand] node index or 0 if dropped
   int keep = min(total, n_cand);
@@ -269,22 +320,22 @@ void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int tota
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
   size_t smem = (size_t)n_cand * 8;
-  k_rerank<<<1, 1024, smem, L.stream>>>(ts, n_cand, K, total, new_tokens + root_tok_index, out_tokens, out_parents,
-                                        out_scores, out_depth, out_mask, out_n_nodes);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_rerank, dim3(1), dim3(1024), smem, ts, n_cand, K, total, new_tokens + root_tok_index, out_tokens,
+             out_parents, out_scores, out_depth, out_mask, out_n_nodes);
 }
 
 // ------------------------------------------------------------------ greedy accept walk (one warp) + hand-over pairs
 template <typename T>
-__global__ void __launch_bounds__(32) k_accept_walk(const int32_t* __restrict__ g, const T* __restrict__ feats,
-                                                    int H, const int32_t* __restrict__ tokens,
-                                                    const int32_t* __restrict__ parents, int rows, int max_depth,
-                                                    int32_t* __restrict__ out_path, int32_t* __restrict__ out_a,
-                                                    int32_t* __restrict__ out_bonus,
-                                                    int32_t* __restrict__ out_new_tokens,
-                                                    T* __restrict__ out_new_features,
-                                                    unsigned long long* __restrict__ counters) {
+__global__ void __launch_bounds__(32) k_accept_walk(const int32_t* g, const T* feats,
+                                                    int H, const int32_t* tokens,
+                                                    const int32_t* parents, int rows, int max_depth,
+                                                    int32_t* out_path, int32_t* out_a,
+                                                    int32_t* out_bonus,
+                                                    int32_t* out_new_tokens,
+                                                    T* out_new_features,
+                                                    unsigned long long* counters) {
   __shared__ int path[POSS_MAX_DEPTH + 1];
+  pdl_enter();
   int lane = threadIdx.x;
   int cur = 0, a = 0;
   if (lane == 0) path[0] = 0;
@@ -319,9 +370,8 @@ void launch_accept_walk(Launcher& L, const int32_t* g, const T* feats, int H, co
                         const int32_t* parents, int rows, int max_depth, int32_t* out_path, int32_t* out_a,
                         int32_t* out_bonus, int32_t* out_new_tokens, T* out_new_features,
                         unsigned long long* counters) {
-  k_accept_walk<T><<<1, 32, 0, L.stream>>>(g, feats, H, tokens, parents, rows, max_depth, out_path, out_a, out_bonus,
-                                           out_new_tokens, out_new_features, counters);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_accept_walk<T>, dim3(1), dim3(32), 0, g, feats, H, tokens, parents, rows, max_depth, out_path, out_a,
+             out_bonus, out_new_tokens, out_new_features, counters);
 }
 template void launch_accept_walk<float>(Launcher&, const int32_t*, const float*, int, const int32_t*, const int32_t*,
                                         int, int, int32_t*, int32_t*, int32_t*, int32_t*, float*,
@@ -333,9 +383,10 @@ template void launch_accept_walk<bf16>(Launcher&, const int32_t*, const bf16*, i
 // Block (layer*2 + kv, head): copies slot prefix_len + path[k] to prefix_len + k for k = 1..a in
 // ascending k.  path[k] >= k, so a source is never overwritten before it is read.
 template <typename T>
-__global__ void __launch_bounds__(128) k_kv_compact(T* __restrict__ kv, int Hkv, int cap, int d, int prefix_len,
-                                                    const int32_t* __restrict__ path,
-                                                    const int32_t* __restrict__ n_accepted) {
+__global__ void __launch_bounds__(128) k_kv_compact(T* kv, int Hkv, int cap, int d, int prefix_len,
+                                                    const int32_t* path,
+                                                    const int32_t* n_accepted) {
+  pdl_enter();
   int a = n_accepted[0];
   T* base = kv + ((size_t)blockIdx.x * Hkv + blockIdx.y) * (size_t)cap * d;
   for (int k = 1; k <= a; ++k) {
@@ -350,8 +401,7 @@ template <typename T>
 void launch_kv_compact(Launcher& L, T* target_kv, int layers, int Hkv, int cap, int d, int prefix_len,
                        const int32_t* path, const int32_t* n_accepted) {
   dim3 grid(layers * 2, Hkv);
-  k_kv_compact<T><<<grid, 128, 0, L.stream>>>(target_kv, Hkv, cap, d, prefix_len, path, n_accepted);
-  LAUNCH_CHECK(L);
+  launch_pdl(L, k_kv_compact<T>, grid, dim3(128), 0, target_kv, Hkv, cap, d, prefix_len, path, n_accepted);
 }
 template void launch_kv_compact<float>(Launcher&, float*, int, int, int, int, int, const int32_t*, const int32_t*);
 template void launch_kv_compact<bf16>(Launcher&, bf16*, int, int, int, int, int, const int32_t*, const int32_t*);

@@ -6,6 +6,7 @@
 #include <new>
 #include <stdlib.h>
 #include <string.h>
+#include <math.h>
 
 namespace {
 
@@ -29,6 +30,7 @@ struct Buffers {
   float* h0;          // [R][H]
   void* xn;           // [R][H] act
   float* qkv;         // [R][(Hq+2Hkv)d]
+  float* ptmp;        // [R][max(H, (Hq+2Hkv)d)] product of a GEMM that did not leave split-K partials
   void* q;            // [R][Hq d] act
   float* attn_part;
   void* o;            // [R][Hq d] act
@@ -49,6 +51,8 @@ struct Buffers {
   int32_t* argmax_tmp;   // [R]
   unsigned long long* counters;  // [POSS_MAX_DEPTH + 2]
   int32_t* status;       // [1]
+  int* merge_done;       // [1] block counter of the top-k merge kernel
+  double* rope_inv;      // [head_dim / 2] inverse rotary frequencies
   void* tc_scratch;      // split-K partials + tile counters of the tensor-core GEMM
   TreeState ts;
 };
@@ -113,6 +117,7 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.h0 = bp.take<float>(R * H, 4);
   b.xn = bp.take<void>(R * H, es);
   b.qkv = bp.take<float>(R * (qd + 2 * kd), 4);
+  b.ptmp = bp.take<float>(R * (H > qd + 2 * kd ? H : qd + 2 * kd), 4);
   b.q = bp.take<void>(R * qd, es);
   b.attn_part = bp.take<float>(attn_partial_floats(R, c.n_q_heads, c.head_dim, ATTN_MAX_SPLITS), 4);
   b.o = bp.take<void>(R * qd, es);
@@ -137,6 +142,8 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.argmax_tmp = bp.take<int32_t>(R, 4);
   b.counters = bp.take<unsigned long long>(POSS_MAX_DEPTH + 2, 8);
   b.status = bp.take<int32_t>(64, 4);
+  b.merge_done = bp.take<int>(64, 4);
+  b.rope_inv = bp.take<double>(64, 8);
   b.tc_scratch = bp.take<void>(tc_gemm_scratch_bytes(), 1);
   b.ts.cand_tok = bp.take<int32_t>(*n_cand_max, 4);
   b.ts.cand_parent = bp.take<int32_t>(*n_cand_max, 4);
@@ -165,12 +172,16 @@ struct Impl {
   // out_act (optional, [M][ldo]) receives the same values in the context dtype
   void gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual, int ldr,
             float* out, int ldo, int impl = 0, T* out_act = nullptr);
+  // x . segs^T handed to a consumer kernel: split-K partials when the tensor-core kernel can leave them,
+  // else the plain product in tmp[M][ldo]
+  SplitKView gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo);
   // act[M][F] = T(silu(x . gate^T) * (x . up^T))
   void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
   bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists);
 
-  void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out) {
+  void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out,
+                    const ExpandArgs* expand = nullptr) {
     const poss_config& g = c->cfg;
     GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = g.vocab;
     float* lg = logits_out ? logits_out : c->b.logits;
@@ -184,7 +195,8 @@ struct Impl {
       launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
       n_lists = c->n_chunks;
     }
-    launch_topk_merge(L, rows, K, n_lists, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp);
+    launch_topk_merge(L, rows, K, n_lists, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, ids, logp, &c->b.ts, expand,
+                      c->b.merge_done);
   }
 
   // fc + norm + K/V(+Q) projection + rotary + cache append for one batch of a specialist
@@ -195,28 +207,34 @@ struct Impl {
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
     launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), W(c->embed), H, A(b.X));
     GemmSegs fc; fc.n = 1; fc.w[0] = lw.fc_w; fc.rows[0] = H;
-    gemm(A(b.X), 2 * H, s.M, fc, 2 * H, W(lw.fc_b), nullptr, 0, b.h0, H);
-    launch_rmsnorm<T>(L, b.h0, s.M, H, W(lw.norm_in), g.rms_eps, A(b.xn));
+    SplitKView v_fc = gemm_view(A(b.X), 2 * H, s.M, fc, 2 * H, b.ptmp, H);
+    launch_reduce_norm<T>(L, v_fc, s.M, H, W(lw.fc_b), nullptr, W(lw.norm_in), g.rms_eps, b.h0, A(b.xn));
     GemmSegs qkv; qkv.n = 3;
     qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
-    gemm(A(b.xn), H, s.M, qkv, H, nullptr, nullptr, 0, b.qkv, qd + 2 * kd);
+    SplitKView v_qkv = gemm_view(A(b.xn), H, s.M, qkv, H, b.ptmp, qd + 2 * kd);
     RopeArgs ra;
+    ra.inv_freq = b.rope_inv;
     ra.mode = 0; ra.s = s; ra.base = 0; ra.depth = nullptr; ra.rows = s.M; ra.q_rows = with_q ? s.Mc : 0;
     ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.draft_kv_slots; ra.theta = g.rope_theta;
-    launch_rope_append<T>(L, ra, b.qkv, kcache, vcache, A(b.q));
+    launch_rope_append<T>(L, ra, v_qkv, kcache, vcache, A(b.q));
   }
 
-  // attention output -> O-proj + residual -> MLP + residual; x0 = layer input rows, result in `out`
-  void layer_tail(const poss_layer_w& lw, const float* x0, int rows, float* out, T* out_act = nullptr) {
+  // attention output -> O-proj + residual -> MLP + residual; x0 = layer input rows.  The result
+  // out = h1 + down(...) is stored in fp32; next_gain != NULL also writes out_act = T(rmsnorm(out) * gain)
+  // (the next layer's input norm or the final norm), next_gain == NULL writes out_act = T(out) if given.
+  void layer_tail(const poss_layer_w& lw, const float* x0, int rows, float* out, T* out_act = nullptr,
+                  const T* next_gain = nullptr) {
     const poss_config& g = c->cfg;
     Buffers& b = c->b;
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, F = g.ffn;
     GemmSegs so; so.n = 1; so.w[0] = lw.wo; so.rows[0] = H;
-    gemm(A(b.o), qd, rows, so, qd, nullptr, x0, H, b.h1, H);
-    launch_rmsnorm<T>(L, b.h1, rows, H, W(lw.norm_post), g.rms_eps, A(b.u));
+    SplitKView v_o = gemm_view(A(b.o), qd, rows, so, qd, b.ptmp, H);
+    launch_reduce_norm<T>(L, v_o, rows, H, nullptr, x0, W(lw.norm_post), g.rms_eps, b.h1, A(b.u));
     gemm_swiglu(A(b.u), rows, lw.w_gate, lw.w_up, F, H, A(b.act));
     GemmSegs sd; sd.n = 1; sd.w[0] = lw.w_down; sd.rows[0] = H;
-    gemm(A(b.act), F, rows, sd, F, nullptr, b.h1, H, out, H, 0, out_act);
+    SplitKView v_d = gemm_view(A(b.act), F, rows, sd, F, b.ptmp, H);
+    if (next_gain) launch_reduce_norm<T>(L, v_d, rows, H, nullptr, b.h1, next_gain, g.rms_eps, out, out_act);
+    else launch_splitk_reduce<T>(L, v_d, rows, H, nullptr, b.h1, H, out, H, out_act);
   }
 
   int draft_prefill(void* draft_kv, int start, const int32_t* tokens, const void* features, int n) {
@@ -269,8 +287,10 @@ struct Impl {
       float* fo = b.fout + (size_t)i * KMAX * H;
       T* fbi = A(b.fb) + (size_t)i * KMAX * H;
       layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo, fbi);
-      lm_head_topk(fbi, sr.Mc, K, b.top_ids, b.top_logp, nullptr);
-      launch_expand(L, b.ts, KMAX, i, sr.Mc, K, cand_base, i == depth - 1, b.top_ids, b.top_logp);
+      ExpandArgs xa;
+      xa.enabled = 1; xa.Kmax = KMAX; xa.step = i; xa.Mc = sr.Mc; xa.K = K; xa.cand_base = cand_base;
+      xa.last = i == depth - 1;
+      lm_head_topk(fbi, sr.Mc, K, b.top_ids, b.top_logp, nullptr, &xa);
       cand_base += sr.Mc * K;
     }
     // specialists the round did not reach still cache the verified pairs
@@ -308,27 +328,31 @@ struct Impl {
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
     size_t per_layer = (size_t)2 * g.n_kv_heads * g.target_kv_slots * g.head_dim;
     launch_embed_rows<T>(L, tokens, rows, W(c->embed), H, b.hx);
+    launch_rmsnorm<T>(L, b.hx, rows, H, W(c->tgt[0].norm_in), g.rms_eps, A(b.xn));
     for (int li = 0; li < g.n_target_layers; ++li) {
       const poss_layer_w& lw = c->tgt[li];
       T* kc = A(target_kv) + li * per_layer;
       T* vc = kc + per_layer / 2;
-      launch_rmsnorm<T>(L, b.hx, rows, H, W(lw.norm_in), g.rms_eps, A(b.xn));
       GemmSegs qkv; qkv.n = 3;
       qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
-      gemm(A(b.xn), H, rows, qkv, H, nullptr, nullptr, 0, b.qkv, qd + 2 * kd);
+      SplitKView v_qkv = gemm_view(A(b.xn), H, rows, qkv, H, b.ptmp, qd + 2 * kd);
       RopeArgs ra;
+      ra.inv_freq = b.rope_inv;
       ra.mode = 1; ra.base = prefix_len; ra.depth = depth; ra.rows = rows; ra.q_rows = rows;
       ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.target_kv_slots;
       ra.theta = g.rope_theta; memset(&ra.s, 0, sizeof(ra.s));
-      launch_rope_append<T>(L, ra, b.qkv, kc, vc, A(b.q));
+      launch_rope_append<T>(L, ra, v_qkv, kc, vc, A(b.q));
       AttnArgs aa;
       aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.target_kv_slots;
       aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = mask_words;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
       run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
-      layer_tail(lw, b.hx, rows, b.hx);
+      // the layer's last reduction also applies the norm that follows it: the next layer's input
+      // norm, or the final norm (whose output is the feature)
+      const bool last = li == g.n_target_layers - 1;
+      const T* next_gain = last ? W(c->final_norm) : W(c->tgt[li + 1].norm_in);
+      layer_tail(lw, b.hx, rows, b.hx, last ? A(out_features) : A(b.xn), next_gain);
     }
-    launch_rmsnorm<T>(L, b.hx, rows, H, W(c->final_norm), g.rms_eps, A(out_features));
     if (out_argmax || out_logits)
       lm_head_topk(A(out_features), rows, 1, out_argmax ? out_argmax : b.argmax_tmp, b.top_logp, out_logits);
     return L.err;
@@ -355,6 +379,29 @@ void Impl<bf16>::gemm(const bf16* x, int ldx, int M, const GemmSegs& segs, int K
     launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
     if (out_act) launch_cast_rows<bf16>(L, out, (size_t)M * ldo, out_act);
   }
+}
+
+template <typename T>
+SplitKView Impl<T>::gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo) {
+  launch_gemm_simt<T>(L, x, ldx, M, segs, K, nullptr, nullptr, 0, tmp, ldo);
+  SplitKView v;
+  memset(&v, 0, sizeof(v));
+  v.direct = tmp; v.ld = ldo;
+  return v;
+}
+template <>
+SplitKView Impl<bf16>::gemm_view(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo) {
+  SplitKView v;
+  memset(&v, 0, sizeof(v));
+  v.direct = tmp; v.ld = ldo;
+  if (tc_gemm_supported(segs, K, ldx, M)) {
+    TcEpilogue ep;
+    ep.mode = TC_EPI_STORE; ep.out = tmp; ep.ldo = ldo; ep.view = &v;
+    launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, ep, c->b.tc_scratch, c->b.status);
+  } else {
+    launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, nullptr, nullptr, 0, tmp, ldo);
+  }
+  return v;
 }
 
 template <typename T>
@@ -443,6 +490,9 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   c->tc = tc_plan_cache_create();
   cudaStream_t st = S(stream);
   bool ok = cudaMemsetAsync(workspace, 0, bp.off, st) == cudaSuccess;
+  double inv[64];
+  for (int j = 0; j < 64; ++j) inv[j] = pow((double)cfg->rope_theta, -2.0 * j / (double)cfg->head_dim);
+  ok = ok && cudaMemcpyAsync(c->b.rope_inv, inv, sizeof(inv), cudaMemcpyHostToDevice, st) == cudaSuccess;
   Launcher L; L.stream = st; L.launches = &c->launches; L.err = POSS_OK;
   launch_chain_mask(L, c->b.chain_mask, c->b.chain_depth, R);
   ok = ok && L.err == POSS_OK && cudaStreamSynchronize(st) == cudaSuccess;
@@ -640,8 +690,16 @@ int poss_linear(poss_ctx* c, const void* x, int M, const void* w, int N, int K, 
   GemmSegs sg; sg.n = 1; sg.w[0] = w; sg.rows[0] = N;
   if (c->cfg.dtype == POSS_BF16) {
     Impl<bf16> im(c, stream);
-    im.gemm(reinterpret_cast<const bf16*>(x), K, M, sg, K, reinterpret_cast<const bf16*>(bias), residual, N, out, N,
-            impl);
+    const bf16* xb = reinterpret_cast<const bf16*>(x);
+    bool can_tc = tc_gemm_supported(sg, K, K, M);
+    if (impl == 2 && !can_tc) return POSS_E_SHAPE;
+    if (impl != 1 && can_tc) {
+      // the product as the round uses it: split-K partials (or the plain product in `out`) + a reducing consumer
+      SplitKView v = im.gemm_view(xb, K, M, sg, K, out, N);
+      launch_splitk_reduce<bf16>(im.L, v, M, N, reinterpret_cast<const bf16*>(bias), residual, N, out, N, nullptr);
+    } else {
+      im.gemm(xb, K, M, sg, K, reinterpret_cast<const bf16*>(bias), residual, N, out, N, 1);
+    }
     return im.L.err;
   }
   if (impl == 2) return POSS_E_SHAPE;

@@ -71,6 +71,103 @@ struct Launcher {
   int err;  // sticky poss_status
 };
 
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_enter(): it lets the next
+// kernel of the stream be scheduled early (that kernel's own pdl_enter, or the GEMM's weight prefetch,
+// then overlaps this kernel's tail) and waits until the previous kernel has completed and its writes are
+// visible.  Because every kernel waits before it touches memory, completion is transitive along the
+// stream and the usual stream-order guarantees hold.  One consequence for the kernels' signatures: a
+// kernel is alive while its predecessor still writes, so nothing a predecessor produces may be read
+// through the read-only data path.  Pointers to activations, indices and caches therefore carry no
+// `const __restrict__` pair (the compiler would turn their loads into non-coherent ones and could hoist
+// them above the wait); only weights, which no kernel writes, may.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(Launcher& L, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  ++*L.launches;
+  if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) L.err = POSS_E_CUDA;
+}
+
+// ------------------------------------------------------------------ split-K results left for the consumer
+// The tensor-core GEMM cuts the (tile, k-block) sequence of a product into one contiguous range per
+// CTA.  For products with few tiles it does not reduce the ranges itself: every CTA parks the fp32
+// partial of each tile segment it computed (128 weight rows x Npad activation rows) in scratch, and
+// the kernel that consumes the product (norm, rotary embedding, plain reduce) adds a tile's partials
+// in range order while it loads.  That reduction is spread over all of the consumer's blocks instead of
+// running in the last CTA of each tile.  A view with deferred == 0 is a plain fp32 matrix.
+//
+// Units are k-blocks in (tile, k-block) order; CTA c owns [range_begin(c), range_begin(c + 1)).  A CTA
+// holds at most two segments here (its range is not longer than a tile): slot 0 is the segment that
+// starts at the range's first unit, slot 1 the one that starts at a tile boundary inside the range.
+struct SplitKView {
+  const float* scratch;   // partial of (cta, slot): scratch + (cta * 2 + slot) * Npad * 128, element [m][row in tile]
+  const float* direct;    // deferred == 0: the product itself, [M][ld]
+  int ld;
+  int deferred, Npad, G, kb_total, n_tiles;
+  int seg_tiles[3], seg_rows[3];   // tiles / rows of each weight segment (tiles never straddle segments)
+  int n_segs;
+};
+
+__host__ __device__ __forceinline__ long long splitk_range_begin(long long c, long long groups, int G, int gran) {
+  return (c * groups / G) * gran;
+}
+// the CTA whose range contains unit u
+__host__ __device__ __forceinline__ int splitk_cta_of_unit(long long u, long long groups, int G, int gran) {
+  long long g = u / gran;                       // group of the unit
+  // largest c with floor(c * groups / G) <= g  <=>  c * groups < (g + 1) * G
+  long long c = ((g + 1) * G + groups - 1) / groups - 1;
+  if (c > G - 1) c = G - 1;
+  return (int)c;
+}
+
+// Contributors of one tile: CTAs c_first .. c_first + count - 1; the first one's partial sits in
+// slot_first, every later one's in slot 0.
+struct TileContrib { int c_first, count, slot_first; };
+__device__ __forceinline__ TileContrib splitk_tile_contrib(const SplitKView& v, int tile) {
+  long long groups = (long long)v.n_tiles * v.kb_total;
+  long long tile_u0 = (long long)tile * v.kb_total;
+  TileContrib t;
+  t.c_first = splitk_cta_of_unit(tile_u0, groups, v.G, 1);
+  int c_last = splitk_cta_of_unit(tile_u0 + v.kb_total - 1, groups, v.G, 1);
+  t.count = c_last - t.c_first + 1;
+  t.slot_first = splitk_range_begin(t.c_first, groups, v.G, 1) >= tile_u0 ? 0 : 1;
+  return t;
+}
+// tile and row-in-tile of output column n (columns of the segments are laid side by side)
+__device__ __forceinline__ void splitk_locate(const SplitKView& v, int n, int* tile, int* t) {
+  int base_tile = 0, nn = n;
+  for (int s = 0; s < v.n_segs - 1 && nn >= v.seg_rows[s]; ++s) { nn -= v.seg_rows[s]; base_tile += v.seg_tiles[s]; }
+  *tile = base_tile + nn / 128;
+  *t = nn % 128;
+}
+// four consecutive columns n .. n+3 of row m (n a multiple of 4, so they share a tile), partials added in
+// range order
+__device__ __forceinline__ float4 splitk_load4(const SplitKView& v, int m, int n, const TileContrib& tc, int t) {
+  if (!v.deferred) return *reinterpret_cast<const float4*>(v.direct + (size_t)m * v.ld + n);
+  const size_t part = (size_t)v.Npad * 128;
+  const float* p = v.scratch + ((size_t)tc.c_first * 2 + tc.slot_first) * part + (size_t)m * 128 + t;
+  float4 acc = __ldcg(reinterpret_cast<const float4*>(p));
+  for (int i = 1; i < tc.count; ++i) {
+    const float* pi = v.scratch + ((size_t)(tc.c_first + i) * 2) * part + (size_t)m * 128 + t;
+    float4 x = __ldcg(reinterpret_cast<const float4*>(pi));
+    acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+  }
+  return acc;
+}
+
 template <typename T>
 void launch_gemm_simt(Launcher& L, const T* X, int ldx, int M, const GemmSegs& segs, int K, const T* bias,
                       const float* residual, int ldr, float* out, int ldo);
@@ -89,6 +186,7 @@ template <typename T>
 void launch_silu_mul(Launcher& L, const float* gu, int rows, int F, T* out);
 
 struct RopeArgs {
+  const double* inv_freq;  // [d/2] theta^(-2j/d), filled at init
   int mode;        // 0 = draft step rows (StepRows mapping), 1 = target rows (slot = base + r, pos = base + depth[r])
   StepRows s;
   int base;
@@ -98,7 +196,15 @@ struct RopeArgs {
   float theta;
 };
 template <typename T>
-void launch_rope_append(Launcher& L, const RopeArgs& a, const float* qkv, T* kcache, T* vcache, T* qout);
+void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout);
+// h[m][n] (fp32) = product + bias[n] + residual[m][n];  xn[m][n] = T(gain[n] * h / rms(h row))  (gain NULL: xn = T(h))
+template <typename T>
+void launch_reduce_norm(Launcher& L, const SplitKView& prod, int rows, int H, const T* bias, const float* residual,
+                        const T* gain, float eps, float* h, T* xn);
+// out[m][n] (fp32, may be NULL) = product + bias[n] + residual[m][n]; out_act (may be NULL) the same in T
+template <typename T>
+void launch_splitk_reduce(Launcher& L, const SplitKView& prod, int rows, int N, const T* bias, const float* residual,
+                          int ldr, float* out, int ldo, T* out_act);
 
 struct AttnArgs {
   int rows, Hq, Hkv, d, cap;
@@ -129,11 +235,14 @@ void launch_tree_attention_mma(Launcher& L, const AttnArgs& a, const bf16* q, co
 #define POSS_TOPK_CHUNK 2048
 void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int K, float* pmax, float* psum,
                          float* pval, int32_t* pidx, int n_chunks);
-void launch_topk_merge(Launcher& L, int rows, int K, int n_chunks, const float* pmax, const float* psum,
-                       const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp);
+// Tree expansion run by the merge kernel's last block (enabled = 0: merge only)
+struct ExpandArgs {
+  int enabled, Kmax, step, Mc, K, cand_base, last;
+};
+void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* pmax, const float* psum,
+                       const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp,
+                       const TreeState* ts = nullptr, const ExpandArgs* x = nullptr, int* done = nullptr);
 
-void launch_expand(Launcher& L, const TreeState& ts, int Kmax, int step, int Mc, int K, int cand_base, int last,
-                   const int32_t* top_ids, const float* top_logp);
 void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, int root_tok_index,
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes);
