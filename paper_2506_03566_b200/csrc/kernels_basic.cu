@@ -416,7 +416,7 @@ template void launch_splitk_reduce<bf16>(Launcher&, const SplitKView&, int, int,
 // cosine of the reduced angle are then taken in fp32.  One block per row; a work item is four
 // neighbouring pairs of one head (two 16-byte loads) or four values.
 template <typename T>
-__global__ void __launch_bounds__(256) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache, T* qout) {
+__global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache, T* qout) {
   __shared__ TileContrib tab[512];
   __shared__ float cs[64], sn[64];
   pdl_enter();
@@ -451,6 +451,7 @@ __global__ void __launch_bounds__(256) k_rope_append(RopeArgs a, SplitKView qkv,
   const int n_qitems = with_q ? a.Hq * per_head : 0;
   const int n_kitems = a.Hkv * per_head;
   const int n_vitems = kd / 4;
+#pragma unroll 2
   for (int i = threadIdx.x; i < n_qitems + n_kitems + n_vitems; i += blockDim.x) {
     if (i < n_qitems + n_kitems) {
       const bool is_q = i < n_qitems;
@@ -477,7 +478,7 @@ __global__ void __launch_bounds__(256) k_rope_append(RopeArgs a, SplitKView qkv,
 template <typename T>
 void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {
   if (a.rows <= 0) return;
-  launch_pdl(L, k_rope_append<T>, dim3(a.rows), dim3(256), 0, a, qkv, kcache, vcache, qout);
+  launch_pdl(L, k_rope_append<T>, dim3(a.rows), dim3(512), 0, a, qkv, kcache, vcache, qout);
 }
 template void launch_rope_append<float>(Launcher&, const RopeArgs&, const SplitKView&, float*, float*, float*);
 template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKView&, bf16*, bf16*, bf16*);

@@ -101,6 +101,84 @@ void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int 
   launch_pdl(L, k_topk_partial, grid, dim3(256), 0, logits, V, K, pmax, psum, pval, pidx, n_chunks);
 }
 
+// ------------------------------------------------------------------ row argmax partials straight from the logits
+// Block (chunk, row): the best (value, lowest id) of POSS_ARGMAX_CHUNK consecutive logits, written in the
+// partial-list format of the merge kernel with K = 1 (max = the value, sum = 1).  bf16 logits are read
+// as they are (16-byte loads), never widened to a second buffer.
+template <typename T>
+__global__ void __launch_bounds__(256) k_argmax_partial(const T* logits, int V, float* pmax, float* psum, float* pval,
+                                                        int32_t* pidx, int n_chunks) {
+  __shared__ float wv[8];
+  __shared__ int wi[8];
+  pdl_enter();
+  const int chunk = blockIdx.x, row = blockIdx.y;
+  const int lo = chunk * POSS_ARGMAX_CHUNK;
+  const int n = min(POSS_ARGMAX_CHUNK, V - lo);
+  const T* src = logits + (size_t)row * V + lo;
+  constexpr int PER = 16 / sizeof(T);
+  float bv = NEG_INF;
+  int bi = 0x7fffffff;
+  const bool vec = (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+  if (vec) {
+    const int n_vec = n / PER;
+    const uint4* s4 = reinterpret_cast<const uint4*>(src);
+    for (int base = 0; base < n_vec; base += 256 * 4) {
+      uint4 raw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int i = base + u * 256 + threadIdx.x;
+        if (i < n_vec) raw[u] = s4[i];
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int i = base + u * 256 + threadIdx.x;
+        if (i < n_vec) {
+          const T* e = reinterpret_cast<const T*>(&raw[u]);
+#pragma unroll
+          for (int q = 0; q < PER; ++q) {
+            float v = to_f(e[q]);
+            int id = i * PER + q;
+            if (better(v, id, bv, bi)) { bv = v; bi = id; }
+          }
+        }
+      }
+    }
+    for (int i = n_vec * PER + threadIdx.x; i < n; i += 256) {
+      float v = to_f(src[i]);
+      if (better(v, i, bv, bi)) { bv = v; bi = i; }
+    }
+  } else {
+    for (int i = threadIdx.x; i < n; i += 256) {
+      float v = to_f(src[i]);
+      if (better(v, i, bv, bi)) { bv = v; bi = i; }
+    }
+  }
+  warp_best(bv, bi);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float v = wv[0];
+    int i = wi[0];
+    for (int w = 1; w < 8; ++w) if (better(wv[w], wi[w], v, i)) { v = wv[w]; i = wi[w]; }
+    size_t pc = (size_t)row * n_chunks + chunk;
+    pmax[pc] = v;
+    psum[pc] = 1.f;
+    pval[pc] = v;
+    pidx[pc] = i == 0x7fffffff ? i : lo + i;
+  }
+}
+template <typename T>
+int launch_argmax_partial(Launcher& L, const T* logits, int rows, int V, float* pmax, float* psum, float* pval,
+                          int32_t* pidx) {
+  int n_chunks = (V + POSS_ARGMAX_CHUNK - 1) / POSS_ARGMAX_CHUNK;
+  if (rows <= 0) return n_chunks;
+  launch_pdl(L, k_argmax_partial<T>, dim3(n_chunks, rows), dim3(256), 0, logits, V, pmax, psum, pval, pidx, n_chunks);
+  return n_chunks;
+}
+template int launch_argmax_partial<float>(Launcher&, const float*, int, int, float*, float*, float*, int32_t*);
+template int launch_argmax_partial<bf16>(Launcher&, const bf16*, int, int, float*, float*, float*, int32_t*);
+
 // ------------------------------------------------------------------ tree expansion after draft step `step`
 // Rows r = 0..Mc-1 are the level-`step` frontier.  Appends Mc*K level-(step+1) candidates in
 // (row, rank) order with score = row score + logp, then (unless last) picks the K best of them as the
@@ -164,9 +242,24 @@ __global__ void __launch_bounds__(128) k_topk_merge(int K, int n_lists, const fl
   const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* rmax = pmax + (size_t)row * n_lists;
   const float* rsum = psum + (size_t)row * n_lists;
-  for (int i = threadIdx.x; i < n_lists * K; i += 128) {
-    vals[i] = pval[(size_t)row * n_lists * K + i];
-    idxs[i] = pidx[(size_t)row * n_lists * K + i];
+  {
+    const float* pv = pval + (size_t)row * n_lists * K;
+    const int32_t* pi = pidx + (size_t)row * n_lists * K;
+    const int n = n_lists * K;
+    for (int base = 0; base < n; base += 128 * 8) {      // eight loads of each kind in flight per thread
+      float v[8];
+      int x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        int i = base + u * 128 + threadIdx.x;
+        if (i < n) { v[u] = __ldcg(pv + i); x[u] = __ldcg(pi + i); }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        int i = base + u * 128 + threadIdx.x;
+        if (i < n) { vals[i] = v[u]; idxs[i] = x[u]; }
+      }
+    }
   }
   float gm = NEG_INF;
   for (int c = threadIdx.x; c < n_lists; c += 128) { gm = fmaxf(gm, rmax[c]); heads[c] = 0; }
@@ -324,45 +417,65 @@ void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int tota
              out_parents, out_scores, out_depth, out_mask, out_n_nodes);
 }
 
-// ------------------------------------------------------------------ greedy accept walk (one warp) + hand-over pairs
+// ------------------------------------------------------------------ greedy accept walk + hand-over pairs
+// One block.  The tree (tokens, parents) and the target's greedy tokens are staged in shared memory,
+// warp 0 walks (every step scans all nodes for the child that carries the wanted token, lowest node
+// index first), then the whole block copies the accepted rows' features with 16-byte accesses.
 template <typename T>
-__global__ void __launch_bounds__(32) k_accept_walk(const int32_t* g, const T* feats,
-                                                    int H, const int32_t* tokens,
-                                                    const int32_t* parents, int rows, int max_depth,
-                                                    int32_t* out_path, int32_t* out_a,
-                                                    int32_t* out_bonus,
-                                                    int32_t* out_new_tokens,
-                                                    T* out_new_features,
-                                                    unsigned long long* counters) {
+__global__ void __launch_bounds__(256) k_accept_walk(const int32_t* g, const T* feats, int H, const int32_t* tokens,
+                                                     const int32_t* parents, int rows, int max_depth,
+                                                     int32_t* out_path, int32_t* out_a, int32_t* out_bonus,
+                                                     int32_t* out_new_tokens, T* out_new_features,
+                                                     unsigned long long* counters) {
+  __shared__ int s_tok[256], s_par[256], s_g[256];
   __shared__ int path[POSS_MAX_DEPTH + 1];
+  __shared__ int s_a;
   pdl_enter();
-  int lane = threadIdx.x;
-  int cur = 0, a = 0;
-  if (lane == 0) path[0] = 0;
-  while (a < max_depth) {
-    int want = g[cur];
-    int found = 0x7fffffff;
-    for (int c = 1 + lane; c < rows; c += 32)
-      if (parents[c] == cur && tokens[c] == want) found = min(found, c);
-    for (int off = 16; off > 0; off >>= 1) found = min(found, __shfl_xor_sync(0xffffffffu, found, off));
-    if (found == 0x7fffffff) break;
-    cur = found;
-    ++a;
-    if (lane == 0) path[a] = cur;
+  for (int i = threadIdx.x; i < rows; i += blockDim.x) { s_tok[i] = tokens[i]; s_par[i] = parents[i]; s_g[i] = g[i]; }
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x < 32) {
+    int cur = 0, a = 0;
+    if (lane == 0) path[0] = 0;
+    while (a < max_depth) {
+      int want = s_g[cur];
+      int found = 0x7fffffff;
+      for (int c = 1 + lane; c < rows; c += 32)
+        if (s_par[c] == cur && s_tok[c] == want) found = min(found, c);
+      for (int off = 16; off > 0; off >>= 1) found = min(found, __shfl_xor_sync(0xffffffffu, found, off));
+      if (found == 0x7fffffff) break;
+      cur = found;
+      ++a;
+      if (lane == 0) path[a] = cur;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      s_a = a;
+      out_a[0] = a;
+      out_bonus[0] = s_g[cur];
+      atomicAdd(&counters[0], 1ull);                         // rounds
+      for (int i = 1; i <= a; ++i) atomicAdd(&counters[i], 1ull);   // N_i
+    }
+    for (int i = lane; i <= POSS_MAX_DEPTH; i += 32) out_path[i] = i <= a ? path[i] : -1;
+    for (int k = lane; k <= a; k += 32) out_new_tokens[k] = k < a ? s_tok[path[k + 1]] : s_g[cur];
   }
-  __syncwarp();
-  if (lane == 0) {
-    out_a[0] = a;
-    out_bonus[0] = g[cur];
-    atomicAdd(&counters[0], 1ull);                         // rounds
-    for (int i = 1; i <= a; ++i) atomicAdd(&counters[i], 1ull);   // N_i
-  }
-  for (int i = lane; i <= POSS_MAX_DEPTH; i += 32) out_path[i] = i <= a ? path[i] : -1;
-  for (int k = lane; k <= a; k += 32) out_new_tokens[k] = k < a ? tokens[path[k + 1]] : g[cur];
-  for (int k = 0; k <= a; ++k) {
-    const T* src = feats + (size_t)path[k] * H;
-    T* dst = out_new_features + (size_t)k * H;
-    for (int i = lane; i < H; i += 32) dst[i] = src[i];
+  __syncthreads();
+  const int a = s_a;
+  constexpr int PER = 16 / sizeof(T);
+  const bool vec = (H % PER) == 0 &&
+                   ((reinterpret_cast<uintptr_t>(feats) | reinterpret_cast<uintptr_t>(out_new_features)) & 15) == 0;
+  if (vec) {
+    const int per_row = H / PER;
+    for (int i = threadIdx.x; i < (a + 1) * per_row; i += blockDim.x) {
+      int k = i / per_row, e = i % per_row;
+      reinterpret_cast<uint4*>(out_new_features + (size_t)k * H)[e] =
+          reinterpret_cast<const uint4*>(feats + (size_t)path[k] * H)[e];
+    }
+  } else {
+    for (int i = threadIdx.x; i < (a + 1) * H; i += blockDim.x) {
+      int k = i / H, e = i % H;
+      out_new_features[(size_t)k * H + e] = feats[(size_t)path[k] * H + e];
+    }
   }
 }
 template <typename T>
@@ -370,7 +483,7 @@ void launch_accept_walk(Launcher& L, const int32_t* g, const T* feats, int H, co
                         const int32_t* parents, int rows, int max_depth, int32_t* out_path, int32_t* out_a,
                         int32_t* out_bonus, int32_t* out_new_tokens, T* out_new_features,
                         unsigned long long* counters) {
-  launch_pdl(L, k_accept_walk<T>, dim3(1), dim3(32), 0, g, feats, H, tokens, parents, rows, max_depth, out_path, out_a,
+  launch_pdl(L, k_accept_walk<T>, dim3(1), dim3(256), 0, g, feats, H, tokens, parents, rows, max_depth, out_path, out_a,
              out_bonus, out_new_tokens, out_new_features, counters);
 }
 template void launch_accept_walk<float>(Launcher&, const int32_t*, const float*, int, const int32_t*, const int32_t*,

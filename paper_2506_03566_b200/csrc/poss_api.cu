@@ -595,17 +595,16 @@ int poss_verify_accept(poss_ctx* c, const void* target_logits, const int32_t* ta
   const poss_config& cf = c->cfg;
   if (target_logits) {
     if (rows > R) return POSS_E_CAPACITY;
-    // row argmax over the vocabulary with the same chunked top-1 kernels (ties -> lowest id)
-    const float* lg;
-    if (cf.dtype == POSS_BF16) {
-      launch_widen_bf16(L, reinterpret_cast<const bf16*>(target_logits), (size_t)rows * cf.vocab, c->b.logits);
-      lg = c->b.logits;
-    } else {
-      lg = reinterpret_cast<const float*>(target_logits);
-    }
-    launch_topk_partial(L, lg, rows, cf.vocab, 1, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
-    launch_topk_merge(L, rows, 1, c->n_chunks, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->b.argmax_tmp,
-                      c->b.top_logp);
+    // row argmax over the vocabulary: per-chunk best (ties -> lowest id) read straight from the logits,
+    // then the list merge
+    int n_lists;
+    if (cf.dtype == POSS_BF16)
+      n_lists = launch_argmax_partial<bf16>(L, reinterpret_cast<const bf16*>(target_logits), rows, cf.vocab, c->b.pmax,
+                                            c->b.psum, c->b.pval, c->b.pidx);
+    else
+      n_lists = launch_argmax_partial<float>(L, reinterpret_cast<const float*>(target_logits), rows, cf.vocab,
+                                             c->b.pmax, c->b.psum, c->b.pval, c->b.pidx);
+    launch_topk_merge(L, rows, 1, n_lists, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->b.argmax_tmp, c->b.top_logp);
     g = c->b.argmax_tmp;
   }
   if (cf.dtype == POSS_BF16)

@@ -158,12 +158,27 @@ __device__ __forceinline__ void splitk_locate(const SplitKView& v, int n, int* t
 __device__ __forceinline__ float4 splitk_load4(const SplitKView& v, int m, int n, const TileContrib& tc, int t) {
   if (!v.deferred) return *reinterpret_cast<const float4*>(v.direct + (size_t)m * v.ld + n);
   const size_t part = (size_t)v.Npad * 128;
-  const float* p = v.scratch + ((size_t)tc.c_first * 2 + tc.slot_first) * part + (size_t)m * 128 + t;
-  float4 acc = __ldcg(reinterpret_cast<const float4*>(p));
-  for (int i = 1; i < tc.count; ++i) {
-    const float* pi = v.scratch + ((size_t)(tc.c_first + i) * 2) * part + (size_t)m * 128 + t;
-    float4 x = __ldcg(reinterpret_cast<const float4*>(pi));
-    acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+  const float* p0 = v.scratch + (size_t)m * 128 + t;
+  // all loads of a batch are issued before the first add (the adds stay in range order)
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int base = 0; base < tc.count; base += 8) {
+    float4 x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int k = base + i;
+      if (k < tc.count) {
+        size_t slot = (size_t)(tc.c_first + k) * 2 + (k == 0 ? tc.slot_first : 0);
+        x[i] = __ldcg(reinterpret_cast<const float4*>(p0 + slot * part));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int k = base + i;
+      if (k < tc.count) {
+        if (k == 0) acc = x[i];
+        else { acc.x += x[i].x; acc.y += x[i].y; acc.z += x[i].z; acc.w += x[i].w; }
+      }
+    }
   }
   return acc;
 }
@@ -233,6 +248,11 @@ void launch_tree_attention_mma(Launcher& L, const AttnArgs& a, const bf16* q, co
                                float* part, bf16* out);
 
 #define POSS_TOPK_CHUNK 2048
+#define POSS_ARGMAX_CHUNK 8192
+// per-chunk argmax of fp32 or bf16 logits in the merge kernel's partial format (K = 1); returns the chunk count
+template <typename T>
+int launch_argmax_partial(Launcher& L, const T* logits, int rows, int V, float* pmax, float* psum, float* pval,
+                          int32_t* pidx);
 void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int K, float* pmax, float* psum,
                          float* pval, int32_t* pidx, int n_chunks);
 // Tree expansion run by the merge kernel's last block (enabled = 0: merge only)
