@@ -110,6 +110,10 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--config", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--alias-specialists", action="store_true",
+                    help="profiler captures only: all specialists share one weight set, so the process holds "
+                         "about 3 GB instead of 10 GB; the launch chain and every launch's traffic are unchanged "
+                         "(one step still streams 1.56 GB, far more than L2)")
     args = ap.parse_args()
 
     import poss_synth as ps
@@ -137,7 +141,7 @@ def main():
 
     # ---------------- inputs: seeded, host-generated, resident in HBM before timing
     seed = 1 + rank          # replicas only: every rank runs an independent request
-    w = ps.make_weights(cfg, seed)
+    w = ps.make_weights(cfg, seed, alias_specialists=args.alias_specialists)
     rows = cfg.total + 1
     cap = cfg.prefix + 8 + cfg.tree_slots
     P = Poss(make_config(cfg, cap), w)

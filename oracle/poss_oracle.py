@@ -292,6 +292,11 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
     forcing of values, so that a comparison is per step and rounding noise does not pile up over
     the depth: follow["features"][i] ([Mc][H]) replaces this step's output features as the input of
     the children, and follow["cand_scores"] (flat) replaces the parents' cumulative scores.
+    With follow["force_head_input"] the forced feature of step i is also what this step's LM head reads, so
+    the head stage is checked on identical inputs while the feature itself is compared separately (a
+    feature of magnitude 16..64 has a bf16 spacing of 2^-4..2^-2: two features that agree to 1e-2
+    still round differently in a few percent of their elements, which moves logits of magnitude ~70
+    by more than any fixed absolute tolerance).
     """
     S, n, K = cfg.S, cfg.n, topk
     H = cfg.hidden
@@ -360,7 +365,8 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
         forced_f = None if follow is None or "features" not in follow else np.asarray(follow["features"][i], dtype=num.dtype)
         for r, nd in enumerate(current):
             nd.fout = fout[r] if forced_f is None else forced_f[r]
-        logits = linear(fout, w["lm_head"], num)
+        head_in = forced_f if forced_f is not None and follow.get("force_head_input") else fout
+        logits = linear(head_in, w["lm_head"], num)
         logp = log_softmax_rows(logits)
         own_ids = topk_rows(logits, K)
         srt = -np.sort(-logits, axis=-1)

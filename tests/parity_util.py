@@ -8,7 +8,9 @@ Rules (written here, used by every parity test):
     about one bf16 unit per rounding boundary, and that noise grows with the draft depth, so the
     numeric comparison is PER STEP WITH TEACHER FORCING: the oracle is re-run following the GPU's
     decisions and taking the GPU's previous-step features and parent scores as inputs (all arithmetic
-    of the step is the oracle's own).  Every GPU decision must be valid up to the margin under the
+    of the step is the oracle's own).  The step's two stages are compared separately: the feature against
+    the oracle's feature from the previous step's inputs, the LM head / log-softmax / top-k against the
+    oracle's head applied to the GPU's feature of the same step.  Every GPU decision must be valid up to the margin under the
     oracle's values; decisions that differ from the oracle's own choice are counted and reported.
 """
 from __future__ import annotations
@@ -119,7 +121,7 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
                 frontier.append(trace["frontier"][i])
         follow = {"top_ids": top_ids, "frontier": frontier, "selected": trace["selected"][: n - 1],
                   "features": [trace["step_features"][i, : (1 if i == 0 else K)] for i in range(depth)],
-                  "cand_scores": trace["cand_scores"]}
+                  "cand_scores": trace["cand_scores"], "force_head_input": True}
         kv_o = po.widen(kv_np, num.dtype).copy()
         fol = po.draft_round(cfg, w, kv_o, prefix_len, new_tok, new_feat, depth, K, T, num, keep_logits=True,
                              follow=follow)

@@ -1,0 +1,110 @@
+"""GPU parity at the full sizes of the named workloads, in the launch configuration bench.py times.
+
+Drafter-only workloads c2 (Llama-3-8B shape, 6 specialists, depth 6, 60 tokens, prefix 1024), c3
+(Llama-2-13B shape, 3 specialists x 2 positions, prefix 2048) and c4 (Llama-3-8B shape, prefix 8192,
+depth 8, 80 tokens, 4 specialists x 2): one draft round through the C ABI against the oracle (fp32
+arithmetic between the bf16 rounding points), under the same rules as the small cases: per-step
+teacher-forced features, log-probs and scores within 2e-2, every decision valid up to the 1e-2 margin.
+Plus the standalone verification stages at target geometry.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import poss_synth as ps
+from oracle import poss_oracle as po
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _poss(cfg, w, draft_slots):
+    from paper_2506_03566_b200 import Poss, make_config
+    return Poss(make_config(cfg, draft_slots), w)
+
+
+def _dev(a):
+    from paper_2506_03566_b200 import to_device
+    return to_device(a)
+
+
+@pytest.mark.parametrize("name,n_new,seed", [("c2", 1, 101), ("c3", 3, 102), ("c4", 2, 103)])
+def test_full_size_draft_round_matches_oracle(name, n_new, seed):
+    cfg = ps.CONFIGS[name]
+    w = ps.make_weights(cfg, seed)
+    cap = cfg.prefix + n_new + cfg.tree_slots
+    P = _poss(cfg, w, cap)
+    kv = ps.make_draft_kv(cfg, seed, cap)
+    tok, feat = ps.make_round_inputs(cfg, seed, n_new)
+    g, trace, dkv = pu.run_gpu_round(P, cfg, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total)
+    # same call again: ordered reductions only, so the bits repeat
+    g2, trace2, _ = pu.run_gpu_round(P, cfg, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total)
+    for k in ("tokens", "parents", "scores", "depth", "anc_mask"):
+        assert np.array_equal(g[k], g2[k]), k
+    assert np.array_equal(trace["step_features"], trace2["step_features"])
+    P.close()
+    del P
+    torch.cuda.empty_cache()
+    num = pu.oracle_num(cfg, big=True)
+    rep = pu.compare_round(cfg, w, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, g, trace, num, False)
+    pu.compare_kv(cfg, dkv, rep["kv_oracle"], cfg.prefix, cfg.prefix + n_new, pu.TOL[cfg.dtype])
+    print(name, {k: v for k, v in rep.items() if k != "kv_oracle"})
+    assert int(g["n_nodes"][0]) == cfg.total + 1
+
+
+@pytest.mark.parametrize("rows,P_len", [(61, 1024), (81, 8192)])
+def test_full_size_verification_attention_matches_oracle(rows, P_len):
+    """Target geometry of the Llama-3-8B shape: 32 query heads, 8 KV heads, head_dim 128."""
+    Hq, Hkv, d = 32, 8, 128
+    cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
+    P = _poss(cfg, ps.make_weights(cfg, 1), 64)
+    cap = P_len + rows
+    q, kv = ps.make_attention_case(7, rows, Hq, Hkv, d, P_len, cap, "bf16")
+    parents = ps.random_tree_parents(8, rows)
+    mask = po.pack_mask(po.ancestor_matrix(parents))
+    scale = 1.0 / math.sqrt(d)
+    got = pu.np_of(P.poss_tree_attention(_dev(q), _dev(kv), P_len, torch.from_numpy(mask.view(np.int64)).cuda(), scale))
+    want = po.tree_attention(q, kv, P_len, parents, scale, pu.oracle_num(cfg))
+    assert np.abs(got - want).max() <= 2e-2
+    # a node's output does not change when a non-ancestor's key/value changes
+    r = rows - 1
+    other = next(j for j in range(1, rows) if not po.ancestor_matrix(parents)[r, j])
+    kv2 = kv.copy()
+    kv2[:, :, P_len + other, :] = ps.normal(9, "perturb", (2, Hkv, d), 1.0, "bf16")
+    got2 = pu.np_of(P.poss_tree_attention(_dev(q), _dev(kv2), P_len, torch.from_numpy(mask.view(np.int64)).cuda(), scale))
+    assert np.array_equal(got[r], got2[r])
+
+
+def test_full_size_verify_accept_over_the_whole_vocabulary():
+    """61 rows of bf16 logits over 128256 ids with a planted path: the accepted path is known by construction."""
+    cfg = ps.CONFIGS["t_bf16"].replace(S=1, n_target_layers=0, vocab=128256)
+    P = _poss(cfg, ps.make_weights(cfg.replace(vocab=64), 3) | {
+        "embed": np.zeros((cfg.vocab, cfg.hidden), np.uint16), "lm_head": np.zeros((cfg.vocab, cfg.hidden), np.uint16)}, 64)
+    rows = 61
+    parents = ps.random_tree_parents(18, rows, max_children=4)
+    rng = np.random.default_rng(5)
+    tokens = np.zeros(rows, dtype=np.int32)
+    for p in range(rows):
+        kids = [c for c in range(rows) if parents[c] == p]
+        tokens[kids] = rng.choice(cfg.vocab, size=len(kids), replace=False)
+    anc = po.ancestor_matrix(parents)
+    feats = ps.normal(9, "tf", (rows, cfg.hidden), 1.0, "bf16")
+    for target_node in (0, int(np.argmax(anc.sum(1)))):
+        path = [j for j in range(rows) if anc[target_node, j]]
+        lg = po.widen(ps.normal(20 + target_node, "lg", (rows, cfg.vocab), 1.0, "bf16"), np.float32).copy()
+        for a_, b_ in zip(path[:-1], path[1:]):
+            lg[a_, tokens[b_]] += 12.0
+        kids = [int(tokens[c]) for c in range(rows) if parents[c] == target_node]
+        lg[target_node, kids] -= 30.0
+        bits = ps._to_bf16_bits(lg.ravel()).reshape(rows, cfg.vocab)
+        want = po.verify_accept(po.widen(bits, np.float64), po.widen(feats, np.float64), tokens, parents)
+        out = P.poss_verify_accept(_dev(bits), None, _dev(feats), torch.from_numpy(tokens).cuda(),
+                                   torch.from_numpy(parents).cuda(), rows)
+        a = int(out["n_accepted"][0])
+        assert a == want[1] == len(path) - 1
+        assert out["path"][: a + 1].cpu().tolist() == want[0]
+        assert int(out["bonus"][0]) == want[2]
+        assert out["new_tokens"][: a + 1].cpu().tolist() == want[3].tolist()
+        assert np.array_equal(pu.np_of(out["new_features"][: a + 1]), want[4])
