@@ -49,7 +49,7 @@ namespace {
 constexpr int TILE_N = 128;          // weight rows per tile (UMMA M)
 constexpr int TILE_K = 64;           // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
-constexpr int MAX_STAGES = 10;
+constexpr int MAX_STAGES = 12;
 constexpr int N_THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr size_t SCRATCH_PARTIAL_BYTES = 96ull << 20;
@@ -59,7 +59,7 @@ constexpr int XCH_STRIDE = 17;
 struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
-  int n_tiles, kb_total, gran, l2_ahead;
+  int n_tiles, kb_total, gran, w_policy;
   const bf16* bias;
   const float* residual;
   int ldr;
@@ -115,6 +115,11 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ uint64_t policy_evict_last() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -127,10 +132,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "[%0], [%1, {%3, %4}], [%2], %5;"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
-}
-// brings a box into L2 only (no shared-memory destination, no barrier)
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c0, int c1) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -259,7 +260,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   if (warp == 0) {
     if (lane == 0 && n_kb > 0) {
       // ---------------- TMA producer
-      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      const uint64_t pol_w = a.w_policy ? policy_evict_first() : policy_evict_normal(), pol_x = policy_evict_last();
       // position of the next k-block to load, advanced without divisions
       struct Cursor { int tile, kb, seg, lt; };
       auto cursor_at = [&](long long u) {
@@ -286,33 +287,19 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
           tma_load_2d(w_tile(s), mw, full_bar(s), kcoord, c.lt * TILE_N, pol_w);
         }
       };
-      auto prefetch_w = [&](const Cursor& c) {
-        int kcoord = c.kb * TILE_K;
-        if (a.mode == 1) {
-          tma_prefetch_l2_2d(&map_w0, kcoord, c.tile * 64);
-          tma_prefetch_l2_2d(&map_w1, kcoord, c.tile * 64);
-        } else {
-          const CUtensorMap* mw = c.seg == 0 ? &map_w0 : (c.seg == 1 ? &map_w1 : &map_w2);
-          tma_prefetch_l2_2d(mw, kcoord, c.lt * TILE_N);
-        }
-      };
       auto load_x = [&](const Cursor& c, int s) {
         tma_load_2d(x_tile(s), &map_x, full_bar(s), c.kb * TILE_K, 0, pol_x);
       };
-      // Weights are never written by a kernel: before waiting for the predecessor (whose results are
-      // the activations) fill the ring with them and ask L2 for the next k-blocks behind the ring, so
-      // the memory system keeps streaming through the predecessor's tail.
+      // Weights are never written by a kernel: fill the ring with them before waiting for the
+      // predecessor, whose results are the activations.  (Asking L2 for further k-blocks at this point
+      // was measured and lost: the extra requests delay the latency-bound kernels in between.)
       const int pre = n_kb < S ? n_kb : S;
-      const int ahead = a.l2_ahead;
       Cursor cw = cursor_at(u0), cx = cw;
       for (int it = 0; it < pre; ++it) {
         mbar_expect_tx(full_bar(it), stage_bytes);
         load_w(cw, it);
         advance(cw);
       }
-      Cursor cp = cw;                          // next k-block to prefetch into L2
-      int n_pf = pre;
-      for (; n_pf < n_kb && n_pf < pre + ahead; ++n_pf) { prefetch_w(cp); advance(cp); }
       pdl_wait();
       for (int it = 0; it < pre; ++it) { load_x(cx, it); advance(cx); }
       int issued = pre, s = 0;
@@ -646,7 +633,7 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
-  int grid = 0, stages = 0, l2_ahead = 16;
+  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -663,7 +650,8 @@ TcGemmPlanCache* tc_plan_cache_create() {
   if (c->grid > TC_MAX_GRID) c->grid = TC_MAX_GRID;
   c->stages = 0;
   if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
-  if (const char* e = getenv("POSS_TC_L2_AHEAD")) { int v = atoi(e); if (v >= 0 && v <= 4096) c->l2_ahead = v; }
+  if (const char* e = getenv("POSS_TC_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 220) c->smem_kb = v; }
+  if (const char* e = getenv("POSS_TC_W_POLICY")) { int v = atoi(e); if (v >= 0 && v <= 1) c->w_policy = v; }
   return c;
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
@@ -766,11 +754,11 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   if (ep.mode == TC_EPI_TOPK) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
-  int stages = cache->stages ? cache->stages : (int)((108u * 1024u - extra) / stage_bytes);
+  int stages = cache->stages ? cache->stages : (int)(((size_t)cache->smem_kb * 1024u - extra - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
-  a.l2_ahead = cache->l2_ahead;
+  a.w_policy = cache->w_policy;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);
@@ -787,7 +775,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   }
   size_t smem = (size_t)stages * stage_bytes + extra + 1024;
   if (!cache->attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }

@@ -267,13 +267,30 @@ __global__ void k_attn_combine_bf16(int n_splits, const float* part, bf16* out) 
   int rh = blockIdx.x;       // row * Hq + head
   int e = threadIdx.x;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);
+  // split order is fixed; loads are issued eight splits at a time before they are used
   float mm = NEG_BIG;
-  for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, pp[s * (D + 2)]);
+  for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, __ldcg(pp + s * (D + 2)));
   float ll = 0.f, oo = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    float c = __expf(pp[s * (D + 2)] - mm);
-    ll += pp[s * (D + 2) + 1] * c;
-    oo += pp[s * (D + 2) + 2 + e] * c;
+  for (int base = 0; base < n_splits; base += 8) {
+    float pm[8], pl[8], po[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      int s = base + u;
+      if (s < n_splits) {
+        pm[u] = __ldcg(pp + s * (D + 2));
+        pl[u] = __ldcg(pp + s * (D + 2) + 1);
+        po[u] = __ldcg(pp + s * (D + 2) + 2 + e);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      int s = base + u;
+      if (s < n_splits) {
+        float c = __expf(pm[u] - mm);
+        ll += pl[u] * c;
+        oo += po[u] * c;
+      }
+    }
   }
   out[(size_t)rh * D + e] = __float2bfloat16_rn(oo / ll);
 }
@@ -304,13 +321,13 @@ bool tree_attention_mma_supported(const AttnArgs& a) {
 
 void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int max_splits, int* n_splits,
                                int* keys_per_split) {
-  // about one block per SM, whole 64-key chunks per split, at least two chunks per block
+  // about one block per SM, whole 64-key chunks per split
   int G = Hq / Hkv;
   int q_tiles = (rows * G + QROWS - 1) / QROWS;
   int want = (148 + Hkv * q_tiles - 1) / (Hkv * q_tiles);
   int chunks = (total_keys + CHUNK - 1) / CHUNK;
   int ns = want;
-  if (ns > (chunks + 1) / 2) ns = (chunks + 1) / 2;
+  if (ns > chunks) ns = chunks;
   if (ns > max_splits) ns = max_splits;
   if (ns < 1) ns = 1;
   int cps = (chunks + ns - 1) / ns;

@@ -286,8 +286,8 @@ __device__ __forceinline__ float4 product4(const SplitKView& v, const TileContri
 // One block per row.  The sum of squares is formed in a fixed order (per-thread partial sums over the
 // thread's column groups, a warp tree, then the warps in order), so a row's result does not depend on
 // the batch around it.
-#define NORM_THREADS 512
-#define NORM_KEEP 4
+#define NORM_THREADS 1024
+#define NORM_KEEP 2
 template <typename T>
 __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, int H, const T* bias,
                                                                const float* residual, const T* gain, float eps,
@@ -298,19 +298,28 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
   pdl_enter();
   fill_tile_table(prod, tab);
   __syncthreads();
+  POSS_TRACE_POINT(21);
   const int m = blockIdx.x;
   const int n_groups = (H + 3) / 4;
   float ss = 0.f;
   // value of one group of four columns: product + bias + residual, stored to h, squares added to ss
   auto group_value = [&](int g) {
     const int n = g * 4;
+    float add[4];                           // bias + residual, loaded before the product's partials are awaited
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      add[q] = 0.f;
+      if (n + q < H) {
+        if (residual) add[q] = residual[(size_t)m * H + n + q];
+        if (bias) add[q] += to_f(bias[n + q]);
+      }
+    }
     float4 v = product4(prod, tab, m, n, H);
     float e[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       if (n + q < H) {
-        if (bias) e[q] += to_f(bias[n + q]);
-        if (residual) e[q] += residual[(size_t)m * H + n + q];
+        e[q] += add[q];
         h[(size_t)m * H + n + q] = e[q];
         ss = fmaf(e[q], e[q], ss);
       } else {
@@ -333,6 +342,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     keep[k] = g < n_groups ? group_value(g) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) group_value(g);
+  POSS_TRACE_POINT(22);
   for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
@@ -444,6 +454,7 @@ __global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv,
     sn[threadIdx.x] = s;
   }
   __syncthreads();
+  POSS_TRACE_POINT(11);
   const int qd = a.Hq * a.d, kd = a.Hkv * a.d, N = qd + 2 * kd;
   const int q0 = a.rows - a.q_rows;
   const bool with_q = m >= q0;
@@ -451,29 +462,51 @@ __global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv,
   const int n_qitems = with_q ? a.Hq * per_head : 0;
   const int n_kitems = a.Hkv * per_head;
   const int n_vitems = kd / 4;
-#pragma unroll 2
-  for (int i = threadIdx.x; i < n_qitems + n_kitems + n_vitems; i += blockDim.x) {
-    if (i < n_qitems + n_kitems) {
-      const bool is_q = i < n_qitems;
-      const int ii = is_q ? i : i - n_qitems;
-      const int hh = ii / per_head, j = (ii % per_head) * 4;
-      const int col = (is_q ? 0 : qd) + hh * a.d + j;
-      float4 lo = product4(qkv, tab, m, col, N), hi = product4(qkv, tab, m, col + half, N);
-      float x0[4] = {lo.x, lo.y, lo.z, lo.w}, x1[4] = {hi.x, hi.y, hi.z, hi.w};
-      T* dst = is_q ? qout + (size_t)(m - q0) * qd + hh * a.d : kcache + ((size_t)hh * a.cap + slot) * a.d;
+  const int n_items = n_qitems + n_kitems + n_vitems;
+  // two items per pass: all loads of the pass are issued before the first use
+  for (int i0 = threadIdx.x; i0 < n_items; i0 += 2 * blockDim.x) {
+    float4 lo[2], hi[2];
+    int col[2];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        dst[j + e] = from_f<T>(x0[e] * cs[j + e] - x1[e] * sn[j + e]);
-        dst[j + e + half] = from_f<T>(x1[e] * cs[j + e] + x0[e] * sn[j + e]);
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * blockDim.x;
+      if (i >= n_items) continue;
+      if (i < n_qitems + n_kitems) {
+        const bool is_q = i < n_qitems;
+        const int ii = is_q ? i : i - n_qitems;
+        const int hh = ii / per_head, j = (ii % per_head) * 4;
+        col[u] = (is_q ? 0 : qd) + hh * a.d + j;
+        lo[u] = product4(qkv, tab, m, col[u], N);
+        hi[u] = product4(qkv, tab, m, col[u] + half, N);
+      } else {
+        col[u] = qd + kd + (i - n_qitems - n_kitems) * 4;
+        lo[u] = product4(qkv, tab, m, col[u], N);
       }
-    } else {
-      const int ii = (i - n_qitems - n_kitems) * 4;
-      const int hh = ii / a.d, j = ii % a.d;
-      float4 v = product4(qkv, tab, m, qd + kd + ii, N);
-      T* dst = vcache + ((size_t)hh * a.cap + slot) * a.d + j;
-      dst[0] = from_f<T>(v.x); dst[1] = from_f<T>(v.y); dst[2] = from_f<T>(v.z); dst[3] = from_f<T>(v.w);
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * blockDim.x;
+      if (i >= n_items) continue;
+      if (i < n_qitems + n_kitems) {
+        const bool is_q = i < n_qitems;
+        const int ii = is_q ? i : i - n_qitems;
+        const int hh = ii / per_head, j = (ii % per_head) * 4;
+        float x0[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w}, x1[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
+        T* dst = is_q ? qout + (size_t)(m - q0) * qd + hh * a.d : kcache + ((size_t)hh * a.cap + slot) * a.d;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          dst[j + e] = from_f<T>(x0[e] * cs[j + e] - x1[e] * sn[j + e]);
+          dst[j + e + half] = from_f<T>(x1[e] * cs[j + e] + x0[e] * sn[j + e]);
+        }
+      } else {
+        const int ii = (i - n_qitems - n_kitems) * 4;
+        const int hh = ii / a.d, j = ii % a.d;
+        T* dst = vcache + ((size_t)hh * a.cap + slot) * a.d + j;
+        dst[0] = from_f<T>(lo[u].x); dst[1] = from_f<T>(lo[u].y); dst[2] = from_f<T>(lo[u].z); dst[3] = from_f<T>(lo[u].w);
+      }
     }
   }
+  POSS_TRACE_POINT(12);
 }
 template <typename T>
 void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {

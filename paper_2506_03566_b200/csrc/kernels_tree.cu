@@ -323,6 +323,147 @@ __global__ void __launch_bounds__(128) k_topk_merge(int K, int n_lists, const fl
   if (threadIdx.x == 0) *done = 0;
 }
 
+// ------------------------------------------------------------------ the same for a draft step, in one block
+// A draft step has at most POSS_MAX_TOPK rows and is followed by the tree expansion, which needs every
+// row's result: one block of 1024 threads stages all partial lists in shared memory with 16-byte loads
+// (one round trip), warp r merges row r, and after one barrier the block expands the tree.  No second
+// kernel, no counter.
+__global__ void __launch_bounds__(1024) k_topk_merge_expand(int rows, int K, int n_lists, const float* pmax,
+                                                            const float* psum, const float* pval,
+                                                            const int32_t* pidx, int32_t* out_ids, float* out_logp,
+                                                            TreeState ts, ExpandArgs x) {
+  extern __shared__ __align__(16) unsigned char me_smem[];
+  const int per_row = n_lists * K;
+  const int total = rows * per_row;
+  const int total4 = (total + 3) & ~3;
+  float* vals = reinterpret_cast<float*>(me_smem);               // [rows][n_lists][K]
+  int* idxs = reinterpret_cast<int*>(vals + total4);             // [rows][n_lists][K]
+  float* smax = reinterpret_cast<float*>(idxs + total4);         // [rows][n_lists]
+  float* ssum = smax + rows * n_lists;                           // [rows][n_lists]
+  int* heads = reinterpret_cast<int*>(ssum + rows * n_lists);    // [rows][n_lists]
+  pdl_enter();
+  {
+    const int n4 = total / 4;
+    const float4* pv4 = reinterpret_cast<const float4*>(pval);
+    const int4* pi4 = reinterpret_cast<const int4*>(pidx);
+    for (int base = 0; base < n4; base += 1024 * 4) {
+      float4 v[4];
+      int4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int i = base + u * 1024 + threadIdx.x;
+        if (i < n4) { v[u] = __ldcg(pv4 + i); q[u] = __ldcg(pi4 + i); }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int i = base + u * 1024 + threadIdx.x;
+        if (i < n4) { reinterpret_cast<float4*>(vals)[i] = v[u]; reinterpret_cast<int4*>(idxs)[i] = q[u]; }
+      }
+    }
+    for (int i = n4 * 4 + threadIdx.x; i < total; i += 1024) { vals[i] = __ldcg(pval + i); idxs[i] = __ldcg(pidx + i); }
+    for (int i = threadIdx.x; i < rows * n_lists; i += 1024) {
+      smax[i] = __ldcg(pmax + i);
+      ssum[i] = __ldcg(psum + i);
+      heads[i] = 0;
+    }
+  }
+  __syncthreads();
+  POSS_TRACE_POINT(1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < rows) {
+    const int row = warp;
+    const float* rmax = smax + row * n_lists;
+    const float* rsum = ssum + row * n_lists;
+    const float* rv = vals + (size_t)row * per_row;
+    const int* ri = idxs + (size_t)row * per_row;
+    int* rh = heads + row * n_lists;
+    float gm = NEG_INF;
+    for (int c = lane; c < n_lists; c += 32) gm = fmaxf(gm, rmax[c]);
+    for (int off = 16; off > 0; off >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, off));
+    float se = 0.f;
+    for (int c = lane; c < n_lists; c += 32) {
+      float m = rmax[c];
+      if (m > NEG_INF) se += rsum[c] * expf(m - gm);
+    }
+    for (int off = 16; off > 0; off >>= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
+    const float lse = gm + logf(se);
+    POSS_TRACE_POINT(2);
+    if (n_lists <= 32 * 6) {
+      // each lane keeps the heads of its (at most six) lists in registers: a round is a register scan,
+      // one warp reduction and one shared-memory load by the winning lane
+      float hv[6];
+      int hi[6], hp[6];
+#pragma unroll
+      for (int j = 0; j < 6; ++j) {
+        int c = lane + 32 * j;
+        hp[j] = 0;
+        hv[j] = c < n_lists ? rv[c * K] : NEG_INF;
+        hi[j] = c < n_lists ? ri[c * K] : 0x7fffffff;
+      }
+      for (int k = 0; k < K; ++k) {
+        float bv = hv[0];
+        int bi = hi[0], bj = 0;
+#pragma unroll
+        for (int j = 1; j < 6; ++j) if (better(hv[j], hi[j], bv, bi)) { bv = hv[j]; bi = hi[j]; bj = j; }
+        float wv = bv;
+        int wi = bi, wl = lane;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          float ov = __shfl_xor_sync(0xffffffffu, wv, off);
+          int oi = __shfl_xor_sync(0xffffffffu, wi, off);
+          int ol = __shfl_xor_sync(0xffffffffu, wl, off);
+          if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
+        }
+        if (lane == 0) {
+          out_ids[(size_t)row * K + k] = wi;
+          out_logp[(size_t)row * K + k] = wv - lse;
+        }
+        if (lane == wl && wi != 0x7fffffff) {
+          // advance the winning list
+#pragma unroll
+          for (int j = 0; j < 6; ++j) {
+            if (j == bj) {
+              int c = lane + 32 * j, h = ++hp[j];
+              hv[j] = h < K ? rv[c * K + h] : NEG_INF;
+              hi[j] = h < K ? ri[c * K + h] : 0x7fffffff;
+            }
+          }
+        }
+      }
+    } else {
+      for (int k = 0; k < K; ++k) {
+        float bv = NEG_INF;
+        int bi = 0x7fffffff, bc = -1;
+        for (int c = lane; c < n_lists; c += 32) {
+          int h = rh[c];
+          if (h < K) {
+            float v = rv[c * K + h];
+            int i = ri[c * K + h];
+            if (better(v, i, bv, bi)) { bv = v; bi = i; bc = c; }
+          }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+          int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+          int oc = __shfl_xor_sync(0xffffffffu, bc, off);
+          if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bc = oc; }
+        }
+        if (lane == 0) {
+          out_ids[(size_t)row * K + k] = bi;
+          out_logp[(size_t)row * K + k] = bv - lse;
+          if (bc >= 0) rh[bc] += 1;
+        }
+        __syncwarp();
+      }
+    }
+  }
+  POSS_TRACE_POINT(3);
+  __syncthreads();                       // every row's ids / log-probs are written (this block's own stores)
+  if (x.enabled) expand_block(ts, x, out_ids, out_logp, vals);
+  POSS_TRACE_POINT(4);
+}
+
 void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* pmax, const float* psum,
                        const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp,
                        const TreeState* ts, const ExpandArgs* x, int* done) {
@@ -332,6 +473,25 @@ void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* p
   TreeState t;
   memset(&t, 0, sizeof(t));
   if (x && ts && x->enabled) { xa = *x; t = *ts; }
+  if (xa.enabled && rows <= POSS_MAX_TOPK) {
+    size_t total4 = ((size_t)rows * n_lists * K + 3) & ~(size_t)3;
+    size_t smem1 = total4 * 8 + (size_t)rows * n_lists * 12;
+    if (smem1 < (size_t)xa.Mc * K * 4) smem1 = (size_t)xa.Mc * K * 4;
+    if (smem1 <= 200 * 1024) {
+      static bool attr1_done = false;
+      if (!attr1_done) {
+        if (cudaFuncSetAttribute(k_topk_merge_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) !=
+            cudaSuccess) {
+          L.err = POSS_E_CUDA;
+          return;
+        }
+        attr1_done = true;
+      }
+      launch_pdl(L, k_topk_merge_expand, dim3(1), dim3(1024), smem1, rows, K, n_lists, pmax, psum, pval, pidx, out_ids,
+                 out_logp, t, xa);
+      return;
+    }
+  }
   size_t elems = (size_t)n_lists * K;
   if (xa.enabled && elems < (size_t)xa.Mc * K) elems = (size_t)xa.Mc * K;      // room for the expansion's scores
   size_t smem = elems * 8 + (size_t)n_lists * 4;

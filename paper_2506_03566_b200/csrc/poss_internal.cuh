@@ -85,6 +85,11 @@ __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// hook for a timeline-recording build; empty in the library
+#ifndef POSS_TRACE_POINT
+#define POSS_TRACE_POINT(id)
+#endif
+
 template <typename... KArgs, typename... Args>
 inline void launch_pdl(Launcher& L, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
   cudaLaunchAttribute at[1];
@@ -138,8 +143,20 @@ __host__ __device__ __forceinline__ int splitk_cta_of_unit(long long u, long lon
 struct TileContrib { int c_first, count, slot_first; };
 __device__ __forceinline__ TileContrib splitk_tile_contrib(const SplitKView& v, int tile) {
   long long groups = (long long)v.n_tiles * v.kb_total;
-  long long tile_u0 = (long long)tile * v.kb_total;
   TileContrib t;
+  if (groups * v.G < (1ll << 31)) {
+    // same arithmetic in 32 bits (the usual case): far cheaper divisions
+    unsigned gr = (unsigned)groups, G = (unsigned)v.G, u0 = (unsigned)tile * (unsigned)v.kb_total;
+    unsigned cf = ((u0 + 1u) * G + gr - 1u) / gr - 1u;
+    unsigned cl = ((u0 + (unsigned)v.kb_total) * G + gr - 1u) / gr - 1u;
+    if (cf > G - 1u) cf = G - 1u;
+    if (cl > G - 1u) cl = G - 1u;
+    t.c_first = (int)cf;
+    t.count = (int)(cl - cf) + 1;
+    t.slot_first = (cf * gr / G) >= u0 ? 0 : 1;
+    return t;
+  }
+  long long tile_u0 = (long long)tile * v.kb_total;
   t.c_first = splitk_cta_of_unit(tile_u0, groups, v.G, 1);
   int c_last = splitk_cta_of_unit(tile_u0 + v.kb_total - 1, groups, v.G, 1);
   t.count = c_last - t.c_first + 1;
