@@ -1,9 +1,12 @@
 """Benchmark of one PosS speculative round on the Llama-3-8B-shaped drafter workload (config c2).
 
 A step = the whole hot path once: poss_draft_round (6 specialist steps, width 10, 60 kept tokens,
-prefix 1024) + tree-masked verification attention over the 61 tree rows at the target's geometry
-+ argmax over target logits and the greedy accept walk.  Weights are random-init, inputs seeded
-and synthetic (poss_synth).  One JSON line on stdout.
+prefix 1024) + the tree-masked target pass over the 61 tree rows (32 Llama-3-8B-shaped layers, final
+norm, LM-head argmax) + the greedy accept walk + KV compaction.  Drafter weights and inputs come from
+the seeded host generator (poss_synth); the 14 GB of target layers are drawn on the device from a
+seeded generator (same recipe, N(0, 0.02) bf16) so that the default run stays within minutes.
+With --no-target the step's verification side is the stand-alone stages instead (61-row attention at
+target geometry, argmax over given logits, accept walk).  One JSON line on stdout.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c2]
 """
@@ -110,6 +113,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--config", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-target", action="store_true", help="verification side = stand-alone stages, no target layers")
     ap.add_argument("--alias-specialists", action="store_true",
                     help="profiler captures only: all specialists share one weight set, so the process holds "
                          "about 3 GB instead of 10 GB; the launch chain and every launch's traffic are unchanged "
@@ -139,33 +143,61 @@ def main():
         dist.barrier()
     warmup = max(args.warmup, 3)
 
-    # ---------------- inputs: seeded, host-generated, resident in HBM before timing
+    # ---------------- inputs: seeded, resident in HBM before timing
     seed = 1 + rank          # replicas only: every rank runs an independent request
+    with_target = not (args.no_target or args.alias_specialists)
+    n_layers = 32 if with_target else 0
     w = ps.make_weights(cfg, seed, alias_specialists=args.alias_specialists)
     rows = cfg.total + 1
     cap = cfg.prefix + 8 + cfg.tree_slots
-    P = Poss(make_config(cfg, cap), w)
+    tcap = cfg.prefix + rows
+    if with_target:
+        gen = torch.Generator(device="cuda").manual_seed(1000 + seed)
+        H, F = cfg.hidden, cfg.ffn
+        qd, kd = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+
+        def dev_normal(*shape, std=0.02):
+            return (torch.randn(*shape, device="cuda", generator=gen) * std).to(torch.bfloat16)
+
+        ones = torch.ones(H, device="cuda", dtype=torch.bfloat16)
+        w["target"] = [{"norm_in": ones, "wq": dev_normal(qd, H), "wk": dev_normal(kd, H), "wv": dev_normal(kd, H),
+                        "wo": dev_normal(H, qd), "norm_post": ones, "w_gate": dev_normal(F, H),
+                        "w_up": dev_normal(F, H), "w_down": dev_normal(H, F)} for _ in range(n_layers)]
+        w["final_norm"] = ones
+    P = Poss(make_config(cfg.replace(n_target_layers=n_layers), cap, tcap), w)
     dkv = to_device(ps.make_draft_kv(cfg, seed, cap))
     tok_h, feat_h = ps.make_round_inputs(cfg, seed, 1)
     tok_pin = torch.from_numpy(tok_h).pin_memory()
     feat_pin = torch.from_numpy(feat_h.view(np.int16)).pin_memory()
     tok_d = tok_pin.cuda()
     feat_d = feat_pin.cuda().view(torch.bfloat16)
-    # verification side: target-geometry KV with the tree rows' keys behind the prefix, queries, logits
-    tcap = cfg.prefix + rows
-    q_h, tkv_h = ps.make_attention_case(seed, rows, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.prefix, tcap, "bf16")
-    q_d, tkv_d = to_device(q_h), to_device(tkv_h)
-    logits_d = to_device(ps.normal(seed, "target_logits", (rows, cfg.vocab), 1.0, "bf16"))
-    tfeat_d = to_device(ps.normal(seed, "target_features", (rows, cfg.hidden), 1.0, "bf16"))
     scale = 1.0 / float(np.sqrt(cfg.head_dim))
     out = P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total)
-    attn_out = torch.empty_like(q_d)
-    del w
+    if with_target:
+        # target cache: prefix keys / values N(0, 1), tree rows appended by the pass itself
+        tkv_t = P.new_target_kv()
+        tkv_t[:, :, :, :cfg.prefix, :] = torch.randn(n_layers, 2, cfg.n_kv_heads, cfg.prefix, cfg.head_dim, device="cuda",
+                                                     generator=gen).to(torch.bfloat16)
 
-    def step(tok, feat):
-        tree = P.poss_draft_round(dkv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, out=out)
-        P.poss_tree_attention(q_d, tkv_d, cfg.prefix, tree["anc_mask"], scale, out=attn_out)
-        return P.poss_verify_accept(logits_d, None, tfeat_d, tree["tokens"], tree["parents"], rows)
+        def step(tok, feat):
+            tree = P.poss_draft_round(dkv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, out=out)
+            tf, targ, _ = P.poss_target_forward(tkv_t, cfg.prefix, tree["tokens"], tree["depth"], tree["anc_mask"], rows)
+            va = P.poss_verify_accept(None, targ, tf, tree["tokens"], tree["parents"], rows)
+            P.poss_kv_compact(tkv_t, cfg.prefix, va["path"], va["n_accepted"])
+            return va
+    else:
+        # stand-alone verification stages: target-geometry KV with the tree rows' keys behind the prefix
+        q_h, tkv_h = ps.make_attention_case(seed, rows, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.prefix, tcap, "bf16")
+        q_d, tkv_d = to_device(q_h), to_device(tkv_h)
+        logits_d = to_device(ps.normal(seed, "target_logits", (rows, cfg.vocab), 1.0, "bf16"))
+        tfeat_d = to_device(ps.normal(seed, "target_features", (rows, cfg.hidden), 1.0, "bf16"))
+        attn_out = torch.empty_like(q_d)
+
+        def step(tok, feat):
+            tree = P.poss_draft_round(dkv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, out=out)
+            P.poss_tree_attention(q_d, tkv_d, cfg.prefix, tree["anc_mask"], scale, out=attn_out)
+            return P.poss_verify_accept(logits_d, None, tfeat_d, tree["tokens"], tree["parents"], rows)
+    del w
 
     def sync_all():
         torch.cuda.synchronize()
@@ -243,11 +275,13 @@ def main():
             "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: Llama-3-8B-shaped drafter, 6 specialists, depth 6, top-k 10, "
-                                   "60 tokens, prefix 1024; step = draft round + 61-row verification attention + accept walk",
+                                   "60 tokens, prefix 1024; step = draft round + " +
+                                   ("61-row tree-masked pass of a 32-layer Llama-3-8B-shaped target + accept walk + KV compaction"
+                                    if with_target else "61-row verification attention + logits argmax + accept walk"),
                        "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "stages_us": {"draft_round": draft_ms * 1e3, "whole_step": ms * 1e3,
-                          "verify_attention_plus_accept": max(ms - draft_ms, 0.0) * 1e3},
+                          "verify_round": max(ms - draft_ms, 0.0) * 1e3},
             "rounds_per_s": world * 1e3 / ms,
             "draft_round_gbs": round_bytes / (draft_ms * 1e-3) / 1e9,
             "draft_round_frac_of_hbm_peak": round_bytes / (draft_ms * 1e-3) / 1e9 / hbm_peak,

@@ -198,8 +198,8 @@ POSS_API int poss_linear(poss_ctx* ctx, const void* x, int M, const void* w, int
 POSS_API int poss_lm_head_topk(poss_ctx* ctx, const void* features, int rows, int topk,
                       int32_t* out_ids, float* out_logp, float* out_logits, poss_stream stream);
 
-/* Device-time bracketing of the dominant kernel, the LM-head matrix product: while enabled, each of
- * its launches sits between two CUDA events on the launching stream (at most 1024 launches between
+/* Device-time bracketing of the dominant kernel, the LM-head matrix product of a draft step: while enabled,
+ * each of those launches (not the target pass's argmax launch) sits between two CUDA events on the launching stream (at most 1024 launches between
  * reads).  poss_profile_read SYNCHRONISES on the last event, returns how many launches were
  * bracketed since the previous read and their summed device time in ms, and starts over. */
 POSS_API int poss_profile(poss_ctx* ctx, int enable);

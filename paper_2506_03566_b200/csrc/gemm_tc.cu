@@ -197,6 +197,7 @@ struct Segment {
 };
 
 // ------------------------------------------------------------------ the kernel
+template <bool ARGMAX>
 __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
                                                        const __grid_constant__ CUtensorMap map_w0,
                                                        const __grid_constant__ CUtensorMap map_w1,
@@ -362,10 +363,20 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     float* st_sum = extra + (size_t)(4 + q) * a.M;
     float* lst_val = extra + (size_t)8 * a.M + (size_t)q * a.M * K;
     int* lst_idx = reinterpret_cast<int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K) + (size_t)q * a.M * K;
-    if (a.mode == 2) {
+    if (!ARGMAX && a.mode == 2) {
       for (int m = lane; m < a.M; m += 32) { st_max[m] = -INFINITY; st_sum[m] = 0.f; }
       for (int i = lane; i < a.M * K; i += 32) { lst_val[i] = -INFINITY; lst_idx[i] = 0x7fffffff; }
       __syncwarp();
+    }
+    // argmax mode: every lane keeps, in registers, the best (value, id) of its own rows for each of up to
+    // 64 activation rows; the lanes are merged once, after the CTA's last tile
+    float abv[ARGMAX ? 4 : 1][16];
+    int abi[ARGMAX ? 4 : 1][16];
+    if (ARGMAX) {
+#pragma unroll
+      for (int cc = 0; cc < (ARGMAX ? 4 : 1); ++cc)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { abv[cc][j] = -INFINITY; abi[cc][j] = 0x7fffffff; }
     }
     bool ok = true;
     int it = 0, seg_i = 0;
@@ -481,7 +492,27 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         }
       };
 
-      if (whole && a.mode != 3) {
+      if (ARGMAX) {
+        // (argmax launches always hand out whole tiles)
+#pragma unroll
+        for (int cc = 0; cc < (ARGMAX ? 4 : 1); ++cc) {
+          const int c0 = cc * 16;
+          if (c0 < a.Npad && c0 < a.M) {
+            float v[16];
+            tmem_ld16(taddr + (uint32_t)c0, v);
+            if (c0 + 16 >= a.Npad || c0 + 16 >= a.M) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(acc_empty(buf));
+            }
+            if (n_ok) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (v[j] > abv[cc][j]) { abv[cc][j] = v[j]; abi[cc][j] = n_local; }   // rows only grow: ties keep the lower id
+            }
+          }
+        }
+      } else if (whole && a.mode != 3) {
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
           float v[16];
           tmem_ld16(taddr + (uint32_t)c0, v);
@@ -557,7 +588,37 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
       ++seg_i;
     }
 
-    if (a.mode == 2) {
+    if (ARGMAX) {
+      // ---- merge the 128 lanes' bests per activation row.  The ring is idle now (every stage was consumed
+      // before the last accumulator was handed to the epilogue), so it serves as the exchange buffer.
+      float* xv = reinterpret_cast<float*>(tiles_ptr);                  // [128][65]
+      int* xi = reinterpret_cast<int*>(tiles_ptr) + 128 * 65;           // [128][65]
+      epi_sync();
+#pragma unroll
+      for (int cc = 0; cc < (ARGMAX ? 4 : 1); ++cc)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { xv[t * 65 + cc * 16 + j] = abv[cc][j]; xi[t * 65 + cc * 16 + j] = abi[cc][j]; }
+      epi_sync();
+      // two threads per row, each scans 64 lanes' entries, then the pair is merged with a shuffle
+      const int m = t >> 1, half_sel = t & 1;
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+      if (m < a.M) {
+        for (int l = half_sel * 64; l < half_sel * 64 + 64; ++l) {
+          float v = xv[l * 65 + m];
+          int i = xi[l * 65 + m];
+          if (better(v, i, bv, bi)) { bv = v; bi = i; }
+        }
+      }
+      float ov = __shfl_xor_sync(0xffffffffu, bv, 1);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, 1);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      if (m < a.M && half_sel == 0) {
+        size_t o = (size_t)m * gridDim.x + blockIdx.x;
+        a.pmax[o] = bv; a.psum[o] = 1.f; a.pval[o] = bv; a.pidx[o] = bi;
+      }
+    }
+    if (!ARGMAX && a.mode == 2) {
       // ---- merge the four warps' running states into this CTA's list (columns dealt round-robin)
       epi_sync();
       const float* all_max = extra;
@@ -633,7 +694,7 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
-  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150;
+  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150, align_ranges = 1;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -651,6 +712,7 @@ TcGemmPlanCache* tc_plan_cache_create() {
   c->stages = 0;
   if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
   if (const char* e = getenv("POSS_TC_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 220) c->smem_kb = v; }
+  if (const char* e = getenv("POSS_TC_ALIGN")) { int v = atoi(e); if (v >= 0 && v <= 1) c->align_ranges = v; }
   if (const char* e = getenv("POSS_TC_W_POLICY")) { int v = atoi(e); if (v >= 0 && v <= 1) c->w_policy = v; }
   return c;
 }
@@ -741,7 +803,15 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   a.gran = no_split ? a.kb_total : 1;
   // never more CTAs than ranges to hand out: every CTA of the grid owns at least one k-block
   long long groups = (long long)n_tiles * a.kb_total / a.gran;
-  const int G = (long long)cache->grid < groups ? cache->grid : (int)groups;
+  int G = (long long)cache->grid < groups ? cache->grid : (int)groups;
+  // Partials left to the consumer: a grid that is a whole multiple of the tile count gives every tile the
+  // same number of equal ranges, none straddling two tiles, so each CTA parks one segment and the
+  // consumer adds grid/tiles partials instead of one or two more.
+  if (a.mode == TC_EPI_PARTIAL && cache->align_ranges && n_tiles * 2 <= G) {
+    int per_tile = G / n_tiles;
+    if (per_tile > a.kb_total) per_tile = a.kb_total;
+    G = per_tile * n_tiles;
+  }
   if (ep.n_lists) *ep.n_lists = G;
   if (a.mode == TC_EPI_PARTIAL) {
     SplitKView* v = ep.view;
@@ -753,7 +823,9 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
-  if (ep.mode == TC_EPI_TOPK) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
+  // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
+  const bool argmax = ep.mode == TC_EPI_TOPK && ep.argmax_only && ep.topk == 1 && a.Npad <= 64;
+  if (ep.mode == TC_EPI_TOPK && !argmax) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
   int stages = cache->stages ? cache->stages : (int)(((size_t)cache->smem_kb * 1024u - extra - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
@@ -775,12 +847,14 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   }
   size_t smem = (size_t)stages * stage_bytes + extra + 1024;
   if (!cache->attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
     cache->attr_set = true;
   }
+  if (argmax && (size_t)stages * stage_bytes < (size_t)128 * 65 * 8) { L.err = POSS_E_SHAPE; return; }   // exchange buffer
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(G);
@@ -792,6 +866,8 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, mx, mw[0], mw[1], mw[2], a) != cudaSuccess) L.err = POSS_E_CUDA;
+  cudaError_t le = argmax ? cudaLaunchKernelEx(&cfg, k_gemm_tc<true>, mx, mw[0], mw[1], mw[2], a)
+                          : cudaLaunchKernelEx(&cfg, k_gemm_tc<false>, mx, mw[0], mw[1], mw[2], a);
+  if (le != cudaSuccess) L.err = POSS_E_CUDA;
   LAUNCH_CHECK(L);
 }

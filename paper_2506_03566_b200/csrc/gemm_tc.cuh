@@ -33,6 +33,7 @@ struct TcEpilogue {
   bf16* out_bf = nullptr;
   int ldo_bf = 0;
   int topk = 0;
+  bool argmax_only = false;   // TC_EPI_TOPK with topk == 1 and no use for max / sum-exp: cheaper epilogue, psum = 1
   float* pmax = nullptr;
   float* psum = nullptr;
   float* pval = nullptr;

@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
   if (v0) { mk0a = a.mask[(size_t)r0 * a.mask_words]; if (a.mask_words > 1) mk0b = a.mask[(size_t)r0 * a.mask_words + 1]; }
   if (v1) { mk1a = a.mask[(size_t)r1 * a.mask_words]; if (a.mask_words > 1) mk1b = a.mask[(size_t)r1 * a.mask_words + 1]; }
 
+  POSS_TRACE_POINT(1);
   float m0 = NEG_BIG, m1 = NEG_BIG, l0 = 0.f, l1 = 0.f;
   float o[NT_D][4];
 #pragma unroll
@@ -230,6 +231,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
     __syncthreads();          // the stage is overwritten by the load issued in the next iteration
   }
 
+  POSS_TRACE_POINT(2);
   if (!warp_active) return;
   if (a.n_splits == 1) {
     const float inv0 = 1.f / l0, inv1 = 1.f / l1;
@@ -321,10 +323,11 @@ bool tree_attention_mma_supported(const AttnArgs& a) {
 
 void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int max_splits, int* n_splits,
                                int* keys_per_split) {
-  // about one block per SM, whole 64-key chunks per split
+  // a few blocks per SM (a block's work is a chain of dependent MMAs: more, shorter blocks finish sooner),
+  // whole 64-key chunks per split
   int G = Hq / Hkv;
   int q_tiles = (rows * G + QROWS - 1) / QROWS;
-  int want = (148 + Hkv * q_tiles - 1) / (Hkv * q_tiles);
+  int want = (3 * 148 + Hkv * q_tiles - 1) / (Hkv * q_tiles);      // up to three blocks per SM fit
   int chunks = (total_keys + CHUNK - 1) / CHUNK;
   int ns = want;
   if (ns > chunks) ns = chunks;

@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
   pdl_enter();
   fill_tile_table(prod, tab);
   __syncthreads();
-  POSS_TRACE_POINT(21);
+  POSS_TRACE_POINT(1);
   const int m = blockIdx.x;
   const int n_groups = (H + 3) / 4;
   float ss = 0.f;
@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     keep[k] = g < n_groups ? group_value(g) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) group_value(g);
-  POSS_TRACE_POINT(22);
+  POSS_TRACE_POINT(2);
   for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
@@ -454,7 +454,7 @@ __global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv,
     sn[threadIdx.x] = s;
   }
   __syncthreads();
-  POSS_TRACE_POINT(11);
+  POSS_TRACE_POINT(1);
   const int qd = a.Hq * a.d, kd = a.Hkv * a.d, N = qd + 2 * kd;
   const int q0 = a.rows - a.q_rows;
   const bool with_q = m >= q0;
@@ -506,7 +506,7 @@ __global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv,
       }
     }
   }
-  POSS_TRACE_POINT(12);
+  POSS_TRACE_POINT(2);
 }
 template <typename T>
 void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {

@@ -178,17 +178,18 @@ struct Impl {
   // act[M][F] = T(silu(x . gate^T) * (x . up^T))
   void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
-  bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists);
+  bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists, bool argmax_only = false);
 
+  // need_logp = false (with K = 1): the caller wants the argmax only; logp is then meaningless
   void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out,
-                    const ExpandArgs* expand = nullptr) {
+                    const ExpandArgs* expand = nullptr, bool need_logp = true) {
     const poss_config& g = c->cfg;
     GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = g.vocab;
     float* lg = logits_out ? logits_out : c->b.logits;
-    bool prof = c->prof_on && c->prof_n < PROF_MAX;
+    bool prof = c->prof_on && c->prof_n < PROF_MAX && expand != nullptr;   // the draft steps' launches only
     if (prof) cudaEventRecord(c->prof_ev[2 * c->prof_n], L.stream);
     int n_lists = 0;
-    bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists);
+    bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists, !need_logp && K == 1);
     if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
     if (prof) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], L.stream); ++c->prof_n; }
     if (!fused) {
@@ -354,7 +355,8 @@ struct Impl {
       layer_tail(lw, b.hx, rows, b.hx, last ? A(out_features) : A(b.xn), next_gain);
     }
     if (out_argmax || out_logits)
-      lm_head_topk(A(out_features), rows, 1, out_argmax ? out_argmax : b.argmax_tmp, b.top_logp, out_logits);
+      lm_head_topk(A(out_features), rows, 1, out_argmax ? out_argmax : b.argmax_tmp, b.top_logp, out_logits, nullptr,
+                   false);
     return L.err;
   }
 };
@@ -424,13 +426,13 @@ void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const voi
 }
 
 template <typename T>
-bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*) { return false; }
+bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*, bool) { return false; }
 template <>
-bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists) {
+bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists, bool argmax_only) {
   GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = c->cfg.vocab;
   if (!tc_gemm_supported(sg, K, K, M)) return false;
   TcEpilogue ep;
-  ep.mode = TC_EPI_TOPK; ep.topk = topk;
+  ep.mode = TC_EPI_TOPK; ep.topk = topk; ep.argmax_only = argmax_only;
   ep.pmax = c->b.pmax; ep.psum = c->b.psum; ep.pval = c->b.pval; ep.pidx = c->b.pidx; ep.n_lists = n_lists;
   launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
   return true;

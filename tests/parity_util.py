@@ -3,7 +3,9 @@ the same seeded inputs, and compare under the stated rules.
 
 Rules (written here, used by every parity test):
   * check mode (fp32): structure, tokens and paths bit-exact; features/logits within 1e-4.
-  * bf16: features/logits/log-probs within 2e-2; structure bit-exact unless the oracle's margin at the
+  * bf16: features/logits/log-probs within 2e-2 (features: 2e-2 x max(1, RMS of the step's features), because
+    bf16 spacing is relative and the random-init residual stream of the full-size shapes has RMS 3..15);
+    structure bit-exact unless the oracle's margin at the
     deciding comparison is below 1e-2.  bf16 results of two correct implementations agree only to
     about one bf16 unit per rounding boundary, and that noise grows with the draft depth, so the
     numeric comparison is PER STEP WITH TEACHER FORCING: the oracle is re-run following the GPU's
@@ -131,7 +133,10 @@ def compare_round(cfg, w, kv_np, prefix_len, new_tok, new_feat, depth, K, T, g, 
         for i, st in enumerate(fol.steps):
             mc = st.fout.shape[0]
             err = np.abs(st.fout - trace["step_features"][i, :mc]).max()
-            assert err <= tol, f"step {i} feature error {err} (following)"
+            # bf16 rounding is relative (spacing 2^-8 of the magnitude): the absolute bound is for activations
+            # of order one and scales with the feature's RMS where the synthetic residual stream is larger
+            ftol = tol * max(1.0, float(np.sqrt(np.mean(np.square(st.fout)))))
+            assert err <= ftol, f"step {i} feature error {err} > {ftol} (following)"
             for r in range(mc):
                 z = st.logits[r]
                 kth = np.sort(z)[-K]
