@@ -225,14 +225,17 @@ template void launch_tree_attention<bf16>(Launcher&, const AttnArgs&, const bf16
 template <>
 void run_tree_attention<float>(Launcher& L, AttnArgs a, int max_splits, const float* q, const float* kc,
                                const float* vc, float* part, float* out) {
+  a.splits_per_block = 1;
   plan_attention_splits(a.rows, a.Hkv, a.n_all + a.n_tree, max_splits, &a.n_splits, &a.keys_per_split);
   launch_tree_attention<float>(L, a, q, kc, vc, part, out);
 }
 template <>
 void run_tree_attention<bf16>(Launcher& L, AttnArgs a, int max_splits, const bf16* q, const bf16* kc, const bf16* vc,
                               float* part, bf16* out) {
+  a.splits_per_block = 1;
   if (tree_attention_mma_supported(a)) {
-    plan_attention_splits_mma(a.rows, a.Hq, a.Hkv, a.n_all + a.n_tree, max_splits, &a.n_splits, &a.keys_per_split);
+    plan_attention_splits_mma(a.rows, a.Hq, a.Hkv, a.n_all + a.n_tree, max_splits, &a.n_splits, &a.keys_per_split,
+                              &a.splits_per_block);
     launch_tree_attention_mma(L, a, q, kc, vc, part, out);
     return;
   }

@@ -86,10 +86,14 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
   const int r0 = v0 ? qi0 / G : 0, r1 = v1 ? qi1 / G : 0;
   const bool warp_active = qtile * QROWS + warp * 16 < n_q;
 
+  // the block walks splits_per_block consecutive splits as one chunk sequence and emits one partial per
+  // split: how many splits a block takes is a scheduling choice, the grouping of the sums is not
   const int total = a.n_all + a.n_tree;
-  const int k_begin = split * a.keys_per_split;
-  const int k_end = min(total, k_begin + a.keys_per_split);
+  const int split0 = split * a.splits_per_block;
+  const int k_begin = split0 * a.keys_per_split;
+  const int k_end = min(total, k_begin + a.splits_per_block * a.keys_per_split);
   const int n_chunks = (k_end - k_begin + CHUNK - 1) / CHUNK;
+  const int chunks_per_split = a.keys_per_split / CHUNK;
   const bf16* kb = kcache + (size_t)kvh * a.cap * D;
   const bf16* vb = vcache + (size_t)kvh * a.cap * D;
 
@@ -135,6 +139,22 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
   float o[NT_D][4];
 #pragma unroll
   for (int j = 0; j < NT_D; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+
+  // online-softmax partial (m, l, o[d]) of one split for this thread's two query rows
+  auto write_partial = [&](int sp) {
+    if (v0) {
+      float* pp = part + (((size_t)r0 * a.Hq + kvh * G + qi0 % G) * a.n_splits + sp) * (D + 2);
+      if (tq == 0) { pp[0] = m0; pp[1] = l0; }
+#pragma unroll
+      for (int j = 0; j < NT_D; ++j) *reinterpret_cast<float2*>(pp + 2 + j * 8 + tq * 2) = make_float2(o[j][0], o[j][1]);
+    }
+    if (v1) {
+      float* pp = part + (((size_t)r1 * a.Hq + kvh * G + qi1 % G) * a.n_splits + sp) * (D + 2);
+      if (tq == 0) { pp[0] = m1; pp[1] = l1; }
+#pragma unroll
+      for (int j = 0; j < NT_D; ++j) *reinterpret_cast<float2*>(pp + 2 + j * 8 + tq * 2) = make_float2(o[j][2], o[j][3]);
+    }
+  };
 
   for (int c = 0; c < n_chunks; ++c) {
     const int stage = c & 1;
@@ -227,6 +247,14 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
           mma_bf16(o[jd + 1], pl, b2, b3);
         }
       }
+      // last chunk of a split (but not of the block): hand the split's partial over and start afresh
+      if (a.n_splits > 1 && (c + 1) % chunks_per_split == 0 && c + 1 < n_chunks) {
+        write_partial(split0 + c / chunks_per_split);
+        m0 = m1 = NEG_BIG;
+        l0 = l1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < NT_D; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+      }
     }
     __syncthreads();          // the stage is overwritten by the load issued in the next iteration
   }
@@ -249,18 +277,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
     }
     return;
   }
-  if (v0) {
-    float* pp = part + (((size_t)r0 * a.Hq + kvh * G + qi0 % G) * a.n_splits + split) * (D + 2);
-    if (tq == 0) { pp[0] = m0; pp[1] = l0; }
-#pragma unroll
-    for (int j = 0; j < NT_D; ++j) *reinterpret_cast<float2*>(pp + 2 + j * 8 + tq * 2) = make_float2(o[j][0], o[j][1]);
-  }
-  if (v1) {
-    float* pp = part + (((size_t)r1 * a.Hq + kvh * G + qi1 % G) * a.n_splits + split) * (D + 2);
-    if (tq == 0) { pp[0] = m1; pp[1] = l1; }
-#pragma unroll
-    for (int j = 0; j < NT_D; ++j) *reinterpret_cast<float2*>(pp + 2 + j * 8 + tq * 2) = make_float2(o[j][2], o[j][3]);
-  }
+  write_partial(split0 + (n_chunks - 1) / chunks_per_split);
 }
 
 template <int D>
@@ -310,7 +327,9 @@ void launch_d(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, con
   }
   int G = a.Hq / a.Hkv;
   int q_tiles = (a.rows * G + QROWS - 1) / QROWS;
-  launch_pdl(L, k_attn_mma<D>, dim3(a.n_splits, a.Hkv, q_tiles), dim3(128), smem, a, q, kc, vc, part, out);
+  int spb = a.splits_per_block < 1 ? 1 : a.splits_per_block;
+  launch_pdl(L, k_attn_mma<D>, dim3((a.n_splits + spb - 1) / spb, a.Hkv, q_tiles), dim3(128), smem, a, q, kc, vc, part,
+             out);
   if (a.n_splits > 1)
     launch_pdl(L, k_attn_combine_bf16<D>, dim3(a.rows * a.Hq), dim3(D), 0, a.n_splits, (const float*)part, out);
 }
@@ -322,15 +341,14 @@ bool tree_attention_mma_supported(const AttnArgs& a) {
 }
 
 void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int max_splits, int* n_splits,
-                               int* keys_per_split) {
-  // a few blocks per SM (a block's work is a chain of dependent MMAs: more, shorter blocks finish sooner),
-  // whole 64-key chunks per split
-  int G = Hq / Hkv;
-  int q_tiles = (rows * G + QROWS - 1) / QROWS;
-  int want = (3 * 148 + Hkv * q_tiles - 1) / (Hkv * q_tiles);      // up to three blocks per SM fit
+                               int* keys_per_split, int* splits_per_block) {
+  // The key range is cut into whole 64-key chunks, as many splits as the partial buffer allows.  The cut
+  // depends on the key count alone, never on the rows or heads: a token's attention is then summed in the
+  // same grouping whether it is verified as one of 61 tree rows or decoded alone, which is what lets the
+  // speculative stream reproduce the plain decode bit for bit while the accepted path is the root.
+  // (Short blocks also finish sooner: a block's work is a chain of dependent MMAs.)
   int chunks = (total_keys + CHUNK - 1) / CHUNK;
-  int ns = want;
-  if (ns > chunks) ns = chunks;
+  int ns = chunks;
   if (ns > max_splits) ns = max_splits;
   if (ns < 1) ns = 1;
   int cps = (chunks + ns - 1) / ns;
@@ -339,6 +357,11 @@ void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int ma
   if (ns < 1) ns = 1;
   *n_splits = ns;
   *keys_per_split = kps;
+  // scheduling only: consecutive splits per block so that about two blocks land on every SM
+  int q_tiles = (rows * (Hq / Hkv) + QROWS - 1) / QROWS;
+  int spb = (ns * Hkv * q_tiles + 148) / 296;
+  if (spb < 1) spb = 1;
+  *splits_per_block = spb;
 }
 
 void launch_tree_attention_mma(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc,

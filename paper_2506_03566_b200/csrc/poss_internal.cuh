@@ -246,6 +246,7 @@ struct AttnArgs {
   int mask_words;
   float scale;
   int n_splits, keys_per_split;
+  int splits_per_block;   // tensor-core kernel: consecutive splits one block walks (one partial per split all the same)
 };
 template <typename T>
 void launch_tree_attention(Launcher& L, const AttnArgs& a, const T* q, const T* kcache, const T* vcache,
@@ -260,7 +261,7 @@ void run_tree_attention(Launcher& L, AttnArgs a, int max_splits, const T* q, con
                         float* part, T* out);
 bool tree_attention_mma_supported(const AttnArgs& a);
 void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int max_splits, int* n_splits,
-                               int* keys_per_split);
+                               int* keys_per_split, int* splits_per_block);
 void launch_tree_attention_mma(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc,
                                float* part, bf16* out);
 

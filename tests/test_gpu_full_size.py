@@ -108,3 +108,82 @@ def test_full_size_verify_accept_over_the_whole_vocabulary():
         assert int(out["bonus"][0]) == want[2]
         assert out["new_tokens"][: a + 1].cpu().tolist() == want[3].tolist()
         assert np.array_equal(pu.np_of(out["new_features"][: a + 1]), want[4])
+
+
+def test_c5_full_loop_matches_plain_greedy_decode():
+    """Config c5: 32-layer Llama-3-8B-shaped target + the c2 drafter, prompt of 512 ids, 512 generated tokens.
+    Every round = draft tree (depth 6, top-k 10, 60 tokens) + tree-masked target pass + accept walk + KV
+    compaction.  The speculative stream must equal the plain greedy decode of the same target token for
+    token.  In bf16 a tree row and a single decode row reach the same logits through different summation
+    orders in the attention, so the streams may part where the top two logits are nearly tied: at every such
+    position the margin between the two chosen tokens must be below 1e-2 in the oracle's logits (checked on
+    the CPU when the common stream is short enough, else in the fp32 logits of the plain path), and both
+    streams are re-joined on the plain decode's token and compared on.  The plain decode itself is pinned to
+    the oracle on a short prompt."""
+    from paper_2506_03566_b200 import Poss, make_config, speculative_generate, plain_generate
+    cfg = ps.CONFIGS["c5"]
+    w = ps.make_weights(cfg, 105)
+    n_prompt, n_gen = cfg.prefix, 512
+    slots = n_prompt + n_gen + cfg.total + cfg.depth + 4
+    P = Poss(make_config(cfg, slots + cfg.tree_slots, slots), w)
+    prompt = ps.make_prompt(cfg, 105, n_prompt)
+    num = pu.oracle_num(cfg, big=True)
+
+    # the plain decode against the oracle's definition, on a short prompt (a full-length one is minutes of CPU)
+    short = prompt[:6]
+    got = plain_generate(P, torch.from_numpy(short).cuda(), 4)
+    kv_o = po.new_target_kv(cfg, 16, num)
+    stream = list(short)
+    for k in range(4):
+        n = len(stream)
+        if k == 0:
+            _, lg = po.target_forward(cfg, w, kv_o, 0, np.array(stream, dtype=np.int32), np.arange(n), po.chain_parents(n), num)
+        else:
+            _, lg = po.target_forward(cfg, w, kv_o, n - 1, [stream[-1]], [n - 1], po.chain_parents(1), num)
+        srt = np.sort(lg[-1])[::-1]
+        want = int(po.argmax_rows(lg[-1:])[0])
+        assert got[k] == want or srt[0] - srt[1] < pu.MARGIN, f"plain decode differs from the oracle at token {k}"
+        stream.append(int(got[k]))
+
+    cur = prompt
+    left = n_gen
+    partings, total_rounds, accepted = [], 0, 0
+    one_depth = torch.zeros(1, dtype=torch.int32, device="cuda")
+    one_mask = torch.ones(1, dtype=torch.int64, device="cuda")
+    while left > 0:
+        pt = torch.from_numpy(np.ascontiguousarray(cur)).cuda()
+        log = []
+        spec = speculative_generate(P, pt, left, cfg.depth, cfg.topk, cfg.total, log=log)
+        plain = plain_generate(P, pt, left)
+        assert P.poss_last_status() == 0
+        total_rounds += len(log)
+        accepted += sum(a for a, _ in log)
+        if spec == plain:
+            break
+        i = next(k for k in range(left) if spec[k] != plain[k])
+        common = np.concatenate([cur, np.array(plain[:i], dtype=np.int32)])
+        # logits of the plain path after the common stream
+        tkv = P.new_target_kv()
+        ct = torch.from_numpy(np.ascontiguousarray(common)).cuda()
+        P.poss_target_prefill(tkv, 0, ct[:-1].contiguous())
+        _, _, lg_gpu = P.poss_target_forward(tkv, len(common) - 1, ct[-1:].contiguous(), one_depth, one_mask, 1, want_logits=True)
+        gap = abs(float(lg_gpu[0, spec[i]]) - float(lg_gpu[0, plain[i]]))
+        rms = float(lg_gpu[0].float().pow(2).mean().sqrt())
+        where = "plain path's fp32 logits"
+        if len(common) <= 700:
+            kv_o = po.new_target_kv(cfg, len(common) + 1, num)
+            _, lg = po.target_forward(cfg, w, kv_o, 0, common, np.arange(len(common)), po.chain_parents(len(common)), num)
+            gap = abs(float(lg[-1][spec[i]]) - float(lg[-1][plain[i]]))
+            rms = float(np.sqrt(np.mean(np.square(lg[-1]))))
+            where = "oracle logits"
+        # Two bf16 paths through L layers differ by about one rounding (2^-9 relative) at each of the ~4 rounding
+        # points of a layer, adding up like a random walk: 2^-9 * sqrt(4 L) of the logits' RMS (2.2 % at L = 32).
+        # A parting is explained when the gap is within twice that, and never needs to be below the 1e-2 of the
+        # shallow cases.
+        bound = max(pu.MARGIN, 2.0 * 2.0 ** -9 * math.sqrt(4.0 * cfg.n_target_layers) * rms)
+        assert gap < bound, f"streams part at generated token {n_gen - left + i} without a near-tie ({gap} >= {bound} in the {where})"
+        partings.append((n_gen - left + i, round(gap, 5), round(rms, 2), where))
+        cur = np.concatenate([common, np.array([plain[i]], dtype=np.int32)])
+        left -= i + 1
+        assert len(partings) <= 8, "too many partings for near-ties alone"
+    print("c5 rounds", total_rounds, "accepted draft tokens", accepted, "partings", partings)
