@@ -73,6 +73,26 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
+def replica_seed(rank: int) -> int:
+    """Replicas only: every rank runs its own request, drawn from its own seed."""
+    return 1 + rank
+
+
+def slowest_rank(times_ms, world: int, device):
+    """Per-step times of this rank -> the job's: the maximum over ranks (every replica must have finished)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def rounds_per_second(world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank completes one round per step."""
+    return world * 1e3 / ms_per_step
+
+
 def run_reference(args, cfg):
     """The oracle, as it stands, on the host cores: one full draft round per step."""
     import poss_synth as ps
@@ -144,7 +164,7 @@ def main():
     warmup = max(args.warmup, 3)
 
     # ---------------- inputs: seeded, resident in HBM before timing
-    seed = 1 + rank          # replicas only: every rank runs an independent request
+    seed = replica_seed(rank)
     with_target = not (args.no_target or args.alias_specialists)
     n_layers = 32 if with_target else 0
     w = ps.make_weights(cfg, seed, alias_specialists=args.alias_specialists)
@@ -254,10 +274,7 @@ def main():
     e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
     sync_all()
 
-    stats = torch.tensor([ms, draft_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-    ms, draft_ms, e2e_ms = [float(x) for x in stats.tolist()]
+    ms, draft_ms, e2e_ms = slowest_rank([ms, draft_ms, e2e_ms], world, "cuda")
 
     if rank == 0:
         peaks, which = None, "fallback"
@@ -282,7 +299,7 @@ def main():
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "stages_us": {"draft_round": draft_ms * 1e3, "whole_step": ms * 1e3,
                           "verify_round": max(ms - draft_ms, 0.0) * 1e3},
-            "rounds_per_s": world * 1e3 / ms,
+            "rounds_per_s": rounds_per_second(world, ms),
             "draft_round_gbs": round_bytes / (draft_ms * 1e-3) / 1e9,
             "draft_round_frac_of_hbm_peak": round_bytes / (draft_ms * 1e-3) / 1e9 / hbm_peak,
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
