@@ -59,7 +59,7 @@ constexpr int XCH_STRIDE = 17;
 struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
-  int n_tiles, kb_total, gran, w_policy;
+  int n_tiles, kb_total, gran, w_policy, slots, pair_tiles;
   const bf16* bias;
   const float* residual;
   int ldr;
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
       };
       auto load_w = [&](const Cursor& c, int s) {
         int kcoord = c.kb * TILE_K;
-        if (a.mode == 1) {           // 64 gate rows + 64 up rows of the same ffn columns
+        if (a.pair_tiles) {          // 64 gate rows + 64 up rows of the same ffn columns
           tma_load_2d(w_tile(s), &map_w0, full_bar(s), kcoord, c.tile * 64, pol_w);
           tma_load_2d(w_tile(s) + W_TILE_BYTES / 2, &map_w1, full_bar(s), kcoord, c.tile * 64, pol_w);
         } else {
@@ -526,9 +526,10 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
       } else {
         // partial K range (or a product whose reduction is left to the consumer): park the fp32 partial;
         // unless deferred, the last arriver of the tile finishes it
-        const int slot = (u == u0) ? 0 : 1;       // a range's first segment, or its trailing one
+        // deferred: segment s of the range goes to slot s; else a range's first segment (0) or its trailing one (1)
+        const int slot = a.mode == 3 ? seg_i : ((u == u0) ? 0 : 1);
         const size_t part_elems = (size_t)a.Npad * TILE_N;
-        float* part = a.scratch + ((size_t)blockIdx.x * 2 + slot) * part_elems;
+        float* part = a.scratch + ((size_t)blockIdx.x * a.slots + slot) * part_elems;
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
           float v[16];
           tmem_ld16(taddr + (uint32_t)c0, v);
@@ -767,6 +768,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   a.M = M;
   a.Npad = (M + 15) / 16 * 16;
   a.mode = ep.mode;
+  a.pair_tiles = ep.mode == TC_EPI_SWIGLU ? 1 : 0;
   a.n_segs = segs.n;
   const int tile_rows = ep.mode == TC_EPI_SWIGLU ? 64 : TILE_N;
   int n_tiles = 0, col = 0;
@@ -780,16 +782,23 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (ep.mode == TC_EPI_SWIGLU) n_tiles = a.seg_tiles[0];   // one tile = 64 gate + 64 up rows
   a.n_tiles = n_tiles;
   a.kb_total = (K + TILE_K - 1) / TILE_K;
-  // Leave the reduction to the consumer when the caller can take a view, every range is at most one
-  // tile long (so a CTA parks at most two segments) and groups of four columns never straddle a tile.
+  // Leave the reduction to the consumer when the caller can take a view, groups of four columns never
+  // straddle a tile and the parked segments fit the scratch (a CTA parks one segment per tile its range
+  // touches).
+  a.slots = 2;
   if (ep.view) {
     bool ok4 = true;
     for (int i = 0; i < segs.n; ++i) ok4 = ok4 && (segs.rows[i] % 4 == 0);
-    size_t need = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
-    bool defer = ep.mode == TC_EPI_STORE && ok4 && n_tiles <= cache->grid && need <= SCRATCH_PARTIAL_BYTES;
+    long long units = (long long)n_tiles * a.kb_total;
+    int g_eff = (long long)cache->grid < units ? cache->grid : (int)units;
+    long long range_max = (units + g_eff - 1) / g_eff;
+    int slots = (int)((range_max + a.kb_total - 1) / a.kb_total) + 1;
+    size_t need = (size_t)cache->grid * slots * a.Npad * TILE_N * sizeof(float);
+    bool defer = (ep.mode == TC_EPI_STORE || ep.mode == TC_EPI_SWIGLU) && ok4 && need <= SCRATCH_PARTIAL_BYTES;
     memset(ep.view, 0, sizeof(*ep.view));
     if (defer) {
       a.mode = TC_EPI_PARTIAL;
+      a.slots = slots;
     } else {
       ep.view->deferred = 0;
       ep.view->direct = ep.out;
@@ -818,6 +827,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
     v->deferred = 1;
     v->scratch = reinterpret_cast<const float*>(scratch);
     v->Npad = a.Npad; v->G = G; v->kb_total = a.kb_total; v->n_tiles = n_tiles; v->n_segs = segs.n;
+    v->slots = a.slots; v->swiglu = ep.mode == TC_EPI_SWIGLU ? 1 : 0;
     for (int i = 0; i < segs.n; ++i) { v->seg_tiles[i] = a.seg_tiles[i]; v->seg_rows[i] = a.seg_rows[i]; }
   }
   uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;

@@ -280,33 +280,37 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
   write_partial(split0 + (n_chunks - 1) / chunks_per_split);
 }
 
+// One block per (row, head), D threads.  Each warp first forms the split weights on its own: lane s loads
+// split s's (m, l) (at most 32 splits), the maximum and the normaliser come from warp reductions in a
+// fixed order; then every thread adds its output element over the splits in split order, all loads of
+// eight splits in flight at once.
 template <int D>
 __global__ void k_attn_combine_bf16(int n_splits, const float* part, bf16* out) {
   pdl_enter();
-  int rh = blockIdx.x;       // row * Hq + head
-  int e = threadIdx.x;
+  const int rh = blockIdx.x;       // row * Hq + head
+  const int e = threadIdx.x, lane = threadIdx.x & 31;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);
-  // split order is fixed; loads are issued eight splits at a time before they are used
-  float mm = NEG_BIG;
-  for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, __ldcg(pp + s * (D + 2)));
+  float pm = NEG_BIG, pl = 0.f;
+  if (lane < n_splits) { pm = __ldcg(pp + lane * (D + 2)); pl = __ldcg(pp + lane * (D + 2) + 1); }
+  float mm = pm;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+  const float c_lane = lane < n_splits ? __expf(pm - mm) : 0.f;
   float ll = 0.f, oo = 0.f;
   for (int base = 0; base < n_splits; base += 8) {
-    float pm[8], pl[8], po[8];
+    float po[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       int s = base + u;
-      if (s < n_splits) {
-        pm[u] = __ldcg(pp + s * (D + 2));
-        pl[u] = __ldcg(pp + s * (D + 2) + 1);
-        po[u] = __ldcg(pp + s * (D + 2) + 2 + e);
-      }
+      if (s < n_splits) po[u] = __ldcg(pp + s * (D + 2) + 2 + e);
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       int s = base + u;
       if (s < n_splits) {
-        float c = __expf(pm[u] - mm);
-        ll += pl[u] * c;
+        float c = __shfl_sync(0xffffffffu, c_lane, s);
+        float l = __shfl_sync(0xffffffffu, pl, s);
+        ll += l * c;
         oo += po[u] * c;
       }
     }

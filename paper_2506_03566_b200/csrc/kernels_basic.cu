@@ -419,6 +419,35 @@ template void launch_splitk_reduce<float>(Launcher&, const SplitKView&, int, int
 template void launch_splitk_reduce<bf16>(Launcher&, const SplitKView&, int, int, const bf16*, const float*, int, float*,
                                          int, bf16*);
 
+// ---- act = T(silu(gate) * up) from the parked partials of a SwiGLU product
+template <typename T>
+__global__ void __launch_bounds__(256) k_splitk_swiglu(SplitKView prod, int F, T* act) {
+  pdl_enter();
+  const int m = blockIdx.y;
+  const int f = (blockIdx.x * 256 + threadIdx.x) * 4;
+  if (f >= F) return;
+  int tile, t;
+  splitk_locate(prod, f, &tile, &t);
+  TileContrib tc = splitk_tile_contrib(prod, tile);
+  float4 g = splitk_load4(prod, m, f, tc, t);
+  float4 u = splitk_load4(prod, m, f, tc, t + 64);
+  float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (f + q < F) {
+      float sgl = gv[q] / (1.f + expf(-gv[q]));
+      act[(size_t)m * F + f + q] = from_f<T>(sgl * uv[q]);
+    }
+  }
+}
+template <typename T>
+void launch_splitk_swiglu(Launcher& L, const SplitKView& prod, int rows, int F, T* act) {
+  if (rows <= 0) return;
+  launch_pdl(L, k_splitk_swiglu<T>, dim3((F + 1023) / 1024, rows), dim3(256), 0, prod, F, act);
+}
+template void launch_splitk_swiglu<float>(Launcher&, const SplitKView&, int, int, float*);
+template void launch_splitk_swiglu<bf16>(Launcher&, const SplitKView&, int, int, bf16*);
+
 // ------------------------------------------------------------------ rotary embedding + KV append + q
 // The product's row layout is [Hq*d q | Hkv*d k | Hkv*d v] fp32.  Rotate-half pairing (j, j + d/2).
 // The angle pos * theta^(-2j/d) is formed in double from a table of the d/2 inverse frequencies and

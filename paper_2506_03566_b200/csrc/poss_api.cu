@@ -418,7 +418,12 @@ void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const voi
   if (tc_gemm_supported(sg, K, K, M)) {
     TcEpilogue ep;
     ep.mode = TC_EPI_SWIGLU; ep.out_bf = act; ep.ldo_bf = F;
+    // few rows: the last CTA of each tile finishes it in the kernel; many rows (the target pass): that
+    // tail grows with the row count, so the partials are left to a consumer kernel spread over all SMs
+    SplitKView v;
+    if (M > 16 && F % 4 == 0) ep.view = &v;
     launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
+    if (ep.view && v.deferred) launch_splitk_swiglu<bf16>(L, v, M, F, act);
     return;
   }
   gemm(x, K, M, sg, K, nullptr, nullptr, 0, c->b.gu, 2 * F);

@@ -115,13 +115,15 @@ inline void launch_pdl(Launcher& L, void (*kernel)(KArgs...), dim3 grid, dim3 bl
 // running in the last CTA of each tile.  A view with deferred == 0 is a plain fp32 matrix.
 //
 // Units are k-blocks in (tile, k-block) order; CTA c owns [range_begin(c), range_begin(c + 1)).  A CTA
-// holds at most two segments here (its range is not longer than a tile): slot 0 is the segment that
-// starts at the range's first unit, slot 1 the one that starts at a tile boundary inside the range.
+// numbers the tile segments of its range 0, 1, 2, ... in order (at most `slots` of them) and parks segment
+// s in its slot s.  In a SwiGLU product a tile holds 64 gate rows (rows 0..63) and the 64 up rows of the
+// same ffn columns (rows 64..127), so a tile covers 64 output columns.
 struct SplitKView {
-  const float* scratch;   // partial of (cta, slot): scratch + (cta * 2 + slot) * Npad * 128, element [m][row in tile]
+  const float* scratch;   // partial of (cta, slot): scratch + (cta * slots + slot) * Npad * 128, element [m][row in tile]
   const float* direct;    // deferred == 0: the product itself, [M][ld]
   int ld;
-  int deferred, Npad, G, kb_total, n_tiles;
+  int deferred, Npad, G, kb_total, n_tiles, slots;
+  int swiglu;             // tile layout: 0 = 128 output columns, 1 = 64 gate + 64 up rows
   int seg_tiles[3], seg_rows[3];   // tiles / rows of each weight segment (tiles never straddle segments)
   int n_segs;
 };
@@ -138,8 +140,9 @@ __host__ __device__ __forceinline__ int splitk_cta_of_unit(long long u, long lon
   return (int)c;
 }
 
-// Contributors of one tile: CTAs c_first .. c_first + count - 1; the first one's partial sits in
-// slot_first, every later one's in slot 0.
+// Contributors of one tile: CTAs c_first .. c_first + count - 1; the first one's partial sits in its slot
+// slot_first (the tile's ordinal among the tiles its range touches), every later one's in slot 0 (their
+// ranges begin inside the tile).
 struct TileContrib { int c_first, count, slot_first; };
 __device__ __forceinline__ TileContrib splitk_tile_contrib(const SplitKView& v, int tile) {
   long long groups = (long long)v.n_tiles * v.kb_total;
@@ -153,18 +156,19 @@ __device__ __forceinline__ TileContrib splitk_tile_contrib(const SplitKView& v, 
     if (cl > G - 1u) cl = G - 1u;
     t.c_first = (int)cf;
     t.count = (int)(cl - cf) + 1;
-    t.slot_first = (cf * gr / G) >= u0 ? 0 : 1;
+    t.slot_first = tile - (int)((cf * gr / G) / (unsigned)v.kb_total);
     return t;
   }
   long long tile_u0 = (long long)tile * v.kb_total;
   t.c_first = splitk_cta_of_unit(tile_u0, groups, v.G, 1);
   int c_last = splitk_cta_of_unit(tile_u0 + v.kb_total - 1, groups, v.G, 1);
   t.count = c_last - t.c_first + 1;
-  t.slot_first = splitk_range_begin(t.c_first, groups, v.G, 1) >= tile_u0 ? 0 : 1;
+  t.slot_first = tile - (int)(splitk_range_begin(t.c_first, groups, v.G, 1) / v.kb_total);
   return t;
 }
 // tile and row-in-tile of output column n (columns of the segments are laid side by side)
 __device__ __forceinline__ void splitk_locate(const SplitKView& v, int n, int* tile, int* t) {
+  if (v.swiglu) { *tile = n >> 6; *t = n & 63; return; }     // gate row; the up row of the same column is t + 64
   int base_tile = 0, nn = n;
   for (int s = 0; s < v.n_segs - 1 && nn >= v.seg_rows[s]; ++s) { nn -= v.seg_rows[s]; base_tile += v.seg_tiles[s]; }
   *tile = base_tile + nn / 128;
@@ -184,7 +188,7 @@ __device__ __forceinline__ float4 splitk_load4(const SplitKView& v, int m, int n
     for (int i = 0; i < 8; ++i) {
       int k = base + i;
       if (k < tc.count) {
-        size_t slot = (size_t)(tc.c_first + k) * 2 + (k == 0 ? tc.slot_first : 0);
+        size_t slot = (size_t)(tc.c_first + k) * v.slots + (k == 0 ? tc.slot_first : 0);
         x[i] = __ldcg(reinterpret_cast<const float4*>(p0 + slot * part));
       }
     }
@@ -233,6 +237,9 @@ void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T
 template <typename T>
 void launch_reduce_norm(Launcher& L, const SplitKView& prod, int rows, int H, const T* bias, const float* residual,
                         const T* gain, float eps, float* h, T* xn);
+// act[m][f] = T(silu(gate_f . x_m) * (up_f . x_m)) from the partials of a SwiGLU product (prod.swiglu == 1)
+template <typename T>
+void launch_splitk_swiglu(Launcher& L, const SplitKView& prod, int rows, int F, T* act);
 // out[m][n] (fp32, may be NULL) = product + bias[n] + residual[m][n]; out_act (may be NULL) the same in T
 template <typename T>
 void launch_splitk_reduce(Launcher& L, const SplitKView& prod, int rows, int N, const T* bias, const float* residual,
