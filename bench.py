@@ -118,7 +118,8 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: Llama-3-8B-shaped drafter, 6 specialists, depth 6, top-k 10, 60 tokens, prefix 1024"},
+            "config": {"workload": f"{cfg.name}: drafter H={cfg.hidden} F={cfg.ffn} V={cfg.vocab}, {cfg.S} specialists x {cfg.n} "
+                                   f"positions, depth {cfg.depth}, top-k {cfg.topk}, {cfg.total} tokens, prefix {cfg.prefix}"},
             "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
                              "sample": "one full draft round (numpy fp32, bf16 rounding contract); verify stages not included"},
             "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -291,8 +292,10 @@ def main():
             "metric": METRIC, "value": draft_ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: Llama-3-8B-shaped drafter, 6 specialists, depth 6, top-k 10, "
-                                   "60 tokens, prefix 1024; step = draft round + " +
+            "config": {"workload": f"{cfg.name}: drafter H={cfg.hidden} F={cfg.ffn} V={cfg.vocab} "
+                                   f"({'Llama-3-8B' if cfg.hidden == 4096 else 'Llama-2-13B' if cfg.hidden == 5120 else 'test'}-shaped), "
+                                   f"{cfg.S} specialists x {cfg.n} positions, depth {cfg.depth}, top-k {cfg.topk}, "
+                                   f"{cfg.total} tokens, prefix {cfg.prefix}; step = draft round + " +
                                    ("61-row tree-masked pass of a 32-layer Llama-3-8B-shaped target + accept walk + KV compaction"
                                     if with_target else "61-row verification attention + logits argmax + accept walk"),
                        "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)",

@@ -466,6 +466,35 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
             float thr = __shfl_sync(0xffffffffu, lv, K - 1);
             unsigned cand = __ballot_sync(0xffffffffu, val > thr);
             bool changed = false;
+            if (__popc(cand) > 8) {
+              // Many rows of this slice beat the list's last entry (a CTA's first tiles): place them all at
+              // once.  A candidate's final place is its rank inside the slice plus the list entries that stay
+              // ahead of it; a list entry's place is its index plus the candidates that pass it.  The order
+              // (value down, id up) is total, so the places 0..K-1 are each written exactly once.
+              int rank = 0;
+#pragma unroll 8
+              for (int l = 0; l < 32; ++l) {
+                float ov = __shfl_sync(0xffffffffu, val, l);
+                rank += better(ov, n_glob - lane + l, val, n_glob) ? 1 : 0;
+              }
+              const bool mine = val > thr && rank < K;
+              int ahead_me = 0, ahead_list = 0;
+              for (int j = 0; j < K; ++j) {
+                float ljv = __shfl_sync(0xffffffffu, lv, j);
+                int lji = __shfl_sync(0xffffffffu, li, j);
+                if (better(ljv, lji, val, n_glob)) ++ahead_me;
+                unsigned who = __ballot_sync(0xffffffffu, mine && rank == j);
+                if (who) {
+                  int src = __ffs(who) - 1;
+                  float cv = __shfl_sync(0xffffffffu, val, src);
+                  if (better(cv, n_glob - lane + src, lv, li)) ++ahead_list;
+                }
+              }
+              __syncwarp();
+              if (lane < K && lane + ahead_list < K) { lst_val[m * K + lane + ahead_list] = lv; lst_idx[m * K + lane + ahead_list] = li; }
+              if (mine && rank + ahead_me < K) { lst_val[m * K + rank + ahead_me] = val; lst_idx[m * K + rank + ahead_me] = n_glob; }
+              cand = 0;
+            }
             while (cand) {
               int src = __ffs(cand) - 1;
               cand &= cand - 1;
@@ -695,7 +724,7 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
-  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150, align_ranges = 1;
+  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150, align_ranges = 1, split_topk = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -713,6 +742,7 @@ TcGemmPlanCache* tc_plan_cache_create() {
   c->stages = 0;
   if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
   if (const char* e = getenv("POSS_TC_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 220) c->smem_kb = v; }
+  if (const char* e = getenv("POSS_TC_SPLIT_TOPK")) { int v = atoi(e); if (v >= 0 && v <= 1) c->split_topk = v; }
   if (const char* e = getenv("POSS_TC_ALIGN")) { int v = atoi(e); if (v >= 0 && v <= 1) c->align_ranges = v; }
   if (const char* e = getenv("POSS_TC_W_POLICY")) { int v = atoi(e); if (v >= 0 && v <= 1) c->w_policy = v; }
   return c;
@@ -805,10 +835,14 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
       ep.view->ld = ep.ldo;
     }
   }
-  // whole tiles per CTA for the LM head (its epilogue keeps running state across tiles), and whenever
-  // the partial buffers or the tile counters could not hold the split
+  // whole tiles per CTA for the argmax epilogue (its state lives in registers and only the whole-tile path
+  // feeds it), and whenever the partial buffers or the tile counters could not hold the split.  The top-k
+  // epilogue takes split tiles like any other: a CTA meets its tiles in increasing order either way, so
+  // "a later equal value loses" still means "the lower id wins".
+  const bool argmax = ep.mode == TC_EPI_TOPK && ep.argmax_only && ep.topk == 1 && a.Npad <= 64;
   size_t part_bytes = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
-  bool no_split = a.mode == TC_EPI_TOPK || part_bytes > SCRATCH_PARTIAL_BYTES || n_tiles > N_COUNTERS;
+  bool no_split = argmax || (a.mode == TC_EPI_TOPK && !cache->split_topk) || part_bytes > SCRATCH_PARTIAL_BYTES ||
+                  n_tiles > N_COUNTERS;
   a.gran = no_split ? a.kb_total : 1;
   // never more CTAs than ranges to hand out: every CTA of the grid owns at least one k-block
   long long groups = (long long)n_tiles * a.kb_total / a.gran;
@@ -834,7 +868,6 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
-  const bool argmax = ep.mode == TC_EPI_TOPK && ep.argmax_only && ep.topk == 1 && a.Npad <= 64;
   if (ep.mode == TC_EPI_TOPK && !argmax) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
   int stages = cache->stages ? cache->stages : (int)(((size_t)cache->smem_kb * 1024u - extra - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;

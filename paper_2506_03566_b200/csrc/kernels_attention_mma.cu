@@ -63,8 +63,9 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
   lo = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
 }
 
-template <int D>
-__global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
+// NW = warps per block: 4 (64 query rows) or, when one KV head has at most 16 query rows, 1
+template <int D, int NW>
+__global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
                                                   const bf16* kcache, const bf16* vcache,
                                                   float* part, bf16* out) {
   constexpr int LD = D + 8;                       // padded shared-memory row, elements
@@ -81,10 +82,10 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
   const int G = a.Hq / a.Hkv;
   const int n_q = a.rows * G;                     // query rows of this KV head
   const int quad = lane >> 2, tq = lane & 3;
-  const int qi0 = qtile * QROWS + warp * 16 + quad, qi1 = qi0 + 8;
+  const int qi0 = qtile * (16 * NW) + warp * 16 + quad, qi1 = qi0 + 8;
   const bool v0 = qi0 < n_q, v1 = qi1 < n_q;
   const int r0 = v0 ? qi0 / G : 0, r1 = v1 ? qi1 / G : 0;
-  const bool warp_active = qtile * QROWS + warp * 16 < n_q;
+  const bool warp_active = qtile * (16 * NW) + warp * 16 < n_q;
 
   // the block walks splits_per_block consecutive splits as one chunk sequence and emits one partial per
   // split: how many splits a block takes is a scheduling choice, the grouping of the sums is not
@@ -102,7 +103,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(AttnArgs a, const bf16* q,
     bf16* kd = Ks + (size_t)stage * CHUNK * LD;
     bf16* vd = Vs + (size_t)stage * CHUNK * LD;
     constexpr int PER_ROW = D / 8;                // 16-byte pieces per key
-    for (int i = threadIdx.x; i < CHUNK * PER_ROW; i += 128) {
+    for (int i = threadIdx.x; i < CHUNK * PER_ROW; i += 32 * NW) {
       int kr = i / PER_ROW, piece = i % PER_ROW;
       int key = key0 + kr;
       bool ok = key < k_end;
@@ -318,24 +319,31 @@ __global__ void k_attn_combine_bf16(int n_splits, const float* part, bf16* out) 
   out[(size_t)rh * D + e] = __float2bfloat16_rn(oo / ll);
 }
 
-template <int D>
-void launch_d(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc, float* part, bf16* out) {
+template <int D, int NW>
+void launch_dn(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc, float* part, bf16* out) {
   constexpr size_t smem = (size_t)2 * 2 * CHUNK * (D + 8) * sizeof(bf16);
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(k_attn_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_attn_mma<D, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
     attr_done = true;
   }
   int G = a.Hq / a.Hkv;
-  int q_tiles = (a.rows * G + QROWS - 1) / QROWS;
+  int q_tiles = (a.rows * G + 16 * NW - 1) / (16 * NW);
   int spb = a.splits_per_block < 1 ? 1 : a.splits_per_block;
-  launch_pdl(L, k_attn_mma<D>, dim3((a.n_splits + spb - 1) / spb, a.Hkv, q_tiles), dim3(128), smem, a, q, kc, vc, part,
-             out);
+  launch_pdl(L, k_attn_mma<D, NW>, dim3((a.n_splits + spb - 1) / spb, a.Hkv, q_tiles), dim3(32 * NW), smem, a, q, kc, vc,
+             part, out);
   if (a.n_splits > 1)
     launch_pdl(L, k_attn_combine_bf16<D>, dim3(a.rows * a.Hq), dim3(D), 0, a.n_splits, (const float*)part, out);
+}
+template <int D>
+void launch_d(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc, float* part, bf16* out) {
+  // few query rows per KV head (multi-head attention with a short row batch): one-warp blocks, so that the
+  // grid has more, shorter blocks instead of blocks with three idle warps
+  if (a.rows * (a.Hq / a.Hkv) <= 16) launch_dn<D, 1>(L, a, q, kc, vc, part, out);
+  else launch_dn<D, 4>(L, a, q, kc, vc, part, out);
 }
 
 }  // namespace
@@ -362,8 +370,10 @@ void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int ma
   *n_splits = ns;
   *keys_per_split = kps;
   // scheduling only: consecutive splits per block so that about two blocks land on every SM
-  int q_tiles = (rows * (Hq / Hkv) + QROWS - 1) / QROWS;
-  int spb = (ns * Hkv * q_tiles + 148) / 296;
+  int nq = rows * (Hq / Hkv);
+  int q_tiles = nq <= 16 ? 1 : (nq + QROWS - 1) / QROWS;
+  int per_sm = nq <= 16 ? 3 : 2;                    // blocks that fit an SM at once
+  int spb = (ns * Hkv * q_tiles + 74 * per_sm) / (148 * per_sm);
   if (spb < 1) spb = 1;
   *splits_per_block = spb;
 }
