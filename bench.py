@@ -311,7 +311,10 @@ def main():
             "clocks": clocks.summary(),
             "roofline": {"bound": "hbm", "kernel": "k_gemm_tc on the LM head (V x H bf16)", "achieved": achieved,
                          "peak": hbm_peak, "peak_source": which, "unit": "GB/s",
-                         "frac": achieved / hbm_peak if achieved else None, "traffic": None,
+                         "frac": achieved / hbm_peak if achieved else None,
+                         # dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch, from the ncu capture
+                         # summarised in profiles/k_gemm_tc_c2_m10_gateup_down_lmhead.md (c2 shapes only)
+                         "traffic": 1050894000 + 9812224 if cfg.name in ("c2", "c4", "c5") else None,
                          "launches_timed": n_lm, "avg_launch_us": lm_dur * 1e3,
                          "algorithmic_bytes_per_launch": lm_bytes},
         }
