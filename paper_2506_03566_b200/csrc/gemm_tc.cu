@@ -23,7 +23,10 @@
 // Epilogues: (0) fp32 store with bias / residual and an optional bf16 copy; (1) SwiGLU: the tile holds
 // 64 gate rows and 64 up rows of the same ffn columns and the epilogue writes bf16(silu(g) * u);
 // (2) LM head: running max / sum-exp / top-k per activation row over the CTA's vocabulary tiles, one
-// partial list per CTA, the logits never reach memory.
+// partial list per CTA, the logits never reach memory (template variant: argmax only, every lane keeps
+// its rows' best in registers); (3) nothing: every tile segment is parked as an fp32 partial and the
+// kernel that consumes the product adds a tile's segments in range order while it loads (no counter, no
+// last-arriver tail: that reduction is spread over all of the consumer's blocks).
 //
 // Programmatic dependent launch: the kernel lets its successor start early and itself prefetches
 // weight tiles (which no kernel writes) before it waits for its predecessor's results.
