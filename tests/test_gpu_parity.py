@@ -208,6 +208,16 @@ ROUND_CASES = [
     ("m_bf16", {}, 1, 12, False),
     ("m_bf16", {"S": 3, "n": 2}, 7, 13, False),
     ("m_bf16", {"S": 4, "n": 2, "depth": 8, "total": 80}, 3, 14, False),
+    # the kernels' limits: 128 rows in one projection batch (8 verified pairs + 120 tree slots = (depth-1)*topk),
+    # 255 kept tokens (four mask words per row), 1815 candidates in the rerank; width 16 at depth 8
+    # (cumulative scores near -50 at depth 9: an fp32 unit there is 4e-6, so two candidates 1e-6 apart in the fp64
+    # oracle may swap places on the GPU; the teacher-forced comparison with the margin rule covers that)
+    ("t_fp32", {"S": 3, "n": 3, "depth": 9, "topk": 15, "total": 255}, 1, 15, False),
+    ("t_bf16", {"S": 2, "n": 5, "depth": 9, "topk": 15, "total": 200}, 8, 16, False),
+    ("t_bf16", {"S": 4, "n": 2, "depth": 8, "topk": 16, "total": 100}, 3, 19, False),
+    # degenerate: one step, one candidate; chain drafting in bf16
+    ("t_bf16", {"depth": 1, "topk": 1, "total": 1}, 1, 17, False),
+    ("t_bf16", {"S": 6, "n": 1, "depth": 6, "topk": 1, "total": 6}, 2, 18, False),
 ]
 
 
