@@ -103,7 +103,7 @@ def test_tree_attention_matches_oracle(name, rows, P_len, Hq, Hkv, d):
 
 
 @pytest.mark.parametrize("name,rows,K", [("t_fp32", 3, 3), ("t_fp32", 1, 16), ("t_bf16", 4, 4), ("m_bf16", 10, 10),
-                                         ("m_bf16", 61, 1)])
+                                         ("m_bf16", 61, 1), ("t_bf16", 128, 16), ("m_bf16", 64, 3), ("m_bf16", 17, 16)])
 def test_lm_head_topk_matches_oracle(name, rows, K):
     cfg = ps.CONFIGS[name]
     w = ps.make_weights(cfg.replace(S=1, n_target_layers=0), 2)
@@ -299,17 +299,17 @@ def test_capacity_and_argument_errors_are_reported():
 
 # ----------------------------------------------------------------------------- target pass and the full loop
 
-@pytest.mark.parametrize("name", ["t_fp32", "t_bf16"])
-def test_target_forward_tree_rows_match_oracle(name):
+@pytest.mark.parametrize("name,n,rows", [("t_fp32", 40, 25), ("t_bf16", 40, 25), ("t_bf16", 130, 64), ("t_bf16", 7, 128)])
+def test_target_forward_tree_rows_match_oracle(name, n, rows):
+    """Prefill (one or two chunks) and a tree pass; 64 rows is the widest argmax-epilogue launch, 128 the row limit."""
     cfg = ps.CONFIGS[name]
     w = ps.make_weights(cfg, 31)
-    n, rows = 40, 25
-    P = make_poss(cfg, w, 64, 128)
+    P = make_poss(cfg, w, 64, n + rows + 8)
     num = pu.oracle_num(cfg)
     prompt = ps.make_prompt(cfg, 31, n)
     tkv = P.new_target_kv()
     feats, arg = P.poss_target_prefill(tkv, 0, torch.from_numpy(prompt).cuda())
-    kv_o = po.new_target_kv(cfg, 128, num)
+    kv_o = po.new_target_kv(cfg, n + rows + 8, num)
     f_o, l_o = po.target_forward(cfg, w, kv_o, 0, prompt, np.arange(n), po.chain_parents(n), num)
     tol = pu.TOL[cfg.dtype]
     assert np.abs(pu.np_of(feats) - f_o).max() <= tol
