@@ -134,6 +134,10 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--config", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--depth", type=int, help="override the workload's draft depth L")
+    ap.add_argument("--total", type=int, help="override the workload's kept draft tokens T")
+    ap.add_argument("--specialists", type=int, help="override the number of position specialists S")
+    ap.add_argument("--positions", type=int, help="override the positions per specialist n (PosS-n)")
     ap.add_argument("--no-target", action="store_true", help="verification side = stand-alone stages, no target layers")
     ap.add_argument("--alias-specialists", action="store_true",
                     help="profiler captures only: all specialists share one weight set, so the process holds "
@@ -143,6 +147,10 @@ def main():
 
     import poss_synth as ps
     cfg = ps.CONFIGS[args.config]
+    over = {k: v for k, v in (("depth", args.depth), ("total", args.total), ("S", args.specialists), ("n", args.positions))
+            if v is not None}
+    if over:
+        cfg = cfg.replace(**over)
     if args.impl == "reference":
         run_reference(args, cfg)
         return
