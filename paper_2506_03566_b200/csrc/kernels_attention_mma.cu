@@ -169,10 +169,13 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
       // ---- S = Q K^T for 16 query rows x 64 keys
       float s[CHUNK / 8][4];
 #pragma unroll
-      for (int j = 0; j < CHUNK / 8; ++j) {
-        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      for (int j = 0; j < CHUNK / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      // k-steps outside, key tiles inside: consecutive MMAs write different accumulators and pipeline
+      // (each accumulator still receives its k-steps in order 0, 1, 2, ...)
 #pragma unroll
-        for (int kk = 0; kk < KSTEPS; kk += 2) {
+      for (int kk = 0; kk < KSTEPS; kk += 2) {
+#pragma unroll
+        for (int j = 0; j < CHUNK / 8; ++j) {
           uint32_t b0, b1, b2, b3;
           uint32_t addr = smem_u32(kd + (j * 8 + (lane & 7)) * LD + kk * 16 + (lane >> 3) * 8);
           ldmatrix_x4(addr, b0, b1, b2, b3);
@@ -243,8 +246,8 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
           uint32_t addr = smem_u32(vd + (ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + (jd + (lane >> 4)) * 8);
           ldmatrix_x4_trans(addr, b0, b1, b2, b3);
           mma_bf16(o[jd], ph, b0, b1);
-          mma_bf16(o[jd], pl, b0, b1);
           mma_bf16(o[jd + 1], ph, b2, b3);
+          mma_bf16(o[jd], pl, b0, b1);
           mma_bf16(o[jd + 1], pl, b2, b3);
         }
       }
