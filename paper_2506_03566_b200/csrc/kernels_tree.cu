@@ -518,25 +518,49 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
                                                  float* out_scores, int32_t* out_depth,
                                                  uint64_t* out_mask, int32_t* out_n_nodes) {
   extern __shared__ unsigned char smem_raw[];
+  __shared__ int wtot[32];
   pdl_enter();
   float* sc = reinterpret_cast<float*>(smem_raw);               // [n_cand]
   int* newidx = reinterpret_cast<int*>(sc + n_cand);            // [n_cand] node index or 0 if dropped
+  int* par = newidx + n_cand;                                   // [n_cand] parent candidate
   int keep = min(total, n_cand);
   int words = (total + 1 + 63) / 64;
-  for (int c = threadIdx.x; c < n_cand; c += blockDim.x) sc[c] = ts.cand_score[c];
+  for (int c = threadIdx.x; c < n_cand; c += blockDim.x) { sc[c] = ts.cand_score[c]; par[c] = ts.cand_parent[c]; }
   __syncthreads();
+  // kept iff fewer than `keep` candidates order before it; the count stops as soon as it says "dropped"
+  // (most candidates: the better ones sit at the low, early-level indices that are scanned first)
   for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
     float s = sc[c];
     int rank = 0;
-    for (int o = 0; o < n_cand; ++o) rank += better(sc[o], o, s, c) ? 1 : 0;
+    for (int o0 = 0; o0 < n_cand && rank < keep; o0 += 8) {
+      int hi = min(o0 + 8, n_cand);
+      for (int o = o0; o < hi; ++o) rank += better(sc[o], o, s, c) ? 1 : 0;
+    }
     newidx[c] = rank < keep ? 1 : 0;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {               // ordered compaction; n_cand is at most a few thousand
-    int nxt = 1;
-    for (int c = 0; c < n_cand; ++c) {
-      if (newidx[c]) { ts.selected[nxt - 1] = c; newidx[c] = nxt++; }
+  // ordered compaction: node index = 1 + number of kept candidates with a lower flat index
+  {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    int base = 0;
+    for (int c0 = 0; c0 < n_cand; c0 += blockDim.x) {
+      int c = c0 + threadIdx.x;
+      bool kept = c < n_cand && newidx[c] != 0;
+      unsigned b = __ballot_sync(0xffffffffu, kept);
+      if (lane == 0) wtot[warp] = __popc(b);
+      __syncthreads();
+      int before = base, all = 0;
+      for (int w = 0; w < n_warps; ++w) { int t = wtot[w]; if (w < warp) before += t; all += t; }
+      if (kept) {
+        int node = 1 + before + __popc(b & ((1u << lane) - 1u));
+        newidx[c] = node;
+        ts.selected[node - 1] = c;
+      }
+      base += all;
+      __syncthreads();
     }
+  }
+  if (threadIdx.x == 0) {
     out_tokens[0] = root_tok[0];
     out_parents[0] = -1;
     out_scores[0] = 0.f;
@@ -544,11 +568,10 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
     for (int w = 0; w < words; ++w) out_mask[w] = w == 0 ? 1ull : 0ull;
     out_n_nodes[0] = keep + 1;
   }
-  __syncthreads();
   for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
     int node = newidx[c];
     if (!node) continue;
-    int pc = ts.cand_parent[c];
+    int pc = par[c];
     out_tokens[node] = ts.cand_tok[c];
     out_parents[node] = pc < 0 ? 0 : newidx[pc];
     out_scores[node] = sc[c];
@@ -558,7 +581,7 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
     while (cur >= 0) {
       int nd = newidx[cur];
       m[nd >> 6] |= 1ull << (nd & 63);
-      cur = ts.cand_parent[cur];
+      cur = par[cur];
     }
     for (int w = 0; w < words; ++w) out_mask[(size_t)node * words + w] = m[w];
   }
@@ -572,7 +595,7 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
 void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, int root_tok_index,
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
-  size_t smem = (size_t)n_cand * 8;
+  size_t smem = (size_t)n_cand * 12;
   launch_pdl(L, k_rerank, dim3(1), dim3(1024), smem, ts, n_cand, K, total, new_tokens + root_tok_index, out_tokens,
              out_parents, out_scores, out_depth, out_mask, out_n_nodes);
 }
