@@ -241,7 +241,7 @@ def main():
 
     # ---------------- timed region 1: inputs resident in HBM
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-    P.poss_profile(True)
+    P.poss_profile(1)
     launches0 = P.poss_launch_count()
     with ClockSampler(local) as clocks:
         sync_all()
@@ -252,8 +252,8 @@ def main():
         sync_all()
     ms = ev[0].elapsed_time(ev[1]) / args.steps
     launches = (P.poss_launch_count() - launches0) // args.steps
-    n_lm, lm_ms = P.poss_profile_read()
-    P.poss_profile(False)
+    n_lm, lm_ms = P.poss_profile_read()["lm_head"]
+    P.poss_profile(0)
 
     # draft round alone (the metric's own quantity)
     sync_all()
@@ -263,6 +263,15 @@ def main():
     ev[3].record()
     sync_all()
     draft_ms = ev[2].elapsed_time(ev[3]) / args.steps
+
+    # every stage kind of the draft steps in isolation (events around each stage cut the launch overlap, so
+    # this loop is slower than the round above and only feeds the per-kernel table)
+    P.poss_profile(2)
+    for _ in range(min(args.steps, 10)):
+        P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total, out=out)
+    per_kind = P.poss_profile_read()
+    P.poss_profile(0)
+    sync_all()
 
     # ---------------- timed region 2: end to end through the C ABI with host buffers
     res_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items() if k != "anc_mask"}
@@ -326,6 +335,17 @@ def main():
                          "launches_timed": n_lm, "avg_launch_us": lm_dur * 1e3,
                          "algorithmic_bytes_per_launch": lm_bytes},
         }
+        H_, F_, V_ = cfg.hidden, cfg.ffn, cfg.vocab
+        qd_, kd_ = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+        avg_keys = cfg.prefix + 1 + cfg.topk * (cfg.depth - 1) / 2.0
+        kind_bytes = {"fc": 2 * 2 * H_ * H_, "qkv": 2 * H_ * (qd_ + 2 * kd_), "attention": 2 * 2 * kd_ * avg_keys,
+                      "o": 2 * qd_ * H_, "gate_up": 2 * 2 * F_ * H_, "down": 2 * F_ * H_, "lm_head": 2 * V_ * H_}
+        line["kernels"] = {
+            k: {"launches": n, "avg_us": t / n * 1e3, "algorithmic_bytes": kind_bytes[k],
+                "gbs": kind_bytes[k] / (t / n * 1e-3) / 1e9, "frac_of_hbm_peak": kind_bytes[k] / (t / n * 1e-3) / 1e9 / hbm_peak}
+            for k, (n, t) in per_kind.items() if n}
+        line["kernels_note"] = ("each stage of the draft steps between two CUDA events of its own (isolated: no overlap with its "
+                                "neighbours); gate_up includes the SwiGLU, attention its combine kernel; bytes = weights (or K/V) only")
         if not args.no_cpu_baseline and world == 1:
             from oracle import poss_oracle as po
             wr = ps.make_weights(cfg, seed)

@@ -198,11 +198,17 @@ POSS_API int poss_linear(poss_ctx* ctx, const void* x, int M, const void* w, int
 POSS_API int poss_lm_head_topk(poss_ctx* ctx, const void* features, int rows, int topk,
                       int32_t* out_ids, float* out_logp, float* out_logits, poss_stream stream);
 
-/* Device-time bracketing of the dominant kernel, the LM-head matrix product of a draft step: while enabled,
- * each of those launches (not the target pass's argmax launch) sits between two CUDA events on the launching stream (at most 1024 launches between
- * reads).  poss_profile_read SYNCHRONISES on the last event, returns how many launches were
- * bracketed since the previous read and their summed device time in ms, and starts over. */
-POSS_API int poss_profile(poss_ctx* ctx, int enable);
+/* Device-time bracketing of the draft steps' stages, for roofline reporting.  mode 0: off; mode 1: the LM-head
+ * matrix product (the dominant kernel) of every draft step sits between two CUDA events on the launching stream;
+ * mode 2: so does every stage kind below (the launches between the two events are the product's kernel, plus the
+ * combine kernel for POSS_PROF_ATTENTION and the in-kernel or consumer-side SwiGLU for POSS_PROF_GATE_UP).  The
+ * events cut the overlap between neighbouring launches, so mode 2 times each stage in isolation and lengthens the
+ * round; at most 1024 brackets between reads.  poss_profile_read SYNCHRONISES on the last event, returns per kind
+ * how many launches were bracketed since the previous read and their summed device time in ms (arrays of
+ * POSS_PROF_KINDS entries), and starts over.  The target pass is never bracketed. */
+enum { POSS_PROF_FC = 0, POSS_PROF_QKV = 1, POSS_PROF_ATTENTION = 2, POSS_PROF_O = 3, POSS_PROF_GATE_UP = 4,
+       POSS_PROF_DOWN = 5, POSS_PROF_LM_HEAD = 6, POSS_PROF_KINDS = 7 };
+POSS_API int poss_profile(poss_ctx* ctx, int mode);
 POSS_API int poss_profile_read(poss_ctx* ctx, int* h_launches, float* h_total_ms);
 
 /* Tree-masked attention for callers that cannot allocate device memory (the paper has no

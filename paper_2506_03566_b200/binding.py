@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(HERE, "libposs.so")
 
 POSS_FP32, POSS_BF16 = 0, 1
 POSS_MAX_ROWS, POSS_MAX_TOPK, POSS_MAX_DEPTH = 128, 16, 16
+PROF_KINDS = ("fc", "qkv", "attention", "o", "gate_up", "down", "lm_head")
 STATUS = {0: "POSS_OK", 1: "POSS_E_INVALID", 2: "POSS_E_SHAPE", 3: "POSS_E_CAPACITY", 4: "POSS_E_WORKSPACE",
           5: "POSS_E_CUDA", 6: "POSS_E_TIMEOUT"}
 
@@ -306,13 +307,15 @@ class Poss:
                                           _stream()), "poss_lm_head_topk")
         return ids, logp, logits
 
-    def poss_profile(self, enable: bool):
-        _check(self.lib.poss_profile(self.ctx, int(enable)), "poss_profile")
+    def poss_profile(self, mode):
+        _check(self.lib.poss_profile(self.ctx, int(mode)), "poss_profile")
 
     def poss_profile_read(self):
-        n, ms = C.c_int(), C.c_float()
-        _check(self.lib.poss_profile_read(self.ctx, C.byref(n), C.byref(ms)), "poss_profile_read")
-        return n.value, ms.value
+        """-> {kind name: (launches, total ms)}"""
+        n = (C.c_int * len(PROF_KINDS))()
+        ms = (C.c_float * len(PROF_KINDS))()
+        _check(self.lib.poss_profile_read(self.ctx, n, ms), "poss_profile_read")
+        return {k: (int(n[i]), float(ms[i])) for i, k in enumerate(PROF_KINDS)}
 
     def poss_launch_count(self) -> int:
         return int(self.lib.poss_launch_count(self.ctx))

@@ -71,8 +71,9 @@ struct poss_ctx {
   int64_t launches;
   int last_depth, last_topk, last_nodes;
   TcGemmPlanCache* tc;
-  bool prof_on;
+  int prof_mode;         // 0 off, 1 = LM-head launches of the draft steps, 2 = every stage kind of the draft steps
   int prof_n;
+  int prof_kind[1024];   // kind of each bracketed launch
   cudaEvent_t* prof_ev;   // 2 * PROF_MAX events, created on first enable
 };
 constexpr int PROF_MAX = 1024;
@@ -165,6 +166,18 @@ struct Impl {
   Launcher L;
   Impl(poss_ctx* ctx, poss_stream s) : c(ctx) { L.stream = S(s); L.launches = &ctx->launches; L.err = POSS_OK; }
 
+  // brackets the launches issued between begin and end with two events (profiling only)
+  int prof_begin(int kind) {
+    if (!c->prof_mode || !in_draft || c->prof_n >= PROF_MAX) return -1;
+    if (c->prof_mode == 1 && kind != POSS_PROF_LM_HEAD) return -1;
+    int i = c->prof_n++;
+    c->prof_kind[i] = kind;
+    cudaEventRecord(c->prof_ev[2 * i], L.stream);
+    return i;
+  }
+  void prof_end(int i) { if (i >= 0) cudaEventRecord(c->prof_ev[2 * i + 1], L.stream); }
+  bool in_draft = false;
+
   const T* W(const void* p) const { return reinterpret_cast<const T*>(p); }
   T* A(void* p) const { return reinterpret_cast<T*>(p); }
 
@@ -186,12 +199,11 @@ struct Impl {
     const poss_config& g = c->cfg;
     GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = g.vocab;
     float* lg = logits_out ? logits_out : c->b.logits;
-    bool prof = c->prof_on && c->prof_n < PROF_MAX && expand != nullptr;   // the draft steps' launches only
-    if (prof) cudaEventRecord(c->prof_ev[2 * c->prof_n], L.stream);
+    int pr = expand != nullptr ? prof_begin(POSS_PROF_LM_HEAD) : -1;   // the draft steps' launches only
     int n_lists = 0;
     bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists, !need_logp && K == 1);
     if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
-    if (prof) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], L.stream); ++c->prof_n; }
+    prof_end(pr);
     if (!fused) {
       launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
       n_lists = c->n_chunks;
@@ -208,11 +220,15 @@ struct Impl {
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
     launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), W(c->embed), H, A(b.X));
     GemmSegs fc; fc.n = 1; fc.w[0] = lw.fc_w; fc.rows[0] = H;
+    int pr = prof_begin(POSS_PROF_FC);
     SplitKView v_fc = gemm_view(A(b.X), 2 * H, s.M, fc, 2 * H, b.ptmp, H);
+    prof_end(pr);
     launch_reduce_norm<T>(L, v_fc, s.M, H, W(lw.fc_b), nullptr, W(lw.norm_in), g.rms_eps, b.h0, A(b.xn));
     GemmSegs qkv; qkv.n = 3;
     qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
+    pr = prof_begin(POSS_PROF_QKV);
     SplitKView v_qkv = gemm_view(A(b.xn), H, s.M, qkv, H, b.ptmp, qd + 2 * kd);
+    prof_end(pr);
     RopeArgs ra;
     ra.inv_freq = b.rope_inv;
     ra.mode = 0; ra.s = s; ra.base = 0; ra.depth = nullptr; ra.rows = s.M; ra.q_rows = with_q ? s.Mc : 0;
@@ -229,11 +245,17 @@ struct Impl {
     Buffers& b = c->b;
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, F = g.ffn;
     GemmSegs so; so.n = 1; so.w[0] = lw.wo; so.rows[0] = H;
+    int pr = prof_begin(POSS_PROF_O);
     SplitKView v_o = gemm_view(A(b.o), qd, rows, so, qd, b.ptmp, H);
+    prof_end(pr);
     launch_reduce_norm<T>(L, v_o, rows, H, nullptr, x0, W(lw.norm_post), g.rms_eps, b.h1, A(b.u));
+    pr = prof_begin(POSS_PROF_GATE_UP);
     gemm_swiglu(A(b.u), rows, lw.w_gate, lw.w_up, F, H, A(b.act));
+    prof_end(pr);
     GemmSegs sd; sd.n = 1; sd.w[0] = lw.w_down; sd.rows[0] = H;
+    pr = prof_begin(POSS_PROF_DOWN);
     SplitKView v_d = gemm_view(A(b.act), F, rows, sd, F, b.ptmp, H);
+    prof_end(pr);
     if (next_gain) launch_reduce_norm<T>(L, v_d, rows, H, nullptr, b.h1, next_gain, g.rms_eps, out, out_act);
     else launch_splitk_reduce<T>(L, v_d, rows, H, nullptr, b.h1, H, out, H, out_act);
   }
@@ -264,6 +286,7 @@ struct Impl {
     size_t half = per_spec / 2;
     bool used[64] = {false};
     int cand_base = 0;
+    in_draft = true;
     for (int i = 0; i < depth; ++i) {
       int s = i / n < Sn - 1 ? i / n : Sn - 1;          // specialist ceil((i+1)/n), clamped, 0-based
       bool first = !used[s < 64 ? s : 63];
@@ -284,7 +307,9 @@ struct Impl {
       aa.n_all = prefix_len + n_new; aa.n_tree = i * K;
       aa.mask = b.ts.node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
+      int pr = prof_begin(POSS_PROF_ATTENTION);
       run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
+      prof_end(pr);
       float* fo = b.fout + (size_t)i * KMAX * H;
       T* fbi = A(b.fb) + (size_t)i * KMAX * H;
       layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo, fbi);
@@ -489,7 +514,7 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   if (c->tgt) memcpy(c->tgt, w->h_target, sizeof(poss_layer_w) * cfg->n_target_layers);
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->target_final_norm;
   c->esize = cfg->dtype == POSS_BF16 ? 2 : 4;
-  c->prof_on = false; c->prof_n = 0; c->prof_ev = nullptr;
+  c->prof_mode = 0; c->prof_n = 0; c->prof_ev = nullptr;
   c->launches = 0; c->last_depth = 0; c->last_topk = 0; c->last_nodes = 0;
   Bump bp;
   bp.base = reinterpret_cast<char*>(workspace);
@@ -730,33 +755,30 @@ int poss_lm_head_topk(poss_ctx* c, const void* features, int rows, int topk, int
   return im.L.err;
 }
 
-int poss_profile(poss_ctx* c, int enable) {
-  if (!c) return POSS_E_INVALID;
-  if (enable && !c->prof_ev) {
+int poss_profile(poss_ctx* c, int mode) {
+  if (!c || mode < 0 || mode > 2) return POSS_E_INVALID;
+  if (mode && !c->prof_ev) {
     c->prof_ev = (cudaEvent_t*)malloc(sizeof(cudaEvent_t) * 2 * PROF_MAX);
     if (!c->prof_ev) return POSS_E_INVALID;
     for (int i = 0; i < 2 * PROF_MAX; ++i)
       if (cudaEventCreate(&c->prof_ev[i]) != cudaSuccess) return POSS_E_CUDA;
   }
-  c->prof_on = enable != 0;
+  c->prof_mode = mode;
   c->prof_n = 0;
   return POSS_OK;
 }
 
 int poss_profile_read(poss_ctx* c, int* h_launches, float* h_total_ms) {
   if (!c || !h_launches || !h_total_ms) return POSS_E_INVALID;
-  *h_launches = 0;
-  *h_total_ms = 0.f;
+  for (int k = 0; k < POSS_PROF_KINDS; ++k) { h_launches[k] = 0; h_total_ms[k] = 0.f; }
   if (!c->prof_ev || c->prof_n == 0) return POSS_OK;
   if (cudaEventSynchronize(c->prof_ev[2 * c->prof_n - 1]) != cudaSuccess) return POSS_E_CUDA;
-  float total = 0.f;
   for (int i = 0; i < c->prof_n; ++i) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) return POSS_E_CUDA;
-    total += ms;
+    h_launches[c->prof_kind[i]] += 1;
+    h_total_ms[c->prof_kind[i]] += ms;
   }
-  *h_launches = c->prof_n;
-  *h_total_ms = total;
   c->prof_n = 0;
   return POSS_OK;
 }
