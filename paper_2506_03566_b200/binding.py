@@ -74,6 +74,7 @@ EXPORTS = {
     "poss_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_float)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
+    "poss_debug_lose_load": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_tree_attention_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                               C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
 }
@@ -316,6 +317,9 @@ class Poss:
         ms = (C.c_float * len(PROF_KINDS))()
         _check(self.lib.poss_profile_read(self.ctx, n, ms), "poss_profile_read")
         return {k: (int(n[i]), float(ms[i])) for i, k in enumerate(PROF_KINDS)}
+
+    def poss_debug_lose_load(self, launches: int):
+        _check(self.lib.poss_debug_lose_load(self.ctx, int(launches)), "poss_debug_lose_load")
 
     def poss_launch_count(self) -> int:
         return int(self.lib.poss_launch_count(self.ctx))

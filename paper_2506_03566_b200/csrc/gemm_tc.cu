@@ -54,7 +54,7 @@ constexpr int TILE_K = 64;           // bf16 elements per k-block = one 128-byte
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
 constexpr int MAX_STAGES = 12;
 constexpr int N_THREADS = 192;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;     // one second: far beyond any launch of this library
 constexpr size_t SCRATCH_PARTIAL_BYTES = 96ull << 20;
 constexpr int N_COUNTERS = 8192;
 constexpr int XCH_STRIDE = 17;
@@ -63,6 +63,7 @@ struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
   int n_tiles, kb_total, gran, w_policy, slots, pair_tiles;
+  int inject_lost_load;   // test hook: the producer leaves out the activation tile of its first stage
   const bf16* bias;
   const float* residual;
   int ldr;
@@ -101,12 +102,23 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// bounded wait; returns false when it gave up or when another role already raised the abort flag
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after WAIT_LIMIT_NS of wall time (the clock is read every 64 polls, a poll may
+// itself suspend for a system-dependent while) or as soon as another role has raised the abort flag.
+// Returns false in both cases; on expiry it raises the flag itself.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*abort_flag) return false;
+      uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_LIMIT_NS) break;
       if (it > 4096u) __nanosleep(64);
     }
   }
@@ -305,7 +317,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         advance(cw);
       }
       pdl_wait();
-      for (int it = 0; it < pre; ++it) { load_x(cx, it); advance(cx); }
+      for (int it = 0; it < pre; ++it) { if (!(a.inject_lost_load && it == 0)) load_x(cx, it); advance(cx); }
       int issued = pre, s = 0;
       uint32_t phase = 0;                     // parity of the "empty" completion that frees stage s next
       for (int it = pre; it < n_kb; ++it) {
@@ -321,7 +333,8 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         // drain: every copy this thread started must land before the CTA's shared memory goes away
         for (int it = max(0, issued - S); it < issued; ++it) {
           uint32_t bar = full_bar(it % S), par = (uint32_t)((it / S) & 1);
-          for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(bar, par); ++w) __nanosleep(64);
+          uint64_t t0 = global_ns();
+          while (!mbar_try_wait(bar, par) && global_ns() - t0 < WAIT_LIMIT_NS / 4) __nanosleep(64);
         }
       }
     }
@@ -727,6 +740,7 @@ struct MapKeyHash {
 struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
+  int inject = 0;          // launches left whose first activation tile is withheld (wait-expiry test hook)
   int grid = 0, stages = 0, w_policy = 1, smem_kb = 150, align_ranges = 1, split_topk = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
@@ -751,6 +765,7 @@ TcGemmPlanCache* tc_plan_cache_create() {
   return c;
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
+void tc_inject_lost_load(TcGemmPlanCache* c, int launches) { c->inject = launches < 0 ? 0 : launches; }
 size_t tc_gemm_scratch_bytes() { return SCRATCH_PARTIAL_BYTES + N_COUNTERS * sizeof(int); }
 
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M) {
@@ -877,6 +892,8 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (stages < 2) stages = 2;
   a.n_stages = stages;
   a.w_policy = cache->w_policy;
+  a.inject_lost_load = cache->inject > 0 ? 1 : 0;
+  if (cache->inject > 0) --cache->inject;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);

@@ -5,6 +5,8 @@
 struct TcGemmPlanCache;
 TcGemmPlanCache* tc_plan_cache_create();
 void tc_plan_cache_destroy(TcGemmPlanCache*);
+// test hook: the next `launches` launches withhold one activation tile, so one of their bounded waits runs out
+void tc_inject_lost_load(TcGemmPlanCache*, int launches);
 size_t tc_gemm_scratch_bytes();
 // true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 8, ...)
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);

@@ -783,6 +783,12 @@ int poss_profile_read(poss_ctx* c, int* h_launches, float* h_total_ms) {
   return POSS_OK;
 }
 
+int poss_debug_lose_load(poss_ctx* c, int launches) {
+  if (!c || launches < 0) return POSS_E_INVALID;
+  tc_inject_lost_load(c->tc, launches);
+  return POSS_OK;
+}
+
 int64_t poss_launch_count(const poss_ctx* c) { return c ? c->launches : 0; }
 
 }  // extern "C"

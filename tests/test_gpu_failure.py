@@ -1,0 +1,39 @@
+"""Failure detection on the device, without a fault: a bounded wait that runs out.
+
+The tensor-core matrix product waits on shared-memory barriers for its TMA copies and for its own tensor-core
+work.  Every such wait gives up after about one second, raises POSS_E_TIMEOUT in the context's status word, and
+the CTA leaves in order (copies in flight awaited, tensor memory freed).  The test hook withholds one activation
+tile from one launch, so exactly that happens; afterwards the same context must work as before."""
+import numpy as np
+import pytest
+import torch
+
+import poss_synth as ps
+from oracle import poss_oracle as po
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    from paper_2506_03566_b200 import Poss, make_config, to_device
+    cfg = ps.CONFIGS["t_bf16"].replace(n_target_layers=0)
+    P = Poss(make_config(cfg, 512), ps.make_weights(cfg, 1))
+    M, N, K = 10, 1408, 512
+    x = ps.normal(5, "x", (M, K), 1.0, "bf16")
+    W = ps.normal(5, "w", (N, K), 0.02, "bf16")
+    xd, Wd = to_device(x), to_device(W)
+    want = po.linear(po.widen(x, np.float64), W, pu.oracle_num(cfg))
+    good = P.poss_linear(xd, Wd, impl=2).cpu().numpy()
+    assert P.poss_last_status() == 0
+    assert np.abs(good - want).max() <= 1e-4
+
+    P.poss_debug_lose_load(1)
+    P.poss_linear(xd, Wd, impl=2)                  # results undefined; must neither fault nor hang
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 6               # POSS_E_TIMEOUT
+
+    P.poss_reset()
+    again = P.poss_linear(xd, Wd, impl=2).cpu().numpy()
+    assert P.poss_last_status() == 0
+    assert np.array_equal(again, good)
