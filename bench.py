@@ -37,40 +37,48 @@ def algorithmic_bytes(cfg):
 
 
 class ClockSampler:
+    """One `nvidia-smi -lms` process for the whole measurement; samples are stamped on arrival and the summary
+    keeps those that fell inside the timed regions."""
     Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
 
-    def __init__(self, index: int):
-        self.rows, self.stop, self.index = [], False, index
-        self.t = threading.Thread(target=self.run, daemon=True)
-
-    def run(self):
-        while not self.stop:
-            try:
-                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
-                self.rows.append([c.strip() for c in out.strip().split(",")])
-            except Exception:
-                pass
-            time.sleep(0.1)
-
-    def __enter__(self):
+    def __init__(self, gpu_id: str, period_ms: int = 20):
+        self.rows, self.windows, self.proc = [], [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", str(period_ms)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            return
+        self.t = threading.Thread(target=self._read, daemon=True)
         self.t.start()
-        return self
 
-    def __exit__(self, *a):
-        self.stop = True
-        self.t.join(timeout=6)
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.strip().split(",")]))
+
+    def window(self, t0: float, t1: float):
+        self.windows.append((t0, t1))
+
+    def close(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
 
     def summary(self):
-        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        inside = [r for t, r in self.rows if len(r) >= 7 and any(a <= t <= b for a, b in self.windows)]
+        num = lambda x: x.replace(".", "", 1).isdigit()
+        sm = [float(r[0]) for r in inside if num(r[0])]
+        mx = [float(r[1]) for r in inside if num(r[1])]
+        pw = [float(r[2]) for r in inside if num(r[2])]
         reasons = []
         for name, col in (("hw_slowdown", 3), ("hw_thermal_slowdown", 4), ("sw_thermal_slowdown", 5), ("sw_power_cap", 6)):
-            if any(len(r) >= 7 and r[col].lower().startswith("active") for r in self.rows):
+            if any(r[col].lower().startswith("active") for r in inside):
                 reasons.append(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+                "power_w_max": max(pw) if pw else None, "reasons": reasons, "samples": len(sm)}
 
 
 def replica_seed(rank: int) -> int:
@@ -243,13 +251,20 @@ def main():
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
     P.poss_profile(1)
     launches0 = P.poss_launch_count()
-    with ClockSampler(local) as clocks:
-        sync_all()
-        ev[0].record()
-        for _ in range(args.steps):
-            step(tok_d, feat_d)
-        ev[1].record()
-        sync_all()
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        gpu_id = str(local)
+    clocks = ClockSampler(gpu_id)
+    time.sleep(0.3)                       # let the sampler come up before the timed region
+    sync_all()
+    t_a = time.perf_counter()
+    ev[0].record()
+    for _ in range(args.steps):
+        step(tok_d, feat_d)
+    ev[1].record()
+    sync_all()
+    clocks.window(t_a, time.perf_counter())
     ms = ev[0].elapsed_time(ev[1]) / args.steps
     launches = (P.poss_launch_count() - launches0) // args.steps
     n_lm, lm_ms = P.poss_profile_read()["lm_head"]
@@ -257,11 +272,14 @@ def main():
 
     # draft round alone (the metric's own quantity)
     sync_all()
+    t_a = time.perf_counter()
     ev[2].record()
     for _ in range(args.steps):
         P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total, out=out)
     ev[3].record()
     sync_all()
+    clocks.window(t_a, time.perf_counter())
+    clocks.close()
     draft_ms = ev[2].elapsed_time(ev[3]) / args.steps
 
     # every stage kind of the draft steps in isolation (events around each stage cut the launch overlap, so
