@@ -9,12 +9,6 @@
 // result does not depend on scheduling.
 #include "poss_internal.cuh"
 
-#define LAUNCH_CHECK(L)                                         \
-  do {                                                          \
-    ++*(L).launches;                                            \
-    if (cudaGetLastError() != cudaSuccess) (L).err = POSS_E_CUDA; \
-  } while (0)
-
 #define NEG_BIG (-1.0e30f)
 
 template <typename T, int D> struct KeyLoad;

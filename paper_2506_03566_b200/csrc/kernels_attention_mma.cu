@@ -18,12 +18,6 @@
 #include "poss_internal.cuh"
 #include <string.h>
 
-#define LAUNCH_CHECK(L)                                         \
-  do {                                                          \
-    ++*(L).launches;                                            \
-    if (cudaGetLastError() != cudaSuccess) (L).err = POSS_E_CUDA; \
-  } while (0)
-
 namespace {
 
 constexpr float NEG_BIG = -1.0e30f;

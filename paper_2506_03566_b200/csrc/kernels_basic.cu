@@ -1,12 +1,6 @@
 // Element-wise stages and the SIMT skinny matrix product (check mode and odd shapes).
 #include "poss_internal.cuh"
 
-#define LAUNCH_CHECK(L)                                         \
-  do {                                                          \
-    ++*(L).launches;                                            \
-    if (cudaGetLastError() != cudaSuccess) (L).err = POSS_E_CUDA; \
-  } while (0)
-
 // ------------------------------------------------------------------ SIMT skinny GEMM
 // out[m][n] = sum_k X[m][k] * W[n][k] (+ bias[n]) (+ residual[m][n]).  One warp per output column n,
 // eight rows of X at a time in registers.  The reduction order of an output element depends only on
@@ -227,16 +221,6 @@ void launch_cast_rows(Launcher& L, const float* x, size_t n, T* out) {
 }
 template void launch_cast_rows<float>(Launcher&, const float*, size_t, float*);
 template void launch_cast_rows<bf16>(Launcher&, const float*, size_t, bf16*);
-
-__global__ void k_widen_bf16(const bf16* x, size_t n, float* out) {
-  pdl_enter();
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = __bfloat162float(x[i]);
-}
-void launch_widen_bf16(Launcher& L, const bf16* x, size_t n, float* out) {
-  if (n == 0) return;
-  launch_pdl(L, k_widen_bf16, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, x, n, out);
-}
 
 // act = T(silu(gate) * up), gate/up stored side by side: gu[row][0..F) gate, [F..2F) up
 template <typename T>

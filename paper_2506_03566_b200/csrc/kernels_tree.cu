@@ -4,12 +4,6 @@
 #include <math.h>
 #include <string.h>
 
-#define LAUNCH_CHECK(L)                                         \
-  do {                                                          \
-    ++*(L).launches;                                            \
-    if (cudaGetLastError() != cudaSuccess) (L).err = POSS_E_CUDA; \
-  } while (0)
-
 #define NEG_INF (-INFINITY)
 
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }

@@ -217,7 +217,6 @@ template <typename T>
 void launch_rmsnorm(Launcher& L, const float* x, int rows, int H, const T* gain, float eps, T* out);
 template <typename T>
 void launch_cast_rows(Launcher& L, const float* x, size_t n, T* out);
-void launch_widen_bf16(Launcher& L, const bf16* x, size_t n, float* out);
 template <typename T>
 void launch_silu_mul(Launcher& L, const float* gu, int rows, int F, T* out);
 
