@@ -187,8 +187,9 @@ POSS_API int poss_last_status(poss_ctx* ctx, poss_stream stream);
 /* ---- single stages, exported for kernel-level parity tests and roofline timing ---- */
 
 /* out[M][N] (fp32) = x[M][K] . w[N][K]^T (+ bias[N]) (+ residual[M][N], fp32).  x, w, bias in the
- * context dtype.  M <= POSS_MAX_ROWS.  impl: 0 = default for the dtype, 1 = SIMT kernel,
- * 2 = tcgen05 tensor-core kernel (bf16 only; K % 64 == 0). */
+ * context dtype.  M <= POSS_MAX_ROWS, K % 8 == 0.  impl: 0 = default for the dtype, 1 = SIMT kernel,
+ * 2 = tcgen05 tensor-core kernel (bf16 only; w 16-byte aligned) followed, as inside a round, by the kernel that
+ * adds its split-K partials.  A row's result does not depend on M or on the row's place in the batch. */
 POSS_API int poss_linear(poss_ctx* ctx, const void* x, int M, const void* w, int N, int K,
                 const void* bias, const float* residual, float* out, int impl, poss_stream stream);
 
