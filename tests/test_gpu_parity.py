@@ -384,3 +384,26 @@ def test_bf16_loop_is_lossless_against_its_own_plain_decode():
         srt = np.sort(lg[-1])[::-1]
         assert srt[0] - srt[1] < pu.MARGIN, "streams diverge without a near-tie"
     assert sum(a for a, _ in log) > 0
+
+
+def test_round_on_a_side_stream_equals_the_default_stream_bitwise():
+    """All work is enqueued on the caller's stream: the same round on a non-default stream, with other work
+    running on the default stream meanwhile, gives the same bits."""
+    cfg = ps.CONFIGS["t_bf16"].replace(n_target_layers=0)
+    w = ps.make_weights(cfg, 51)
+    cap = cfg.prefix + 2 + cfg.tree_slots
+    P = make_poss(cfg, w, cap)
+    kv = ps.make_draft_kv(cfg, 51, cap)
+    tok, feat = ps.make_round_inputs(cfg, 51, 2)
+    g, trace, _ = pu.run_gpu_round(P, cfg, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total)
+    side = torch.cuda.Stream()
+    noise = torch.randn(4096, 4096, device="cuda")
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            noise_out = noise @ noise                    # unrelated work on the default stream's neighbour
+        g2, trace2, _ = pu.run_gpu_round(P, cfg, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total)
+    torch.cuda.synchronize()
+    for k in ("tokens", "parents", "scores", "depth", "anc_mask"):
+        assert np.array_equal(g[k], g2[k]), k
+    assert np.array_equal(trace["step_features"], trace2["step_features"])
+    assert P.poss_last_status() == 0
