@@ -266,6 +266,31 @@ __device__ __forceinline__ float4 product4(const SplitKView& v, const TileContri
   return r;
 }
 
+// four consecutive elements at a 4-element-aligned position, as one access
+template <typename T> __device__ __forceinline__ void load4(const T* p, float* o);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float* o) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+template <> __device__ __forceinline__ void load4<bf16>(const bf16* p, float* o) {
+  uint2 raw = *reinterpret_cast<const uint2*>(p);
+  float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+  float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+  o[0] = a.x; o[1] = a.y; o[2] = b.x; o[3] = b.y;
+}
+template <typename T> __device__ __forceinline__ void store4(T* p, const float* v);
+template <> __device__ __forceinline__ void store4<float>(float* p, const float* v) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ __forceinline__ void store4<bf16>(bf16* p, const float* v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  uint2 raw;
+  raw.x = *reinterpret_cast<uint32_t*>(&a);
+  raw.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = raw;
+}
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
 // ---- h = product + bias + residual (fp32, stored);  xn = T(gain * h / rms(h))
 // One block per row.  The sum of squares is formed in a fixed order (per-thread partial sums over the
 // thread's column groups, a warp tree, then the warps in order), so a row's result does not depend on
@@ -286,16 +311,23 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
   const int m = blockIdx.x;
   const int n_groups = (H + 3) / 4;
   float ss = 0.f;
+  // whole 16-byte (fp32) / 8-byte (bf16) accesses when the row length and every base pointer allow it
+  const bool vec = (H & 3) == 0 && aligned16(h) && aligned16(xn) && (!residual || aligned16(residual)) &&
+                   (!bias || aligned16(bias)) && (!gain || aligned16(gain));
   // value of one group of four columns: product + bias + residual, stored to h, squares added to ss
   auto group_value = [&](int g) {
     const int n = g * 4;
-    float add[4];                           // bias + residual, loaded before the product's partials are awaited
+    float add[4] = {0.f, 0.f, 0.f, 0.f};    // bias + residual, loaded before the product's partials are awaited
+    if (vec) {
+      if (residual) load4<float>(residual + (size_t)m * H + n, add);
+      if (bias) { float b4[4]; load4<T>(bias + n, b4); add[0] += b4[0]; add[1] += b4[1]; add[2] += b4[2]; add[3] += b4[3]; }
+    } else {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      add[q] = 0.f;
-      if (n + q < H) {
-        if (residual) add[q] = residual[(size_t)m * H + n + q];
-        if (bias) add[q] += to_f(bias[n + q]);
+      for (int q = 0; q < 4; ++q) {
+        if (n + q < H) {
+          if (residual) add[q] = residual[(size_t)m * H + n + q];
+          if (bias) add[q] += to_f(bias[n + q]);
+        }
       }
     }
     float4 v = product4(prod, tab, m, n, H);
@@ -304,17 +336,31 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     for (int q = 0; q < 4; ++q) {
       if (n + q < H) {
         e[q] += add[q];
-        h[(size_t)m * H + n + q] = e[q];
         ss = fmaf(e[q], e[q], ss);
       } else {
         e[q] = 0.f;
       }
+    }
+    if (vec) store4<float>(h + (size_t)m * H + n, e);
+    else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) if (n + q < H) h[(size_t)m * H + n + q] = e[q];
     }
     return make_float4(e[0], e[1], e[2], e[3]);
   };
   auto group_store = [&](int g, float4 v, float inv) {
     const int n = g * 4;
     float e[4] = {v.x, v.y, v.z, v.w};
+    if (vec) {
+      if (gain) {
+        float g4[4];
+        load4<T>(gain + n, g4);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) e[q] = e[q] * inv * g4[q];
+      }
+      store4<T>(xn + (size_t)m * H + n, e);
+      return;
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q)
       if (n + q < H) xn[(size_t)m * H + n + q] = gain ? from_f<T>(e[q] * inv * to_f(gain[n + q])) : from_f<T>(e[q]);
