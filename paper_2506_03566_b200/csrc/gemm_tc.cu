@@ -455,8 +455,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
               int m = c0 + j;
               if (m < a.M && n_ok) {
                 float g = v[j], up = xch[t * XCH_STRIDE + j];
-                float s = g / (1.f + expf(-g));
-                a.out_bf[(size_t)m * a.ldo_bf + col] = __float2bfloat16_rn(s * up);
+                a.out_bf[(size_t)m * a.ldo_bf + col] = __float2bfloat16_rn(silu_f(g) * up);
               }
             }
           }

@@ -278,42 +278,56 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
   write_partial(split0 + (n_chunks - 1) / chunks_per_split);
 }
 
-// One block per (row, head), D threads.  Each warp first forms the split weights on its own: lane s loads
-// split s's (m, l) (at most 32 splits), the maximum and the normaliser come from warp reductions in a
-// fixed order; then every thread adds its output element over the splits in split order, all loads of
-// eight splits in flight at once.
+// One warp per (row, head), four warps per block.  Lane s loads split s's (m, l) (at most 32 splits); the
+// maximum comes from a warp reduction, the normaliser and the outputs are added over the splits in split
+// order.  A lane owns D/32 output elements as pairs (2*lane, 2*lane+1) (+64 for the second pair of D = 128):
+// 8-byte loads, eight splits in flight at once.
 template <int D>
-__global__ void k_attn_combine_bf16(int n_splits, const float* part, bf16* out) {
+__global__ void __launch_bounds__(128) k_attn_combine_bf16(int n_splits, int n_rh, const float* part, bf16* out) {
+  constexpr int NP = D / 64;             // pairs per lane
   pdl_enter();
-  const int rh = blockIdx.x;       // row * Hq + head
-  const int e = threadIdx.x, lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31;
+  const int rh = blockIdx.x * 4 + (threadIdx.x >> 5);       // row * Hq + head
+  if (rh >= n_rh) return;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);
   float pm = NEG_BIG, pl = 0.f;
-  if (lane < n_splits) { pm = __ldcg(pp + lane * (D + 2)); pl = __ldcg(pp + lane * (D + 2) + 1); }
+  if (lane < n_splits) {
+    float2 ml = __ldcg(reinterpret_cast<const float2*>(pp + lane * (D + 2)));
+    pm = ml.x;
+    pl = ml.y;
+  }
   float mm = pm;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
   const float c_lane = lane < n_splits ? __expf(pm - mm) : 0.f;
-  float ll = 0.f, oo = 0.f;
+  const float lc_lane = pl * c_lane;
+  float ll = 0.f;
+  float2 oo[NP];
+#pragma unroll
+  for (int h = 0; h < NP; ++h) oo[h] = make_float2(0.f, 0.f);
+  const float* pe = pp + 2 + 2 * lane;
   for (int base = 0; base < n_splits; base += 8) {
-    float po[8];
+    float2 po[8][NP];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      int s = base + u;
-      if (s < n_splits) po[u] = __ldcg(pp + s * (D + 2) + 2 + e);
+      if (base + u < n_splits) {
+#pragma unroll
+        for (int h = 0; h < NP; ++h) po[u][h] = __ldcg(reinterpret_cast<const float2*>(pe + (base + u) * (D + 2) + 64 * h));
+      }
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      int s = base + u;
-      if (s < n_splits) {
-        float c = __shfl_sync(0xffffffffu, c_lane, s);
-        float l = __shfl_sync(0xffffffffu, pl, s);
-        ll += l * c;
-        oo += po[u] * c;
+      if (base + u < n_splits) {
+        const float c = __shfl_sync(0xffffffffu, c_lane, base + u);
+        ll += __shfl_sync(0xffffffffu, lc_lane, base + u);
+#pragma unroll
+        for (int h = 0; h < NP; ++h) { oo[h].x += po[u][h].x * c; oo[h].y += po[u][h].y * c; }
       }
     }
   }
-  out[(size_t)rh * D + e] = __float2bfloat16_rn(oo / ll);
+#pragma unroll
+  for (int h = 0; h < NP; ++h)
+    *reinterpret_cast<__nv_bfloat162*>(out + (size_t)rh * D + 2 * lane + 64 * h) = __floats2bfloat162_rn(oo[h].x / ll, oo[h].y / ll);
 }
 
 template <int D, int NW>
@@ -333,7 +347,8 @@ void launch_dn(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, co
   launch_pdl(L, k_attn_mma<D, NW>, dim3((a.n_splits + spb - 1) / spb, a.Hkv, q_tiles), dim3(32 * NW), smem, a, q, kc, vc,
              part, out);
   if (a.n_splits > 1)
-    launch_pdl(L, k_attn_combine_bf16<D>, dim3(a.rows * a.Hq), dim3(D), 0, a.n_splits, (const float*)part, out);
+    launch_pdl(L, k_attn_combine_bf16<D>, dim3((a.rows * a.Hq + 3) / 4), dim3(128), 0, a.n_splits, a.rows * a.Hq,
+               (const float*)part, out);
 }
 template <int D>
 void launch_d(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc, float* part, bf16* out) {

@@ -230,8 +230,7 @@ __global__ void k_silu_mul(const float* gu, int F, T* out) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= F) return;
   float g = gu[(size_t)row * 2 * F + i], u = gu[(size_t)row * 2 * F + F + i];
-  float s = g / (1.f + expf(-g));
-  out[(size_t)row * F + i] = from_f<T>(s * u);
+  out[(size_t)row * F + i] = from_f<T>(silu_f(g) * u);
 }
 template <typename T>
 void launch_silu_mul(Launcher& L, const float* gu, int rows, int F, T* out) {
@@ -291,10 +290,21 @@ template <> __device__ __forceinline__ void store4<bf16>(bf16* p, const float* v
 }
 __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// four consecutive entries of a weight vector (bias, gain) as floats; `fill` where there is none
+template <typename T>
+__device__ __forceinline__ void load_w4(const T* w, int n, int N, bool vec, float fill, float* o) {
+  o[0] = o[1] = o[2] = o[3] = fill;
+  if (!w) return;
+  if (vec) { load4<T>(w + n, o); return; }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) if (n + q < N) o[q] = to_f(w[n + q]);
+}
+
 // ---- h = product + bias + residual (fp32, stored);  xn = T(gain * h / rms(h))
 // One block per row.  The sum of squares is formed in a fixed order (per-thread partial sums over the
 // thread's column groups, a warp tree, then the warps in order), so a row's result does not depend on
-// the batch around it.
+// the batch around it.  bias and gain are weights (no kernel writes them): they are read, and the
+// contributors of every tile worked out, before the predecessor is awaited.
 #define NORM_THREADS 1024
 #define NORM_KEEP 2
 template <typename T>
@@ -304,32 +314,39 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
   __shared__ TileContrib tab[512];
   __shared__ float red[NORM_THREADS / 32];
   __shared__ float inv_s;
-  pdl_enter();
+  pdl_begin();
   fill_tile_table(prod, tab);
-  __syncthreads();
-  POSS_TRACE_POINT(1);
   const int m = blockIdx.x;
   const int n_groups = (H + 3) / 4;
-  float ss = 0.f;
   // whole 16-byte (fp32) / 8-byte (bf16) accesses when the row length and every base pointer allow it
   const bool vec = (H & 3) == 0 && aligned16(h) && aligned16(xn) && (!residual || aligned16(residual)) &&
                    (!bias || aligned16(bias)) && (!gain || aligned16(gain));
-  // value of one group of four columns: product + bias + residual, stored to h, squares added to ss
-  auto group_value = [&](int g) {
-    const int n = g * 4;
-    float add[4] = {0.f, 0.f, 0.f, 0.f};    // bias + residual, loaded before the product's partials are awaited
-    if (vec) {
-      if (residual) load4<float>(residual + (size_t)m * H + n, add);
-      if (bias) { float b4[4]; load4<T>(bias + n, b4); add[0] += b4[0]; add[1] += b4[1]; add[2] += b4[2]; add[3] += b4[3]; }
-    } else {
+  float kb[NORM_KEEP][4], kg[NORM_KEEP][4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (n + q < H) {
-          if (residual) add[q] = residual[(size_t)m * H + n + q];
-          if (bias) add[q] += to_f(bias[n + q]);
-        }
+  for (int k = 0; k < NORM_KEEP; ++k) {
+    const int g = threadIdx.x + k * NORM_THREADS;
+    if (g < n_groups) {
+      load_w4<T>(bias, g * 4, H, vec, 0.f, kb[k]);
+      load_w4<T>(gain, g * 4, H, vec, 1.f, kg[k]);
+    }
+  }
+  __syncthreads();
+  pdl_sync();
+  POSS_TRACE_POINT(1);
+  float ss = 0.f;
+  // value of one group of four columns: product + (residual + bias), stored to h, squares added to ss
+  auto group_value = [&](int g, const float* b4) {
+    const int n = g * 4;
+    float add[4] = {0.f, 0.f, 0.f, 0.f};
+    if (residual) {
+      if (vec) load4<float>(residual + (size_t)m * H + n, add);
+      else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) if (n + q < H) add[q] = residual[(size_t)m * H + n + q];
       }
     }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) add[q] += b4[q];
     float4 v = product4(prod, tab, m, n, H);
     float e[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -348,30 +365,30 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     }
     return make_float4(e[0], e[1], e[2], e[3]);
   };
-  auto group_store = [&](int g, float4 v, float inv) {
+  auto group_store = [&](int g, float4 v, float inv, const float* g4) {
     const int n = g * 4;
     float e[4] = {v.x, v.y, v.z, v.w};
-    if (vec) {
-      if (gain) {
-        float g4[4];
-        load4<T>(gain + n, g4);
+    if (gain) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) e[q] = e[q] * inv * g4[q];
-      }
-      store4<T>(xn + (size_t)m * H + n, e);
-      return;
+      for (int q = 0; q < 4; ++q) e[q] = e[q] * inv * g4[q];
     }
+    if (vec) store4<T>(xn + (size_t)m * H + n, e);
+    else {
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      if (n + q < H) xn[(size_t)m * H + n + q] = gain ? from_f<T>(e[q] * inv * to_f(gain[n + q])) : from_f<T>(e[q]);
+      for (int q = 0; q < 4; ++q) if (n + q < H) xn[(size_t)m * H + n + q] = from_f<T>(e[q]);
+    }
   };
   float4 keep[NORM_KEEP];
 #pragma unroll
   for (int k = 0; k < NORM_KEEP; ++k) {
     int g = threadIdx.x + k * NORM_THREADS;
-    keep[k] = g < n_groups ? group_value(g) : make_float4(0.f, 0.f, 0.f, 0.f);
+    keep[k] = g < n_groups ? group_value(g, kb[k]) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) group_value(g);
+  for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) {
+    float b4[4];
+    load_w4<T>(bias, g * 4, H, vec, 0.f, b4);
+    group_value(g, b4);
+  }
   POSS_TRACE_POINT(2);
   for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -386,7 +403,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
 #pragma unroll
   for (int k = 0; k < NORM_KEEP; ++k) {
     int g = threadIdx.x + k * NORM_THREADS;
-    if (g < n_groups) group_store(g, keep[k], inv);
+    if (g < n_groups) group_store(g, keep[k], inv, kg[k]);
   }
   for (int g = threadIdx.x + NORM_KEEP * NORM_THREADS; g < n_groups; g += NORM_THREADS) {
     const int n = g * 4;                                    // wider rows: re-read this thread's own stores
@@ -395,7 +412,9 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     v.y = n + 1 < H ? h[(size_t)m * H + n + 1] : 0.f;
     v.z = n + 2 < H ? h[(size_t)m * H + n + 2] : 0.f;
     v.w = n + 3 < H ? h[(size_t)m * H + n + 3] : 0.f;
-    group_store(g, v, inv);
+    float g4[4];
+    load_w4<T>(gain, n, H, vec, 1.f, g4);
+    group_store(g, v, inv, g4);
   }
 }
 template <typename T>
@@ -450,30 +469,42 @@ template void launch_splitk_reduce<bf16>(Launcher&, const SplitKView&, int, int,
                                          int, bf16*);
 
 // ---- act = T(silu(gate) * up) from the parked partials of a SwiGLU product
+// One block per (tile of 64 ffn columns, 32 rows): 16 threads across the tile's columns (four each), two
+// rows per thread.  The tile, and with it the contributor list, is the same for the whole block.
 template <typename T>
-__global__ void __launch_bounds__(256) k_splitk_swiglu(SplitKView prod, int F, T* act) {
-  pdl_enter();
-  const int m = blockIdx.y;
-  const int f = (blockIdx.x * 256 + threadIdx.x) * 4;
-  if (f >= F) return;
-  int tile, t;
-  splitk_locate(prod, f, &tile, &t);
-  TileContrib tc = splitk_tile_contrib(prod, tile);
-  float4 g = splitk_load4(prod, m, f, tc, t);
-  float4 u = splitk_load4(prod, m, f, tc, t + 64);
-  float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+__global__ void __launch_bounds__(256) k_splitk_swiglu(SplitKView prod, int M, int F, T* act) {
+  pdl_begin();
+  const TileContrib tc = splitk_tile_contrib(prod, blockIdx.x);
+  const int cg = (threadIdx.x & 15) * 4;
+  const int f = blockIdx.x * 64 + cg;
+  const int m0 = blockIdx.y * 32 + (threadIdx.x >> 4), m1 = m0 + 16;
+  const int l0 = m0 < M ? m0 : M - 1, l1 = m1 < M ? m1 : M - 1;      // rows loaded (clamped), stored if < M
+  const int off[4] = {l0 * 128 + cg, l0 * 128 + cg + 64, l1 * 128 + cg, l1 * 128 + cg + 64};
+  const bool vec = (F & 3) == 0 && (reinterpret_cast<uintptr_t>(act) & 15) == 0;
+  pdl_sync();
+  if (f >= F || m0 >= M) return;
+  float4 x[4];
+  splitk_sum<4>(prod, tc, off, x);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    if (f + q < F) {
-      float sgl = gv[q] / (1.f + expf(-gv[q]));
-      act[(size_t)m * F + f + q] = from_f<T>(sgl * uv[q]);
+  for (int r = 0; r < 2; ++r) {
+    const int m = r ? m1 : m0;
+    if (m >= M) break;
+    const float gv[4] = {x[2 * r].x, x[2 * r].y, x[2 * r].z, x[2 * r].w};
+    const float uv[4] = {x[2 * r + 1].x, x[2 * r + 1].y, x[2 * r + 1].z, x[2 * r + 1].w};
+    float e[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) e[q] = silu_f(gv[q]) * uv[q];
+    if (vec) store4<T>(act + (size_t)m * F + f, e);
+    else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) if (f + q < F) act[(size_t)m * F + f + q] = from_f<T>(e[q]);
     }
   }
 }
 template <typename T>
 void launch_splitk_swiglu(Launcher& L, const SplitKView& prod, int rows, int F, T* act) {
   if (rows <= 0) return;
-  launch_pdl(L, k_splitk_swiglu<T>, dim3((F + 1023) / 1024, rows), dim3(256), 0, prod, F, act);
+  launch_pdl(L, k_splitk_swiglu<T>, dim3(prod.n_tiles, (rows + 31) / 32), dim3(256), 0, prod, rows, F, act);
 }
 template void launch_splitk_swiglu<float>(Launcher&, const SplitKView&, int, int, float*);
 template void launch_splitk_swiglu<bf16>(Launcher&, const SplitKView&, int, int, bf16*);
@@ -482,15 +513,55 @@ template void launch_splitk_swiglu<bf16>(Launcher&, const SplitKView&, int, int,
 // The product's row layout is [Hq*d q | Hkv*d k | Hkv*d v] fp32.  Rotate-half pairing (j, j + d/2).
 // The angle pos * theta^(-2j/d) is formed in double from a table of the d/2 inverse frequencies and
 // reduced to [-pi, pi] in double (2 pi split in two terms), so long positions lose nothing; sine and
-// cosine of the reduced angle are then taken in fp32.  One block per row; a work item is four
-// neighbouring pairs of one head (two 16-byte loads) or four values.
+// cosine of the reduced angle are then taken in fp32.
+// A block serves one row and ROPE_ITEMS work items (an item: four neighbouring pairs of one head, i.e. two
+// 16-byte groups of the product, or four values of v).  Its last two warps form the row's cos/sin table
+// while the item threads have their loads of the product in flight.  Item decoding and the contributors
+// of every tile need only the launch parameters and are done before the predecessor is awaited.
+#define ROPE_ITEMS 256
 template <typename T>
-__global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache, T* qout) {
+__global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache,
+                                                                  T* qout) {
   __shared__ TileContrib tab[512];
-  __shared__ float cs[64], sn[64];
-  pdl_enter();
+  __shared__ __align__(16) float cs[64], sn[64];
+  pdl_begin();
   fill_tile_table(qkv, tab);
   const int m = blockIdx.x;
+  const int half = a.d / 2;
+  const int qd = a.Hq * a.d, kd = a.Hkv * a.d, N = qd + 2 * kd;
+  const int q0 = a.rows - a.q_rows;
+  const bool with_q = m >= q0;
+  const int per_head = half / 4;                         // items per rotated head (d is a multiple of 8)
+  const int n_qitems = with_q ? a.Hq * per_head : 0;
+  const int n_kitems = a.Hkv * per_head;
+  const int n_items = n_qitems + n_kitems + kd / 4;
+  const bool item_thread = threadIdx.x < ROPE_ITEMS;
+  const int i = blockIdx.y * ROPE_ITEMS + threadIdx.x;
+  const bool active = item_thread && i < n_items;
+  // kind 0 = q, 1 = k (rotated), 2 = v; hh = head, j = first of the four elements inside the head
+  int kind = 2, hh = 0, j = 0, col = 0;
+  if (active) {
+    if (i < n_qitems + n_kitems) {
+      kind = i < n_qitems ? 0 : 1;
+      const int ii = kind == 0 ? i : i - n_qitems;
+      hh = ii / per_head;
+      j = (ii - hh * per_head) * 4;
+      col = (kind == 0 ? 0 : qd) + hh * a.d + j;
+    } else {
+      const int ii = (i - n_qitems - n_kitems) * 4;
+      hh = ii / a.d;
+      j = ii - hh * a.d;
+      col = qd + kd + ii;
+    }
+  }
+  int tile_lo = 0, t_lo = 0, tile_hi = 0, t_hi = 0;
+  if (active && qkv.deferred) {
+    splitk_locate(qkv, col, &tile_lo, &t_lo);
+    if (kind != 2) splitk_locate(qkv, col + half, &tile_hi, &t_hi);
+  }
+  const bool vec = aligned16(kcache) && aligned16(vcache) && (a.q_rows == 0 || aligned16(qout));
+  __syncthreads();
+  pdl_sync();
   int slot, pos;
   if (a.mode == 0) {
     RowInfo r = row_info(a.s, m);
@@ -500,77 +571,71 @@ __global__ void __launch_bounds__(512) k_rope_append(RopeArgs a, SplitKView qkv,
     slot = a.base + m;
     pos = a.base + a.depth[m];
   }
-  const int half = a.d / 2;
-  if ((int)threadIdx.x < half) {
-    const double two_pi_hi = 6.283185307179586, two_pi_lo = 2.4492935982947064e-16;
-    double x = (double)pos * a.inv_freq[threadIdx.x];
-    double k = rint(x * 0.15915494309189535);
-    double r = fma(-k, two_pi_hi, x);
-    r = fma(-k, two_pi_lo, r);
-    float s, c;
-    sincosf((float)r, &s, &c);
-    cs[threadIdx.x] = c;
-    sn[threadIdx.x] = s;
+  float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+  if (!item_thread) {
+    const int jj = threadIdx.x - ROPE_ITEMS;
+    if (jj < half) {
+      const double two_pi_hi = 6.283185307179586, two_pi_lo = 2.4492935982947064e-16;
+      double x = (double)pos * a.inv_freq[jj];
+      double k = rint(x * 0.15915494309189535);
+      double r = fma(-k, two_pi_hi, x);
+      r = fma(-k, two_pi_lo, r);
+      float sv, cv;
+      sincosf((float)r, &sv, &cv);
+      cs[jj] = cv;
+      sn[jj] = sv;
+    }
+  } else if (active) {
+    if (!qkv.deferred) {
+      lo = product4(qkv, tab, m, col, N);
+      if (kind != 2) hi = product4(qkv, tab, m, col + half, N);
+    } else if (kind == 2) {
+      lo = splitk_load4(qkv, m, col, tab[tile_lo], t_lo);
+    } else if (tile_lo == tile_hi) {
+      const int off[2] = {m * 128 + t_lo, m * 128 + t_hi};
+      float4 x[2];
+      splitk_sum<2>(qkv, tab[tile_lo], off, x);
+      lo = x[0];
+      hi = x[1];
+    } else {
+      lo = splitk_load4(qkv, m, col, tab[tile_lo], t_lo);
+      hi = splitk_load4(qkv, m, col + half, tab[tile_hi], t_hi);
+    }
   }
   __syncthreads();
   POSS_TRACE_POINT(1);
-  const int qd = a.Hq * a.d, kd = a.Hkv * a.d, N = qd + 2 * kd;
-  const int q0 = a.rows - a.q_rows;
-  const bool with_q = m >= q0;
-  const int per_head = half / 4;                         // items per rotated head (d is a multiple of 8)
-  const int n_qitems = with_q ? a.Hq * per_head : 0;
-  const int n_kitems = a.Hkv * per_head;
-  const int n_vitems = kd / 4;
-  const int n_items = n_qitems + n_kitems + n_vitems;
-  // two items per pass: all loads of the pass are issued before the first use
-  for (int i0 = threadIdx.x; i0 < n_items; i0 += 2 * blockDim.x) {
-    float4 lo[2], hi[2];
-    int col[2];
+  if (!active) return;
+  if (kind == 2) {
+    T* dst = vcache + ((size_t)hh * a.cap + slot) * a.d + j;
+    const float e[4] = {lo.x, lo.y, lo.z, lo.w};
+    if (vec) store4<T>(dst, e);
+    else { dst[0] = from_f<T>(e[0]); dst[1] = from_f<T>(e[1]); dst[2] = from_f<T>(e[2]); dst[3] = from_f<T>(e[3]); }
+    return;
+  }
+  const float x0[4] = {lo.x, lo.y, lo.z, lo.w}, x1[4] = {hi.x, hi.y, hi.z, hi.w};
+  float r0[4], r1[4];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * blockDim.x;
-      if (i >= n_items) continue;
-      if (i < n_qitems + n_kitems) {
-        const bool is_q = i < n_qitems;
-        const int ii = is_q ? i : i - n_qitems;
-        const int hh = ii / per_head, j = (ii % per_head) * 4;
-        col[u] = (is_q ? 0 : qd) + hh * a.d + j;
-        lo[u] = product4(qkv, tab, m, col[u], N);
-        hi[u] = product4(qkv, tab, m, col[u] + half, N);
-      } else {
-        col[u] = qd + kd + (i - n_qitems - n_kitems) * 4;
-        lo[u] = product4(qkv, tab, m, col[u], N);
-      }
-    }
+  for (int e = 0; e < 4; ++e) {
+    r0[e] = x0[e] * cs[j + e] - x1[e] * sn[j + e];
+    r1[e] = x1[e] * cs[j + e] + x0[e] * sn[j + e];
+  }
+  T* dst = kind == 0 ? qout + (size_t)(m - q0) * qd + hh * a.d : kcache + ((size_t)hh * a.cap + slot) * a.d;
+  if (vec) {
+    store4<T>(dst + j, r0);
+    store4<T>(dst + j + half, r1);
+  } else {
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * blockDim.x;
-      if (i >= n_items) continue;
-      if (i < n_qitems + n_kitems) {
-        const bool is_q = i < n_qitems;
-        const int ii = is_q ? i : i - n_qitems;
-        const int hh = ii / per_head, j = (ii % per_head) * 4;
-        float x0[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w}, x1[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
-        T* dst = is_q ? qout + (size_t)(m - q0) * qd + hh * a.d : kcache + ((size_t)hh * a.cap + slot) * a.d;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          dst[j + e] = from_f<T>(x0[e] * cs[j + e] - x1[e] * sn[j + e]);
-          dst[j + e + half] = from_f<T>(x1[e] * cs[j + e] + x0[e] * sn[j + e]);
-        }
-      } else {
-        const int ii = (i - n_qitems - n_kitems) * 4;
-        const int hh = ii / a.d, j = ii % a.d;
-        T* dst = vcache + ((size_t)hh * a.cap + slot) * a.d + j;
-        dst[0] = from_f<T>(lo[u].x); dst[1] = from_f<T>(lo[u].y); dst[2] = from_f<T>(lo[u].z); dst[3] = from_f<T>(lo[u].w);
-      }
-    }
+    for (int e = 0; e < 4; ++e) { dst[j + e] = from_f<T>(r0[e]); dst[j + e + half] = from_f<T>(r1[e]); }
   }
   POSS_TRACE_POINT(2);
 }
 template <typename T>
 void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {
   if (a.rows <= 0) return;
-  launch_pdl(L, k_rope_append<T>, dim3(a.rows), dim3(512), 0, a, qkv, kcache, vcache, qout);
+  const int per_head = a.d / 8;
+  const int n_items = (a.q_rows > 0 ? a.Hq * per_head : 0) + a.Hkv * per_head + a.Hkv * a.d / 4;
+  launch_pdl(L, k_rope_append<T>, dim3(a.rows, (n_items + ROPE_ITEMS - 1) / ROPE_ITEMS), dim3(ROPE_ITEMS + 64), 0, a, qkv,
+             kcache, vcache, qout);
 }
 template void launch_rope_append<float>(Launcher&, const RopeArgs&, const SplitKView&, float*, float*, float*);
 template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKView&, bf16*, bf16*, bf16*);

@@ -84,6 +84,10 @@ __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// The two halves, for kernels with work that needs nothing from a predecessor (index arithmetic on the
+// launch parameters, loads of weights): pdl_begin(), that work, pdl_sync(), then everything else.
+__device__ __forceinline__ void pdl_begin() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // hook for a timeline-recording build; empty in the library
 #ifndef POSS_TRACE_POINT
@@ -169,40 +173,61 @@ __device__ __forceinline__ TileContrib splitk_tile_contrib(const SplitKView& v, 
 // tile and row-in-tile of output column n (columns of the segments are laid side by side)
 __device__ __forceinline__ void splitk_locate(const SplitKView& v, int n, int* tile, int* t) {
   if (v.swiglu) { *tile = n >> 6; *t = n & 63; return; }     // gate row; the up row of the same column is t + 64
-  int base_tile = 0, nn = n;
-  for (int s = 0; s < v.n_segs - 1 && nn >= v.seg_rows[s]; ++s) { nn -= v.seg_rows[s]; base_tile += v.seg_tiles[s]; }
+  int base_tile = 0, nn = n;              // (at most three segments; constant indices keep the view in registers)
+  if (v.n_segs > 1 && nn >= v.seg_rows[0]) {
+    nn -= v.seg_rows[0]; base_tile += v.seg_tiles[0];
+    if (v.n_segs > 2 && nn >= v.seg_rows[1]) { nn -= v.seg_rows[1]; base_tile += v.seg_tiles[1]; }
+  }
   *tile = base_tile + nn / 128;
   *t = nn % 128;
 }
-// four consecutive columns n .. n+3 of row m (n a multiple of 4, so they share a tile), partials added in
-// range order
-__device__ __forceinline__ float4 splitk_load4(const SplitKView& v, int m, int n, const TileContrib& tc, int t) {
-  if (!v.deferred) return *reinterpret_cast<const float4*>(v.direct + (size_t)m * v.ld + n);
-  const size_t part = (size_t)v.Npad * 128;
-  const float* p0 = v.scratch + (size_t)m * 128 + t;
-  // all loads of a batch are issued before the first add (the adds stay in range order)
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int base = 0; base < tc.count; base += 8) {
-    float4 x[8];
+// Sum of one tile's partials, in range order, for NV 16-byte values that sit at the float offsets off[]
+// inside a partial (offset of element [m][t] = m * 128 + t).  The first contributor's loads and those of
+// the next three are in flight together; the adds stay in range order.
+template <int NV>
+__device__ __forceinline__ void splitk_sum(const SplitKView& v, const TileContrib& tc, const int (&off)[NV],
+                                           float4 (&acc)[NV]) {
+  const size_t part = (size_t)v.Npad * 128, step = (size_t)v.slots * part;
+  const float* p = v.scratch + ((size_t)tc.c_first * v.slots + tc.slot_first) * part;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int k = base + i;
-      if (k < tc.count) {
-        size_t slot = (size_t)(tc.c_first + k) * v.slots + (k == 0 ? tc.slot_first : 0);
-        x[i] = __ldcg(reinterpret_cast<const float4*>(p0 + slot * part));
-      }
+  for (int i = 0; i < NV; ++i) acc[i] = __ldcg(reinterpret_cast<const float4*>(p + off[i]));
+  p = v.scratch + (size_t)(tc.c_first + 1) * step;          // every later contributor parks in its slot 0
+  for (int k = 1; k < tc.count; k += 3, p += 3 * step) {
+    const int nb = tc.count - k;
+    float4 x0[NV], x1[NV], x2[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) x0[i] = __ldcg(reinterpret_cast<const float4*>(p + off[i]));
+    if (nb > 1) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) x1[i] = __ldcg(reinterpret_cast<const float4*>(p + step + off[i]));
+    }
+    if (nb > 2) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) x2[i] = __ldcg(reinterpret_cast<const float4*>(p + 2 * step + off[i]));
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int k = base + i;
-      if (k < tc.count) {
-        if (k == 0) acc = x[i];
-        else { acc.x += x[i].x; acc.y += x[i].y; acc.z += x[i].z; acc.w += x[i].w; }
-      }
+    for (int i = 0; i < NV; ++i) { acc[i].x += x0[i].x; acc[i].y += x0[i].y; acc[i].z += x0[i].z; acc[i].w += x0[i].w; }
+    if (nb > 1) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) { acc[i].x += x1[i].x; acc[i].y += x1[i].y; acc[i].z += x1[i].z; acc[i].w += x1[i].w; }
+    }
+    if (nb > 2) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) { acc[i].x += x2[i].x; acc[i].y += x2[i].y; acc[i].z += x2[i].z; acc[i].w += x2[i].w; }
     }
   }
-  return acc;
 }
+// four consecutive columns n .. n+3 of row m (n a multiple of 4, so they share a tile); t = n's row in the tile
+__device__ __forceinline__ float4 splitk_load4(const SplitKView& v, int m, int n, const TileContrib& tc, int t) {
+  if (!v.deferred) return *reinterpret_cast<const float4*>(v.direct + (size_t)m * v.ld + n);
+  const int off[1] = {m * 128 + t};
+  float4 acc[1];
+  splitk_sum<1>(v, tc, off, acc);
+  return acc[0];
+}
+// SiLU as every kernel of the library forms it (the in-kernel SwiGLU epilogue and the consumer kernels must
+// agree to the bit: which of them runs depends on the row count)
+__device__ __forceinline__ float silu_f(float g) { return g / (1.f + expf(-g)); }
 
 template <typename T>
 void launch_gemm_simt(Launcher& L, const T* X, int ldx, int M, const GemmSegs& segs, int K, const T* bias,
