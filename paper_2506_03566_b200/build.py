@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libposs.so")
-SOURCES = ["kernels_basic.cu", "kernels_attention.cu", "kernels_attention_mma.cu", "kernels_tree.cu", "gemm_tc.cu", "poss_api.cu", "no_alloc.cu"]
+SOURCES = ["kernels_basic.cu", "kernels_attention.cu", "kernels_attention_mma.cu", "kernels_tree.cu", "gemm_tc.cu", "attention_tc.cu", "poss_api.cu", "no_alloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

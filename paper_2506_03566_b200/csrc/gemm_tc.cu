@@ -34,6 +34,7 @@
 // Every wait on an mbarrier is bounded; on expiry the CTA raises POSS_E_TIMEOUT in the status word,
 // stops issuing work, drains its own copies (bounded), frees its TMEM and returns.
 #include "gemm_tc.cuh"
+#include "tc_ptx.cuh"
 #include <cuda.h>
 #include <unordered_map>
 #include <string>
@@ -49,12 +50,13 @@
 
 namespace {
 
+using namespace tcptx;
+
 constexpr int TILE_N = 128;          // weight rows per tile (UMMA M)
 constexpr int TILE_K = 64;           // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
 constexpr int MAX_STAGES = 12;
 constexpr int N_THREADS = 192;
-constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;     // one second: far beyond any launch of this library
 constexpr size_t SCRATCH_PARTIAL_BYTES = 96ull << 20;
 constexpr int N_COUNTERS = 8192;
 constexpr int XCH_STRIDE = 17;
@@ -79,131 +81,8 @@ struct TcArgs {
   float* pmax; float* psum; float* pval; int32_t* pidx;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: gives up after WAIT_LIMIT_NS of wall time (the clock is read every 64 polls, a poll may
-// itself suspend for a system-dependent while) or as soon as another role has raised the abort flag.
-// Returns false in both cases; on expiry it raises the flag itself.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  uint64_t t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
-      uint64_t now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) break;
-      if (it > 4096u) __nanosleep(64);
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t policy_evict_normal() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-      "[%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
-      : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
-  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
-      "[%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
 // barrier among the four epilogue warps only
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes (64 bf16), 128-byte swizzle,
-// 8-row groups 1024 bytes apart; descriptor version 1 (Blackwell), swizzle code 2 in bits 61..63.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
-  d |= (uint64_t)(1024u >> 4) << 32;             // stride between 8-row groups
-  d |= 1ull << 46;                               // descriptor version
-  d |= 2ull << 61;                               // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor of kind::f16: fp32 accumulate, bf16 x bf16, both operands K-major.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
 
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
@@ -222,7 +101,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   __shared__ uint32_t tmem_slot;
   __shared__ int s_abort, s_last, s_epi_ok;
 
-  pdl_launch_dependents();
+  pdl_begin();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -316,7 +195,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         load_w(cw, it);
         advance(cw);
       }
-      pdl_wait();
+      pdl_sync();
       for (int it = 0; it < pre; ++it) { if (!(a.inject_lost_load && it == 0)) load_x(cx, it); advance(cx); }
       int issued = pre, s = 0;
       uint32_t phase = 0;                     // parity of the "empty" completion that frees stage s next
@@ -370,7 +249,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     }
   } else {
     // ---------------- epilogue warps: TMEM lane = weight row
-    pdl_wait();
+    pdl_sync();
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int t = q * 32 + lane;                  // row inside the tile
     const int K = a.topk;
@@ -767,6 +646,18 @@ void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
 void tc_inject_lost_load(TcGemmPlanCache* c, int launches) { c->inject = launches < 0 ? 0 : launches; }
 size_t tc_gemm_scratch_bytes() { return SCRATCH_PARTIAL_BYTES + N_COUNTERS * sizeof(int); }
 
+void* tc_encode_fn(TcGemmPlanCache* c) {
+  if (!c->tried) {
+    c->tried = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  return reinterpret_cast<void*>(c->encode);
+}
+
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M) {
   if (M < 1 || M > 128 || K < 8 || (K % 8) || (ldx % 8)) return false;
   for (int i = 0; i < segs.n; ++i)
@@ -781,15 +672,7 @@ bool get_map(TcGemmPlanCache* c, const void* p, int rows, int cols, int ld, int 
   MapKey key{p, rows, cols, ld, box_rows};
   auto it = c->maps.find(key);
   if (it != c->maps.end()) { *out = it->second; return true; }
-  if (!c->tried) {
-    c->tried = true;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  }
-  if (!c->encode) return false;
+  if (!tc_encode_fn(c)) return false;
   cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
   cuuint32_t box[2] = {(cuuint32_t)TILE_K, (cuuint32_t)box_rows};

@@ -8,6 +8,16 @@ void tc_plan_cache_destroy(TcGemmPlanCache*);
 // test hook: the next `launches` launches withhold one activation tile, so one of their bounded waits runs out
 void tc_inject_lost_load(TcGemmPlanCache*, int launches);
 size_t tc_gemm_scratch_bytes();
+// the driver's tensor-map encoder (cuTensorMapEncodeTiled), resolved once; NULL when it cannot be had
+void* tc_encode_fn(TcGemmPlanCache*);
+
+// Tree attention on tcgen05 (bf16, head dimension 128, at most 2048 keys).  `part` holds one partial per
+// (row, head, 256 keys): rows * Hq * 8 * 132 floats at most, which the split-KV kernels' buffer always covers.
+// Returns false, having launched nothing, when the call is not covered; errors of a launch go to *status.
+bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out);
+bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
+                              const bf16* vc, float* part, bf16* out, int32_t* status);
+
 // true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 8, ...)
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);
 

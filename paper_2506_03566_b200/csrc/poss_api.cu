@@ -71,6 +71,7 @@ struct poss_ctx {
   int64_t launches;
   int last_depth, last_topk, last_nodes;
   TcGemmPlanCache* tc;
+  bool attn_tc;          // tree attention on the tcgen05 kernel where it covers the call
   int prof_mode;         // 0 off, 1 = LM-head launches of the draft steps, 2 = every stage kind of the draft steps
   int prof_n;
   int prof_kind[1024];   // kind of each bracketed launch
@@ -190,6 +191,9 @@ struct Impl {
   SplitKView gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo);
   // act[M][F] = T(silu(x . gate^T) * (x . up^T))
   void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
+  // tree-masked attention: the tcgen05 kernel where it covers the call (bf16, head dimension 128, at most
+  // 2048 keys), else the split-KV kernels with their partial buffer
+  void attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc, T* out);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
   bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists, bool argmax_only = false);
 
@@ -308,7 +312,7 @@ struct Impl {
       aa.mask = b.ts.node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
       int pr = prof_begin(POSS_PROF_ATTENTION);
-      run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
+      attention(aa, A(b.q), kc, vc, A(b.o));
       prof_end(pr);
       float* fo = b.fout + (size_t)i * KMAX * H;
       T* fbi = A(b.fb) + (size_t)i * KMAX * H;
@@ -342,7 +346,7 @@ struct Impl {
     aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = (rows + 63) / 64; aa.scale = scale;
     const T* kc = W(kv);
     const T* vc = kc + (size_t)g.n_kv_heads * kv_slots * g.head_dim;
-    run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, W(q), kc, vc, c->b.attn_part, A(out));
+    attention(aa, W(q), kc, vc, A(out));
     return L.err;
   }
 
@@ -372,7 +376,7 @@ struct Impl {
       aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.target_kv_slots;
       aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = mask_words;
       aa.scale = 1.0f / sqrtf((float)g.head_dim);
-      run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, A(b.q), kc, vc, b.attn_part, A(b.o));
+      attention(aa, A(b.q), kc, vc, A(b.o));
       // the layer's last reduction also applies the norm that follows it: the next layer's input
       // norm, or the final norm (whose output is the feature)
       const bool last = li == g.n_target_layers - 1;
@@ -456,6 +460,16 @@ void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const voi
 }
 
 template <typename T>
+void Impl<T>::attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc, T* out) {
+  run_tree_attention<T>(L, aa, ATTN_MAX_SPLITS, q, kc, vc, c->b.attn_part, out);
+}
+template <>
+void Impl<bf16>::attention(const AttnArgs& aa, const bf16* q, const bf16* kc, const bf16* vc, bf16* out) {
+  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, q, kc, vc, c->b.attn_part, out, c->b.status)) return;
+  run_tree_attention<bf16>(L, aa, ATTN_MAX_SPLITS, q, kc, vc, c->b.attn_part, out);
+}
+
+template <typename T>
 bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*, bool) { return false; }
 template <>
 bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists, bool argmax_only) {
@@ -520,6 +534,8 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   bp.base = reinterpret_cast<char*>(workspace);
   layout(*cfg, bp, c->b, &c->n_chunks, &c->n_cand_max);
   c->tc = tc_plan_cache_create();
+  c->attn_tc = true;
+  if (const char* e = getenv("POSS_ATTN_TC")) c->attn_tc = atoi(e) != 0;
   cudaStream_t st = S(stream);
   bool ok = cudaMemsetAsync(workspace, 0, bp.off, st) == cudaSuccess;
   double inv[64];
