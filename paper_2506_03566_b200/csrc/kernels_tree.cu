@@ -399,15 +399,14 @@ __global__ void __launch_bounds__(1024) k_topk_merge_expand(int rows, int K, int
         int bi = hi[0], bj = 0;
 #pragma unroll
         for (int j = 1; j < 6; ++j) if (better(hv[j], hi[j], bv, bi)) { bv = hv[j]; bi = hi[j]; bj = j; }
-        float wv = bv;
-        int wi = bi, wl = lane;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-          float ov = __shfl_xor_sync(0xffffffffu, wv, off);
-          int oi = __shfl_xor_sync(0xffffffffu, wi, off);
-          int ol = __shfl_xor_sync(0xffffffffu, wl, off);
-          if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
-        }
+        // the warp's best (largest value, then lowest id) with two integer reductions: the value as an
+        // order-preserving unsigned key, then the lowest id among the lanes that hold that value
+        const uint32_t bits = bv == 0.f ? 0u : __float_as_uint(bv);      // -0 and +0 are one value
+        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+        const uint32_t wkey = __reduce_max_sync(0xffffffffu, key);
+        const int wi = (int)__reduce_min_sync(0xffffffffu, key == wkey ? (uint32_t)bi : 0xffffffffu);
+        const int wl = __ffs(__ballot_sync(0xffffffffu, key == wkey && bi == wi)) - 1;
+        const float wv = __shfl_sync(0xffffffffu, bv, wl);
         if (lane == 0) {
           out_ids[(size_t)row * K + k] = wi;
           out_logp[(size_t)row * K + k] = wv - lse;
