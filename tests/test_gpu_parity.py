@@ -102,6 +102,48 @@ def test_tree_attention_matches_oracle(name, rows, P_len, Hq, Hkv, d):
     assert np.abs(got_c - want_c).max() <= tol
 
 
+@pytest.mark.parametrize("rows,P_len,Hq,Hkv", [
+    (1, 0, 8, 8), (16, 0, 8, 2), (5, 123, 8, 1), (5, 124, 8, 1), (61, 195, 16, 4), (61, 196, 16, 4),
+    (128, 128, 4, 1), (40, 1987, 8, 2), (61, 1987, 8, 8), (61, 1988, 8, 2),
+])
+def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv):
+    """Head dimension 128 (the tcgen05 kernel): key counts of 1 and 16, around the 128-key groups (128 / 129), the
+    256-key blocks of a CTA (256 / 257) and the 2048-key limit (2027, 2048; at 2049 the split-KV kernels take the
+    call); GQA groups of 1, 4 and 8; one and several query tiles; one and two mask words."""
+    d = 128
+    cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
+    P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
+    num = pu.oracle_num(cfg)
+    cap = P_len + rows + 5
+    q, kv = ps.make_attention_case(11, rows, Hq, Hkv, d, P_len, cap, cfg.dtype)
+    scale = 1.0 / math.sqrt(d)
+    for parents in (ps.random_tree_parents(12, rows), po.chain_parents(rows)):
+        mask = po.pack_mask(po.ancestor_matrix(parents))
+        got = pu.np_of(P.poss_tree_attention(dev(q), dev(kv), P_len, torch.from_numpy(mask.view(np.int64)).cuda(), scale))
+        assert P.poss_last_status() == 0
+        want = po.tree_attention(q, kv, P_len, parents, scale, num)
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= 2e-2
+
+
+def test_tree_root_row_equals_its_single_row_decode_bitwise():
+    """The property the lossless loop rests on: a token whose visible keys are the prefix and itself gets the same
+    attention output, bit for bit, as the root of a 61-row tree pass and as a single decoded row, also where the
+    two calls cut their keys into different numbers of blocks (prefix 1000: 1061 against 1001 keys)."""
+    Hq, Hkv, d, rows = 32, 8, 128, 61
+    cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
+    P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
+    scale = 1.0 / math.sqrt(d)
+    tree = po.pack_mask(po.ancestor_matrix(ps.random_tree_parents(13, rows)))
+    one = po.pack_mask(po.ancestor_matrix(po.chain_parents(1)))
+    for P_len in (0, 100, 250, 1000, 1023, 1980):
+        q, kv = ps.make_attention_case(14 + P_len, rows, Hq, Hkv, d, P_len, P_len + rows + 2, cfg.dtype)
+        full = pu.np_of(P.poss_tree_attention(dev(q), dev(kv), P_len, torch.from_numpy(tree.view(np.int64)).cuda(), scale))
+        single = pu.np_of(P.poss_tree_attention(dev(q[:1]), dev(kv), P_len, torch.from_numpy(one.view(np.int64)).cuda(), scale))
+        assert P.poss_last_status() == 0
+        assert np.array_equal(full[0], single[0]), f"root row differs at prefix {P_len}"
+
+
 @pytest.mark.parametrize("name,rows,K", [("t_fp32", 3, 3), ("t_fp32", 1, 16), ("t_bf16", 4, 4), ("m_bf16", 10, 10),
                                          ("m_bf16", 61, 1), ("t_bf16", 128, 16), ("m_bf16", 64, 3), ("m_bf16", 17, 16)])
 def test_lm_head_topk_matches_oracle(name, rows, K):
