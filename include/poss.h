@@ -232,11 +232,12 @@ POSS_API int poss_tree_attention_noalloc(const void* q, const void* kv, int kv_s
                                          int rows, int n_q_heads, int n_kv_heads, int head_dim, int dtype,
                                          const uint64_t* anc_mask, float scale, void* out, poss_stream stream);
 
-/* Failure-detection test hook (the paper has no counterpart).  The next `launches` tensor-core matrix-product
- * launches of this context withhold one activation tile from their own pipeline, so the bounded wait on that tile
- * runs out (after about one second): every CTA stops issuing work, waits (bounded) for its copies in flight,
- * frees its tensor memory and returns; the device status word becomes POSS_E_TIMEOUT (poss_last_status) and the
- * launch's results are undefined.  Nothing faults and the context stays usable: poss_reset clears the status. */
+/* Failure-detection test hook (the paper has no counterpart).  The next `launches` tensor-core launches of this
+ * context (matrix products and tcgen05 tree attention alike) withhold one tile from their own pipeline (a product:
+ * one activation tile; attention: the value tiles), so the bounded wait on that tile runs out (after about one
+ * second): every CTA stops issuing work, waits (bounded) for its copies in flight, frees its tensor memory and
+ * returns; the device status word becomes POSS_E_TIMEOUT (poss_last_status) and the launch's results are undefined.
+ * Nothing faults and the context stays usable: poss_reset clears the status. */
 POSS_API int poss_debug_lose_load(poss_ctx* ctx, int launches);
 
 /* Number of kernels this context has launched so far (host counter). */

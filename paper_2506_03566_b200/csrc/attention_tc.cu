@@ -56,6 +56,7 @@ struct AttnTcArgs {
   const uint64_t* mask;
   int mask_words;
   float scale_log2;                   // softmax scale times log2(e)
+  int inject_lost_load;               // test hook: the value tiles are never requested
   float* part;                        // [rows][Hq][n_splits][O_LD]: a CTA's merged partial, 128 outputs then (m, l)
   bf16* out;
   int32_t* status;
@@ -194,8 +195,10 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
       tma_load_3d(base + k_off, &map_k, bar_qk, 0, k_begin, kvh);
       tma_load_3d(base + k_off + k_half, &map_k, bar_qk, 64, k_begin, kvh);
       mbar_expect_tx(bar_v, 2u * k_half);
-      tma_load_3d(base + v_off, &map_v, bar_v, 0, k_begin, kvh);
-      tma_load_3d(base + v_off + k_half, &map_v, bar_v, 64, k_begin, kvh);
+      if (!a.inject_lost_load) {
+        tma_load_3d(base + v_off, &map_v, bar_v, 0, k_begin, kvh);
+        tma_load_3d(base + v_off + k_half, &map_v, bar_v, 64, k_begin, kvh);
+      }
       bool ok = mbar_wait(bar_qk, 0, abort_flag);
       if (ok) {
         tc_fence_after();
@@ -456,6 +459,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   k.mask = a.mask; k.mask_words = a.mask_words;
   k.scale_log2 = a.scale * 1.4426950408889634f;
   k.part = part; k.out = out; k.status = status;
+  k.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
   const uint32_t k_half = (uint32_t)k.cta_keys * 128u, p_bytes = 2u * (uint32_t)(k.cta_keys / 64) * HALF_TILE;
   uint32_t region_a = 2u * HALF_TILE + 2u * k_half;
   if (region_a < p_bytes) region_a = p_bytes;

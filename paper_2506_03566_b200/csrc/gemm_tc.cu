@@ -644,6 +644,11 @@ TcGemmPlanCache* tc_plan_cache_create() {
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
 void tc_inject_lost_load(TcGemmPlanCache* c, int launches) { c->inject = launches < 0 ? 0 : launches; }
+bool tc_take_injection(TcGemmPlanCache* c) {
+  if (c->inject <= 0) return false;
+  --c->inject;
+  return true;
+}
 size_t tc_gemm_scratch_bytes() { return SCRATCH_PARTIAL_BYTES + N_COUNTERS * sizeof(int); }
 
 void* tc_encode_fn(TcGemmPlanCache* c) {
@@ -774,8 +779,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (stages < 2) stages = 2;
   a.n_stages = stages;
   a.w_policy = cache->w_policy;
-  a.inject_lost_load = cache->inject > 0 ? 1 : 0;
-  if (cache->inject > 0) --cache->inject;
+  a.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);

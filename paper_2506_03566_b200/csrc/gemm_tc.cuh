@@ -5,8 +5,11 @@
 struct TcGemmPlanCache;
 TcGemmPlanCache* tc_plan_cache_create();
 void tc_plan_cache_destroy(TcGemmPlanCache*);
-// test hook: the next `launches` launches withhold one activation tile, so one of their bounded waits runs out
+// test hook: the next `launches` tensor-core launches (products or attention) withhold one tile of their own
+// pipeline, so one of their bounded waits runs out
 void tc_inject_lost_load(TcGemmPlanCache*, int launches);
+// consumes one pending injection (true when this launch has to withhold its tile)
+bool tc_take_injection(TcGemmPlanCache*);
 size_t tc_gemm_scratch_bytes();
 // the driver's tensor-map encoder (cuTensorMapEncodeTiled), resolved once; NULL when it cannot be had
 void* tc_encode_fn(TcGemmPlanCache*);

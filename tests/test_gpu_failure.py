@@ -37,3 +37,29 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     again = P.poss_linear(xd, Wd, impl=2).cpu().numpy()
     assert P.poss_last_status() == 0
     assert np.array_equal(again, good)
+
+
+def test_the_attention_kernel_reports_a_wait_that_runs_out_and_the_context_stays_usable():
+    """The tcgen05 tree attention: its value tiles are never requested, the wait for them runs out, every CTA of
+    every cluster still meets its peers at the cluster barrier and leaves in order."""
+    import math
+    from paper_2506_03566_b200 import Poss, make_config, to_device
+    Hq, Hkv, d, rows, P_len = 8, 2, 128, 20, 300
+    cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64,
+                                       n_target_layers=0)
+    P = Poss(make_config(cfg, 64), ps.make_weights(cfg, 1))
+    q, kv = ps.make_attention_case(21, rows, Hq, Hkv, d, P_len, P_len + rows + 2, cfg.dtype)
+    mask = torch.from_numpy(po.pack_mask(po.ancestor_matrix(ps.random_tree_parents(22, rows))).view(np.int64)).cuda()
+    qd, kvd, scale = to_device(q), to_device(kv), 1.0 / math.sqrt(d)
+    good = pu.np_of(P.poss_tree_attention(qd, kvd, P_len, mask, scale))
+    assert P.poss_last_status() == 0
+
+    P.poss_debug_lose_load(1)
+    P.poss_tree_attention(qd, kvd, P_len, mask, scale)      # results undefined; must neither fault nor hang
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 6                        # POSS_E_TIMEOUT
+
+    P.poss_reset()
+    again = pu.np_of(P.poss_tree_attention(qd, kvd, P_len, mask, scale))
+    assert P.poss_last_status() == 0
+    assert np.array_equal(again, good)
