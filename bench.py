@@ -151,6 +151,10 @@ def main():
                     help="profiler captures only: all specialists share one weight set, so the process holds "
                          "about 3 GB instead of 10 GB; the launch chain and every launch's traffic are unchanged "
                          "(one step still streams 1.56 GB, far more than L2)")
+    ap.add_argument("--target-layers", type=int,
+                    help="layers of the target pass (default 32, the workload; 0 with --alias-specialists).  Fewer "
+                         "layers keep a profiler capture of the target-pass kernels small: every layer launches the "
+                         "same kernels on the same shapes")
     args = ap.parse_args()
 
     import poss_synth as ps
@@ -182,8 +186,10 @@ def main():
 
     # ---------------- inputs: seeded, resident in HBM before timing
     seed = replica_seed(rank)
-    with_target = not (args.no_target or args.alias_specialists)
-    n_layers = 32 if with_target else 0
+    n_layers = args.target_layers if args.target_layers is not None else (0 if args.alias_specialists else 32)
+    with_target = not args.no_target and n_layers > 0
+    if not with_target:
+        n_layers = 0
     w = ps.make_weights(cfg, seed, alias_specialists=args.alias_specialists)
     rows = cfg.total + 1
     cap = cfg.prefix + 8 + cfg.tree_slots
@@ -343,7 +349,7 @@ def main():
                                    f"({'Llama-3-8B' if cfg.hidden == 4096 else 'Llama-2-13B' if cfg.hidden == 5120 else 'test'}-shaped), "
                                    f"{cfg.S} specialists x {cfg.n} positions, depth {cfg.depth}, top-k {cfg.topk}, "
                                    f"{cfg.total} tokens, prefix {cfg.prefix}; step = draft round + " +
-                                   ("61-row tree-masked pass of a 32-layer Llama-3-8B-shaped target + accept walk + KV compaction"
+                                   (f"61-row tree-masked pass of a {n_layers}-layer Llama-3-8B-shaped target + accept walk + KV compaction"
                                     if with_target else "61-row verification attention + logits argmax + accept walk"),
                        "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -362,7 +368,7 @@ def main():
                          "frac": achieved / hbm_peak if achieved else None,
                          # dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch, from the ncu capture
                          # summarised in profiles/k_gemm_tc_c2_m10_gateup_down_lmhead.md (c2 shapes only)
-                         "traffic": 1050894000 + 9812224 if cfg.name in ("c2", "c4", "c5") else None,
+                         "traffic": 1050836000 + 8128000 if cfg.name in ("c2", "c4", "c5") else None,
                          "launches_timed": n_lm, "avg_launch_us": lm_dur * 1e3,
                          "algorithmic_bytes_per_launch": lm_bytes},
         }
