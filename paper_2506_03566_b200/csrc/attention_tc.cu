@@ -39,12 +39,12 @@ using namespace tcptx;
 
 constexpr int D = 128;
 constexpr int QT = 128;               // query rows per CTA (UMMA M)
-constexpr int N_SOFTMAX = 256;        // eight warps: TMEM lane quarter x half of the keys
+constexpr int N_SOFTMAX = 256;        // eight warps: TMEM lane quarter x key group
 constexpr int N_THREADS = N_SOFTMAX + 32;
 constexpr int KG = 128;               // keys per group: the unit of the softmax partials, at absolute positions
 constexpr int MAX_CTA_KEYS = 2 * KG;  // keys per CTA (UMMA N of the first product)
 constexpr int MAX_SPLITS = 8;         // portable cluster size
-constexpr int O_LD = D + 4;            // floats per parked partial: 128 outputs, m, l, padding to 16 bytes
+constexpr int O_LD = D + 4;           // floats per parked partial: 128 outputs, m, l, padding to 16 bytes
 constexpr int HALF_TILE = QT * 128;   // bytes of a [128 rows][64 bf16] tile
 constexpr float NEG_BIG = -1.0e30f;
 
@@ -52,7 +52,7 @@ struct AttnTcArgs {
   int rows, Hq, G, n_q;               // n_q = rows * G query rows per KV head
   int n_all, n_tree, total;
   int cta_keys, n_splits;             // keys per CTA (128 or 256); CTAs per cluster
-  uint32_t region_a_bytes;            // Q + K, later P (hi, lo); V sits behind it; the parked O lies over both
+  uint32_t region_a_bytes;            // Q + K, later P (hi, lo); V sits behind it
   const uint64_t* mask;
   int mask_words;
   float scale_log2;                   // softmax scale times log2(e)
