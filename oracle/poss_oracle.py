@@ -543,6 +543,51 @@ def verify_accept(target_logits, target_features, tokens, parents):
     return path, a, bonus, np.array(new_tokens, dtype=np.int32), new_features
 
 
+def sample_walk(target_logits, tokens, parents, temperature, uniforms):
+    """Verification at a temperature > 0 (the second acceptance setting of Section 5; the rejection-sampling
+    phase of Section 2.1): the emitted tokens must be distributed as the target's own sampling.  The draft
+    tree proposes its candidates deterministically (top-k, no sampling in the drafter), i.e. each candidate is
+    a point mass q(x) = 1, for which rejection sampling reads: at the current node with target distribution
+    p = softmax(logits / temperature), test the node's children in node order; child x is accepted with
+    probability min(1, p(x) / q(x)) = p(x) (u < p(x) for the next uniform u); on rejection the residual
+    distribution norm(max(p - q, 0)) = p with p(x) removed and renormalised replaces p and the next child is
+    tested; when no child is left, the bonus token is drawn from the current p by inverse CDF (first index
+    whose cumulative probability exceeds u).  One uniform per tested child plus one for the bonus, consumed
+    in order.  Returns (path incl. root, n_accepted, bonus token, uniforms used)."""
+    z = np.asarray(target_logits, dtype=np.float64)
+    cur, path, k = 0, [0], 0
+    while True:
+        t = z[cur] / float(temperature)
+        p = np.exp(t - t.max())
+        p /= p.sum()
+        nxt = -1
+        for c in range(len(tokens)):
+            if parents[c] != cur:
+                continue
+            x = int(tokens[c])
+            u = float(uniforms[k])
+            k += 1
+            if u < p[x]:
+                nxt = c
+                break
+            p[x] = 0.0
+            total = p.sum()
+            if total <= 0.0:            # the children carried all of the mass: nothing is left to draw from
+                p[x] = 1.0
+                total = 1.0
+            p /= total
+        if nxt >= 0:
+            cur = nxt
+            path.append(cur)
+            continue
+        u = float(uniforms[k])
+        k += 1
+        cdf = np.cumsum(p)
+        bonus = int(np.searchsorted(cdf, u * cdf[-1], side="right"))
+        last = int(np.nonzero(p > 0)[0][-1])
+        return path, len(path) - 1, min(bonus, last), k
+
+
 @dataclass
 class Counters:
     """Per-position acceptance counters: N_i = rounds in which draft position i was accepted."""

@@ -449,6 +449,121 @@ def test_accept_walk_is_longest_path_matching_teacher_forced_greedy():
     assert [int(tree.tokens[j]) for j in path[1:]] == list(cont[:a]) and bonus == cont[a]
 
 
+# ----------------------------------------------------------------------------- verification at temperature > 0
+
+_SW_TOKENS = np.array([9, 2, 5, 0, 3, 1, 4], dtype=np.int32)       # node 0 is the root; siblings differ
+_SW_PARENTS = np.array([-1, 0, 0, 0, 1, 1, 2], dtype=np.int32)
+
+
+def _softmax(z, t):
+    e = np.exp(z / t - np.max(z / t))
+    return e / e.sum()
+
+
+def _sample_walk_statistics(walk, n_draws, temperature, seed):
+    """Empirical distribution of the first emitted token, and of the second one given the accepted child."""
+    g = np.random.default_rng(seed)
+    V = 7
+    logits = np.random.default_rng(3).standard_normal((7, V)) * 1.5
+    first = np.zeros(V)
+    second = {c: np.zeros(V) for c in (1, 2, 3)}
+    for _ in range(n_draws):
+        u = g.random(8)
+        path, a, bonus, used = walk(logits, _SW_TOKENS, _SW_PARENTS, temperature, u)
+        emitted = [int(_SW_TOKENS[j]) for j in path[1:]] + [bonus]
+        assert len(emitted) == a + 1 and 1 <= used <= 8
+        first[emitted[0]] += 1
+        if a >= 1:
+            second[path[1]][emitted[1]] += 1
+    return logits, first, second
+
+
+def _worst_sigma(counts, p):
+    """Largest deviation of a frequency from its probability in standard deviations (categories with an expected
+    count below 20 are left out: the normal approximation does not hold there)."""
+    n = counts.sum()
+    keep = n * p >= 20
+    return np.max(np.abs(counts[keep] / n - p[keep]) / np.sqrt(p[keep] * (1 - p[keep]) / n))
+
+
+def test_sample_walk_emits_the_target_distribution():
+    """Rejection sampling is lossless: the first emitted token is distributed as softmax(logits[root] / T) whether it
+    is an accepted draft token or the bonus, and after an accepted child c the next emitted token is distributed as
+    softmax(logits[c] / T).  60,000 draws; every frequency within 4.5 standard deviations."""
+    for temperature in (1.0, 0.7):
+        logits, first, second = _sample_walk_statistics(po.sample_walk, 60000, temperature, 11)
+        assert _worst_sigma(first, _softmax(logits[0], temperature)) < 4.5
+        for c, counts in second.items():
+            assert counts.sum() > 300
+            assert _worst_sigma(counts, _softmax(logits[c], temperature)) < 4.5
+
+
+def test_the_distribution_pin_catches_a_walk_without_renormalisation():
+    """The same statistic must reject a plausible mistake: testing the later siblings against the original
+    probabilities instead of the residual distribution."""
+    def wrong(target_logits, tokens, parents, temperature, uniforms):
+        z = np.asarray(target_logits, dtype=np.float64)
+        cur, path, k = 0, [0], 0
+        while True:
+            p = _softmax(z[cur], temperature)
+            nxt = -1
+            for c in range(len(tokens)):
+                if parents[c] != cur:
+                    continue
+                u = uniforms[k]; k += 1
+                if u < p[int(tokens[c])]:
+                    nxt = c
+                    break
+                p[int(tokens[c])] = 0.0                      # removed, but the rest is not rescaled
+            if nxt >= 0:
+                cur = nxt; path.append(cur)
+                continue
+            u = uniforms[k]; k += 1
+            cdf = np.cumsum(p)
+            return path, len(path) - 1, int(min(np.searchsorted(cdf, u * cdf[-1], side="right"), len(p) - 1)), k
+    logits, first, _ = _sample_walk_statistics(wrong, 60000, 1.0, 11)
+    assert _worst_sigma(first, _softmax(logits[0], 1.0)) > 8.0
+
+
+def test_sample_walk_extreme_uniforms_and_uniform_count():
+    logits = np.random.default_rng(5).standard_normal((7, 7))
+    # u = 0: every tested child is accepted (its probability is positive), the bonus is the first token with mass
+    path, a, bonus, used = po.sample_walk(logits, _SW_TOKENS, _SW_PARENTS, 1.0, np.zeros(8))
+    assert path == [0, 1, 4] and a == 2 and bonus == 0 and used == 3
+    # u just below 1: every child is rejected, the bonus is the last token that still has mass (6; 2, 5, 0 were removed)
+    path, a, bonus, used = po.sample_walk(logits, _SW_TOKENS, _SW_PARENTS, 1.0, np.full(8, 1.0 - 1e-12))
+    assert path == [0] and a == 0 and bonus == 6 and used == 4
+    # first child rejected, second accepted, its only child rejected: 2 + 1 + 1 uniforms
+    p0 = _softmax(logits[0], 1.0)
+    u = np.array([p0[2] + 1e-9, 0.0, 1.0 - 1e-12, 0.5, 0, 0, 0, 0])
+    path, a, bonus, used = po.sample_walk(logits, _SW_TOKENS, _SW_PARENTS, 1.0, u)
+    assert path == [0, 2] and a == 1 and used == 4
+    p2 = _softmax(logits[2], 1.0)
+    p2[4] = 0.0
+    assert bonus == int(np.searchsorted(np.cumsum(p2 / p2.sum()), 0.5, side="right"))
+
+
+def test_sample_walk_at_low_temperature_is_the_greedy_walk():
+    """As T -> 0 the target distribution is a point mass on its argmax: a child is accepted iff its token is the
+    greedy token, the bonus is the greedy token."""
+    parents = ps.random_tree_parents(31, 30)
+    g = np.random.default_rng(6)
+    tokens = np.zeros(30, dtype=np.int32)
+    for p in range(30):
+        kids = [c for c in range(30) if parents[c] == p]
+        tokens[kids] = g.permutation(50)[: len(kids)] + 100
+    anc = po.ancestor_matrix(parents)
+    for target_node in (0, 9, 29):
+        logits = g.standard_normal((30, 200))
+        path = [j for j in range(30) if anc[target_node, j]]
+        for a_, b_ in zip(path[:-1], path[1:]):
+            logits[a_, tokens[b_]] += 12.0
+        logits[target_node, 42] += 12.0
+        want = po.accept_walk(tokens, parents, po.argmax_rows(logits))
+        got = po.sample_walk(logits, tokens, parents, 0.02, g.uniform(0.001, 0.999, 31))
+        assert (got[0], got[1], got[2]) == want
+
+
 def test_pos_acc_identities():
     c = po.Counters(6)
     g = np.random.default_rng(5)
