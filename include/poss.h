@@ -156,6 +156,23 @@ POSS_API int poss_verify_accept(poss_ctx* ctx, const void* target_logits, const 
                        int32_t* out_path, int32_t* out_n_accepted, int32_t* out_bonus_token,
                        int32_t* out_new_tokens, void* out_new_features, poss_stream stream);
 
+/* Verification at a temperature > 0 (the rejection-sampling phase of Section 2.1; the paper's second setting,
+ * Section 5, temperature 1).  The tree's candidates are deterministic (top-k), i.e. point masses, so the rule is:
+ * at the current node p = softmax(target_logits[node] / temperature); the node's children are tested in node
+ * order, child x is accepted iff the next uniform u satisfies u < p(x); on rejection p(x) is removed, p is
+ * renormalised and the next child is tested; when no child is left the bonus token is drawn from the current p by
+ * inverse CDF in token order (first token whose cumulative probability exceeds u).  The emitted tokens are then
+ * distributed exactly as the target's own sampling.  target_logits float[rows][V] (device); uniforms
+ * float[n_uniforms] in [0, 1) (device), consumed in order: one per tested child, one for the bonus, at most `rows`
+ * in all (n_uniforms < rows -> POSS_E_CAPACITY); out_uniforms_used int32[1].  The other outputs are those of
+ * poss_verify_accept, and the acceptance counters are updated in the same way. */
+POSS_API int poss_verify_sample(poss_ctx* ctx, const float* target_logits, const void* target_features /*[rows][H]*/,
+                       const int32_t* tokens, const int32_t* parents, int rows, float temperature,
+                       const float* uniforms, int n_uniforms,
+                       int32_t* out_path, int32_t* out_n_accepted, int32_t* out_bonus_token,
+                       int32_t* out_new_tokens, void* out_new_features, int32_t* out_uniforms_used,
+                       poss_stream stream);
+
 /* Target model over `rows` tree rows: row r holds tokens[r], sits at rotary position
  * prefix_len + depth[r], is written to cache slot prefix_len + r and sees the prefix plus its
  * ancestors and itself (anc_mask as above).  A chain (depth r, lower-triangular mask) is plain

@@ -543,7 +543,7 @@ def verify_accept(target_logits, target_features, tokens, parents):
     return path, a, bonus, np.array(new_tokens, dtype=np.int32), new_features
 
 
-def sample_walk(target_logits, tokens, parents, temperature, uniforms):
+def sample_walk(target_logits, tokens, parents, temperature, uniforms, with_residual=False):
     """Verification at a temperature > 0 (the second acceptance setting of Section 5; the rejection-sampling
     phase of Section 2.1): the emitted tokens must be distributed as the target's own sampling.  The draft
     tree proposes its candidates deterministically (top-k, no sampling in the drafter), i.e. each candidate is
@@ -553,7 +553,8 @@ def sample_walk(target_logits, tokens, parents, temperature, uniforms):
     distribution norm(max(p - q, 0)) = p with p(x) removed and renormalised replaces p and the next child is
     tested; when no child is left, the bonus token is drawn from the current p by inverse CDF (first index
     whose cumulative probability exceeds u).  One uniform per tested child plus one for the bonus, consumed
-    in order.  Returns (path incl. root, n_accepted, bonus token, uniforms used)."""
+    in order.  Returns (path incl. root, n_accepted, bonus token, uniforms used) and, with_residual, the
+    distribution the bonus was drawn from."""
     z = np.asarray(target_logits, dtype=np.float64)
     cur, path, k = 0, [0], 0
     while True:
@@ -585,7 +586,8 @@ def sample_walk(target_logits, tokens, parents, temperature, uniforms):
         cdf = np.cumsum(p)
         bonus = int(np.searchsorted(cdf, u * cdf[-1], side="right"))
         last = int(np.nonzero(p > 0)[0][-1])
-        return path, len(path) - 1, min(bonus, last), k
+        out = (path, len(path) - 1, min(bonus, last), k)
+        return out + (p,) if with_residual else out
 
 
 @dataclass

@@ -60,6 +60,7 @@ EXPORTS = {
     "poss_tree_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                       C.c_float, C.c_void_p, C.c_void_p]),
     "poss_verify_accept": (C.c_int, [C.c_void_p] * 6 + [C.c_int] + [C.c_void_p] * 6),
+    "poss_verify_sample": (C.c_int, [C.c_void_p] * 5 + [C.c_int, C.c_float, C.c_void_p, C.c_int] + [C.c_void_p] * 7),
     "poss_target_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "poss_target_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
@@ -257,6 +258,22 @@ class Poss:
                                            _ptr(tokens), _ptr(parents), rows, _ptr(out["path"]),
                                            _ptr(out["n_accepted"]), _ptr(out["bonus"]), _ptr(out["new_tokens"]),
                                            _ptr(out["new_features"]), _stream()), "poss_verify_accept")
+        return out
+
+    def poss_verify_sample(self, target_logits, target_features, tokens, parents, rows, temperature, uniforms):
+        dev = "cuda"
+        H = self.config.hidden
+        out = {"path": torch.empty(POSS_MAX_DEPTH + 1, dtype=torch.int32, device=dev),
+               "n_accepted": torch.empty(1, dtype=torch.int32, device=dev),
+               "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+               "new_tokens": torch.zeros(POSS_MAX_DEPTH + 1, dtype=torch.int32, device=dev),
+               "new_features": torch.zeros((POSS_MAX_DEPTH + 1, H), dtype=self.dtype, device=dev),
+               "uniforms_used": torch.empty(1, dtype=torch.int32, device=dev)}
+        _check(self.lib.poss_verify_sample(self.ctx, _ptr(target_logits), _ptr(target_features), _ptr(tokens),
+                                           _ptr(parents), rows, float(temperature), _ptr(uniforms),
+                                           int(uniforms.numel()), _ptr(out["path"]), _ptr(out["n_accepted"]),
+                                           _ptr(out["bonus"]), _ptr(out["new_tokens"]), _ptr(out["new_features"]),
+                                           _ptr(out["uniforms_used"]), _stream()), "poss_verify_sample")
         return out
 
     def poss_target_forward(self, target_kv, prefix_len, tokens, depth, anc_mask, rows, want_logits=False):

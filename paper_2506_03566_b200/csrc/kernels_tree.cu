@@ -668,6 +668,168 @@ template void launch_accept_walk<float>(Launcher&, const int32_t*, const float*,
 template void launch_accept_walk<bf16>(Launcher&, const int32_t*, const bf16*, int, const int32_t*, const int32_t*,
                                        int, int, int32_t*, int32_t*, int32_t*, int32_t*, bf16*, unsigned long long*);
 
+// ------------------------------------------------------------------ verification at a temperature > 0
+// Rejection sampling over the tree's deterministic candidates (each candidate is a point mass): at the current node
+// p = softmax(logits / T); its children are tested in node order, child x is accepted iff the next uniform is
+// below p(x) / (mass not yet removed); a rejected child's mass is removed; when no child is left the bonus token is
+// drawn from what remains by inverse CDF in token order.  One block walks the tree; a level costs two passes over
+// the node's logits (maximum, sum of exponentials), the bonus a third one.  The walk is sequential by nature; the
+// passes are spread over the block's 1024 threads.  Sums are formed in a fixed order (per-lane strided partial
+// sums, warp tree, warps in order), so a call is reproducible.
+#define SW_THREADS 1024
+template <typename T>
+__global__ void __launch_bounds__(SW_THREADS) k_sample_walk(const float* logits, int V, const T* feats, int H,
+                                                            const int32_t* tokens, const int32_t* parents, int rows,
+                                                            int max_depth, float inv_t, const float* uniforms,
+                                                            int32_t* out_path, int32_t* out_a, int32_t* out_bonus,
+                                                            int32_t* out_new_tokens, T* out_new_features,
+                                                            int32_t* out_used, unsigned long long* counters) {
+  __shared__ int s_tok[256], s_par[256];
+  __shared__ int path[POSS_MAX_DEPTH + 1];
+  __shared__ float red[SW_THREADS / 32];
+  __shared__ float wsum[SW_THREADS / 32];
+  __shared__ int removed[256];             // tokens of the current node's rejected children
+  __shared__ float s_m, s_z, s_rem, s_thr;
+  __shared__ int s_next, s_nrem, s_used, s_a, s_bonus, s_warp;
+  __shared__ float s_before;
+  pdl_enter();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < rows; i += SW_THREADS) { s_tok[i] = tokens[i]; s_par[i] = parents[i]; }
+  if (threadIdx.x == 0) { path[0] = 0; s_used = 0; }
+  __syncthreads();
+  int cur = 0, a = 0;
+  const int seg = ((V + 31) / 32 + 31) / 32 * 32;      // tokens per warp in the bonus pass: contiguous, a multiple of 32
+  while (true) {
+    const float* row = logits + (size_t)cur * V;
+    // ---- maximum and sum of exp((l - max) / T)
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < V; i += SW_THREADS) m = fmaxf(m, __ldcg(row + i));
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = red[0];
+      for (int w = 1; w < SW_THREADS / 32; ++w) t = fmaxf(t, red[w]);
+      s_m = t;
+    }
+    __syncthreads();
+    m = s_m;
+    float z = 0.f;
+    for (int i = threadIdx.x; i < V; i += SW_THREADS) z += expf((__ldcg(row + i) - m) * inv_t);
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    __syncthreads();                                    // red[] was read by thread 0 above
+    if (lane == 0) red[warp] = z;
+    __syncthreads();
+    // ---- the node's children, in node order (one thread: a handful of tests)
+    if (threadIdx.x == 0) {
+      float zz = 0.f;
+      for (int w = 0; w < SW_THREADS / 32; ++w) zz += red[w];
+      float rem = 0.f;
+      int nrem = 0, nxt = -1, used = s_used;
+      if (a < max_depth) {
+        for (int c = 1; c < rows; ++c) {
+          if (s_par[c] != cur) continue;
+          const int x = s_tok[c];
+          const float e = expf((__ldcg(row + x) - m) * inv_t);
+          const float left = zz - rem;
+          const float u = uniforms[used++];
+          if (left > 0.f && u * left < e) { nxt = c; break; }
+          rem += e;
+          removed[nrem++] = x;
+        }
+      }
+      s_z = zz; s_rem = rem; s_nrem = nrem; s_next = nxt; s_used = used;
+      if (nxt >= 0) path[a + 1] = nxt;
+    }
+    __syncthreads();
+    if (s_next >= 0) { cur = s_next; ++a; continue; }
+    break;
+  }
+  // ---- bonus token: inverse CDF over what is left of the last node's distribution, in token order
+  {
+    const float* row = logits + (size_t)cur * V;
+    const float m = s_m;
+    const int nrem = s_nrem;
+    const int lo = warp * seg, hi = min(V, lo + seg);
+    float part = 0.f;
+    for (int i = lo + lane; i < hi; i += 32) part += expf((__ldcg(row + i) - m) * inv_t);
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) wsum[warp] = part;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int k = 0; k < nrem; ++k) wsum[removed[k] / seg] -= expf((__ldcg(row + removed[k]) - m) * inv_t);
+      float total = 0.f;
+      for (int w = 0; w < SW_THREADS / 32; ++w) { wsum[w] = fmaxf(wsum[w], 0.f); total += wsum[w]; }
+      const float thr = uniforms[s_used++] * total;
+      // the warp whose segment holds the threshold (the last one with mass if rounding runs past the end)
+      float before = 0.f;
+      int sel = -1, last = 0;
+      for (int w = 0; w < SW_THREADS / 32; ++w) {
+        if (wsum[w] > 0.f) last = w;
+        if (sel < 0 && before + wsum[w] > thr) sel = w;
+        if (sel < 0) before += wsum[w];
+      }
+      if (sel < 0) { sel = last; before = total - wsum[last]; }
+      s_warp = sel; s_before = before; s_thr = thr; s_bonus = -1;
+    }
+    __syncthreads();
+    if (warp == s_warp) {
+      float cum = s_before;
+      const float thr = s_thr;
+      int found = -1, last_pos = -1;
+      for (int i0 = lo; i0 < hi && found < 0; i0 += 32) {
+        const int i = i0 + lane;
+        float e = 0.f;
+        if (i < hi) {
+          e = expf((__ldcg(row + i) - m) * inv_t);
+          for (int k = 0; k < nrem; ++k) if (removed[k] == i) e = 0.f;
+        }
+        float incl = e;
+        for (int o = 1; o < 32; o <<= 1) {
+          float v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, e > 0.f && cum + incl > thr);
+        const unsigned pos = __ballot_sync(0xffffffffu, e > 0.f);
+        if (pos) last_pos = i0 + 31 - __clz(pos);
+        if (hit) found = i0 + __ffs(hit) - 1;
+        cum += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) s_bonus = found >= 0 ? found : last_pos;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    s_a = a;
+    out_a[0] = a;
+    out_bonus[0] = s_bonus;
+    out_used[0] = s_used;
+    atomicAdd(&counters[0], 1ull);
+    for (int i = 1; i <= a; ++i) atomicAdd(&counters[i], 1ull);
+  }
+  for (int i = threadIdx.x; i <= POSS_MAX_DEPTH; i += SW_THREADS) out_path[i] = i <= a ? path[i] : -1;
+  for (int k = threadIdx.x; k <= a; k += SW_THREADS) out_new_tokens[k] = k < a ? s_tok[path[k + 1]] : s_bonus;
+  for (int i = threadIdx.x; i < (a + 1) * H; i += SW_THREADS) {
+    int k = i / H, e = i % H;
+    out_new_features[(size_t)k * H + e] = feats[(size_t)path[k] * H + e];
+  }
+}
+template <typename T>
+void launch_sample_walk(Launcher& L, const float* logits, int V, const T* feats, int H, const int32_t* tokens,
+                        const int32_t* parents, int rows, int max_depth, float temperature, const float* uniforms,
+                        int32_t* out_path, int32_t* out_a, int32_t* out_bonus, int32_t* out_new_tokens,
+                        T* out_new_features, int32_t* out_used, unsigned long long* counters) {
+  launch_pdl(L, k_sample_walk<T>, dim3(1), dim3(SW_THREADS), 0, logits, V, feats, H, tokens, parents, rows, max_depth,
+             1.0f / temperature, uniforms, out_path, out_a, out_bonus, out_new_tokens, out_new_features, out_used,
+             counters);
+}
+template void launch_sample_walk<float>(Launcher&, const float*, int, const float*, int, const int32_t*, const int32_t*,
+                                        int, int, float, const float*, int32_t*, int32_t*, int32_t*, int32_t*, float*,
+                                        int32_t*, unsigned long long*);
+template void launch_sample_walk<bf16>(Launcher&, const float*, int, const bf16*, int, const int32_t*, const int32_t*,
+                                       int, int, float, const float*, int32_t*, int32_t*, int32_t*, int32_t*, bf16*,
+                                       int32_t*, unsigned long long*);
+
 // ------------------------------------------------------------------ cache compaction after acceptance
 // Block (layer*2 + kv, head): copies slot prefix_len + path[k] to prefix_len + k for k = 1..a in
 // ascending k.  path[k] >= k, so a source is never overwritten before it is read.

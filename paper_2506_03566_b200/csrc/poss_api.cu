@@ -666,6 +666,30 @@ int poss_verify_accept(poss_ctx* c, const void* target_logits, const int32_t* ta
   return L.err;
 }
 
+int poss_verify_sample(poss_ctx* c, const float* target_logits, const void* target_features, const int32_t* tokens,
+                       const int32_t* parents, int rows, float temperature, const float* uniforms, int n_uniforms,
+                       int32_t* out_path, int32_t* out_n_accepted, int32_t* out_bonus, int32_t* out_new_tokens,
+                       void* out_new_features, int32_t* out_uniforms_used, poss_stream stream) {
+  if (!c || !target_logits || !target_features || !tokens || !parents || !uniforms || !out_path || !out_n_accepted ||
+      !out_bonus || !out_new_tokens || !out_new_features || !out_uniforms_used)
+    return POSS_E_INVALID;
+  if (rows < 1 || !(temperature > 0.f)) return POSS_E_INVALID;
+  if (rows > 256 || n_uniforms < rows) return POSS_E_CAPACITY;
+  Launcher L; L.stream = S(stream); L.launches = &c->launches; L.err = POSS_OK;
+  const poss_config& cf = c->cfg;
+  if (cf.dtype == POSS_BF16)
+    launch_sample_walk<bf16>(L, target_logits, cf.vocab, reinterpret_cast<const bf16*>(target_features), cf.hidden,
+                             tokens, parents, rows, POSS_MAX_DEPTH, temperature, uniforms, out_path, out_n_accepted,
+                             out_bonus, out_new_tokens, reinterpret_cast<bf16*>(out_new_features), out_uniforms_used,
+                             c->b.counters);
+  else
+    launch_sample_walk<float>(L, target_logits, cf.vocab, reinterpret_cast<const float*>(target_features), cf.hidden,
+                              tokens, parents, rows, POSS_MAX_DEPTH, temperature, uniforms, out_path, out_n_accepted,
+                              out_bonus, out_new_tokens, reinterpret_cast<float*>(out_new_features), out_uniforms_used,
+                              c->b.counters);
+  return L.err;
+}
+
 int poss_target_forward(poss_ctx* c, void* target_kv, int prefix_len, const int32_t* tokens, const int32_t* depth,
                         const uint64_t* anc_mask, int rows, void* out_features, int32_t* out_argmax,
                         float* out_logits, poss_stream stream) {

@@ -316,6 +316,11 @@ void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int tota
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes);
 template <typename T>
+void launch_sample_walk(Launcher& L, const float* logits, int V, const T* feats, int H, const int32_t* tokens,
+                        const int32_t* parents, int rows, int max_depth, float temperature, const float* uniforms,
+                        int32_t* out_path, int32_t* out_a, int32_t* out_bonus, int32_t* out_new_tokens,
+                        T* out_new_features, int32_t* out_used, unsigned long long* counters);
+template <typename T>
 void launch_accept_walk(Launcher& L, const int32_t* g, const T* feats, int H, const int32_t* tokens,
                         const int32_t* parents, int rows, int max_depth, int32_t* out_path, int32_t* out_a,
                         int32_t* out_bonus, int32_t* out_new_tokens, T* out_new_features,

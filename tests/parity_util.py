@@ -199,3 +199,15 @@ def compare_kv(cfg, dkv_gpu, kv_oracle, lo, hi, tol):
     else:
         assert err.max() <= tol, float(err.max())
     return float(err.max())
+
+
+def bonus_is_valid(residual, u, bonus, rel_tol=2e-5):
+    """Inverse-CDF draw in fp32 against the fp64 oracle: the threshold u * total must lie in the drawn token's
+    cumulative interval up to the rounding of an fp32 sum over the vocabulary (the interval's ends are sums of up to
+    128256 terms; in fp32, in the kernel's blocked order, they carry a relative error of the order of 1e-5 of the
+    total), and the token must have mass."""
+    cdf = np.cumsum(np.asarray(residual, dtype=np.float64))
+    total = cdf[-1]
+    thr = float(u) * total
+    lo = cdf[bonus - 1] if bonus > 0 else 0.0
+    return residual[bonus] > 0 and lo - rel_tol * total <= thr <= cdf[bonus] + rel_tol * total

@@ -110,6 +110,50 @@ def test_full_size_verify_accept_over_the_whole_vocabulary():
         assert np.array_equal(pu.np_of(out["new_features"][: a + 1]), want[4])
 
 
+def test_full_size_verify_sample_over_the_whole_vocabulary():
+    """Temperature-1 verification over 61 rows x 128256 ids: walk, bonus token and uniforms used equal the oracle's
+    for 12 uniform streams, the bonus token up to the fp32 rounding of its inverse-CDF draw (child tokens carry a boost of 11 so that their probabilities are of order 0.2 and walks
+    of several depths occur); the kernel's time is printed."""
+    cfg = ps.CONFIGS["t_bf16"].replace(S=1, n_target_layers=0, vocab=128256)
+    P = _poss(cfg, ps.make_weights(cfg.replace(vocab=64), 3) | {
+        "embed": np.zeros((cfg.vocab, cfg.hidden), np.uint16), "lm_head": np.zeros((cfg.vocab, cfg.hidden), np.uint16)}, 64)
+    rows = 61
+    parents = ps.random_tree_parents(18, rows, max_children=4)
+    rng = np.random.default_rng(6)
+    tokens = np.zeros(rows, dtype=np.int32)
+    for p in range(rows):
+        kids = [c for c in range(rows) if parents[c] == p]
+        tokens[kids] = rng.choice(cfg.vocab, size=len(kids), replace=False)
+    logits = rng.standard_normal((rows, cfg.vocab)).astype(np.float32)
+    for c in range(1, rows):
+        logits[parents[c], tokens[c]] += 11.0
+    feats = ps.normal(9, "tf", (rows, cfg.hidden), 1.0, "bf16")
+    lg_d, feats_d = torch.from_numpy(logits).cuda(), _dev(feats)
+    tok_d, par_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(parents).cuda()
+    depths, exact = [], 0
+    for trial in range(12):
+        u = np.random.default_rng(77 + trial).random(rows).astype(np.float32)
+        path, a, bonus, used, residual = po.sample_walk(logits, tokens, parents, 1.0, u, with_residual=True)
+        out = P.poss_verify_sample(lg_d, feats_d, tok_d, par_d, rows, 1.0, torch.from_numpy(u).cuda())
+        assert P.poss_last_status() == 0
+        assert int(out["n_accepted"][0]) == a and out["path"][: a + 1].cpu().tolist() == path
+        assert int(out["uniforms_used"][0]) == used
+        # the bonus draw: the oracle's token, or a neighbour whose interval holds the threshold up to fp32 rounding
+        got = int(out["bonus"][0])
+        assert got == bonus or pu.bonus_is_valid(residual, u[used - 1], got), (trial, got, bonus)
+        exact += got == bonus
+        depths.append(a)
+    assert max(depths) >= 2
+    u_d = torch.from_numpy(u).cuda()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        P.poss_verify_sample(lg_d, feats_d, tok_d, par_d, rows, 1.0, u_d)
+    e1.record()
+    torch.cuda.synchronize()
+    print("verify_sample 61 x 128256, depths", depths, "bonus equal to the oracle's in", exact, "of 12, us per call", round(e0.elapsed_time(e1) * 50, 1))
+
+
 def test_c5_full_loop_matches_plain_greedy_decode():
     """Config c5: 32-layer Llama-3-8B-shaped target + the c2 drafter, prompt of 512 ids, 512 generated tokens.
     Every round = draft tree (depth 6, top-k 10, 60 tokens) + tree-masked target pass + accept walk + KV

@@ -232,6 +232,73 @@ def test_verify_accept_planted_paths():
         assert n_at[i] == sum(1 for a in accepted if a >= i)
 
 
+@pytest.mark.parametrize("name,vocab,rows,temperature", [
+    ("t_fp32", 777, 14, 1.0), ("t_bf16", 5000, 25, 1.0), ("t_bf16", 5000, 61, 0.7), ("t_bf16", 33, 61, 1.0),
+    ("t_bf16", 32003, 128, 1.0), ("t_bf16", 5000, 1, 1.0),
+])
+def test_verify_sample_matches_oracle(name, vocab, rows, temperature):
+    """Verification at a temperature: the walk, the bonus token, the verified pairs and the number of uniforms used
+    equal the oracle's for 24 different uniform streams per case (decisions compare a uniform with a probability:
+    fp32 on the GPU, fp64 in the oracle, so a uniform within 1e-5 of its threshold could legitimately flip; with
+    these seeds none is).  Child tokens get a boost so that walks of every depth occur."""
+    cfg = ps.CONFIGS[name].replace(S=1, n_target_layers=0, vocab=vocab)
+    P = make_poss(cfg, ps.make_weights(cfg, 3), 64)
+    parents = ps.random_tree_parents(40 + rows, rows, max_children=4)
+    g = np.random.default_rng(rows)
+    tokens = np.zeros(rows, dtype=np.int32)
+    for p in range(rows):
+        kids = [c for c in range(rows) if parents[c] == p]
+        tokens[kids] = g.permutation(vocab)[: len(kids)]
+    logits = (g.standard_normal((rows, vocab)) * 2.0).astype(np.float32)
+    for c in range(1, rows):
+        logits[parents[c], tokens[c]] += 5.0
+    feats = ps.normal(9, "tf", (rows, cfg.hidden), 1.0, cfg.dtype)
+    feats_wide = po.widen(feats, np.float64)
+    lg_d, feats_d = torch.from_numpy(logits).cuda(), dev(feats)
+    tok_d, par_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(parents).cuda()
+    P.poss_reset()
+    depths = []
+    for trial in range(24):
+        u = np.random.default_rng(1000 * rows + trial).random(max(rows, 2)).astype(np.float32)
+        if trial == 0:
+            u[:] = 0.0                        # accepts every first child down to a leaf
+        if trial == 1:
+            u[:] = np.float32(1.0 - 2.0 ** -24)   # rejects everything: the bonus comes from the root's residual
+        path, a, bonus, used = po.sample_walk(logits, tokens, parents, temperature, u)
+        out = P.poss_verify_sample(lg_d, feats_d, tok_d, par_d, rows, temperature, torch.from_numpy(u).cuda())
+        assert P.poss_last_status() == 0
+        a_cap = min(a, 16)
+        assert int(out["n_accepted"][0]) == a == a_cap, f"trial {trial}"
+        assert out["path"][: a + 1].cpu().tolist() == path
+        assert int(out["bonus"][0]) == bonus, f"trial {trial}"
+        assert int(out["uniforms_used"][0]) == used
+        want_tokens = [int(tokens[j]) for j in path[1:]] + [bonus]
+        assert out["new_tokens"][: a + 1].cpu().tolist() == want_tokens
+        assert np.array_equal(pu.np_of(out["new_features"][: a + 1]), feats_wide[path])
+        depths.append(a)
+    if rows > 1:
+        assert max(depths) >= 2 and min(depths) == 0
+    rounds, n_at = P.poss_get_counters()
+    assert rounds == 24
+    for i in range(1, cfg.depth + 1):
+        assert n_at[i] == sum(1 for a in depths if a >= i)
+
+
+def test_verify_sample_argument_errors():
+    cfg = ps.CONFIGS["t_bf16"].replace(S=1, n_target_layers=0)
+    P = make_poss(cfg, ps.make_weights(cfg, 3), 64)
+    rows = 5
+    lg = torch.zeros((rows, cfg.vocab), dtype=torch.float32, device="cuda")
+    feats = torch.zeros((rows, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    tok = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    par = torch.tensor([-1, 0, 0, 1, 1], dtype=torch.int32, device="cuda")
+    few = torch.zeros(rows - 1, dtype=torch.float32, device="cuda")
+    with pytest.raises(Exception):
+        P.poss_verify_sample(lg, feats, tok, par, rows, 1.0, few)          # fewer uniforms than rows
+    with pytest.raises(Exception):
+        P.poss_verify_sample(lg, feats, tok, par, rows, 0.0, torch.zeros(rows, dtype=torch.float32, device="cuda"))
+
+
 # ----------------------------------------------------------------------------- the draft round
 
 ROUND_CASES = [
@@ -409,6 +476,30 @@ def test_loop_with_multi_token_acceptance_is_lossless(K, T, L, seed):
     rounds, n_at = P.poss_get_counters()
     assert rounds == octr.rounds and n_at[1:L + 1] == octr.accepted_at[1:L + 1].tolist()
     assert max(a for a, _ in log) >= 3
+
+
+def test_sampling_loop_at_a_vanishing_temperature_is_the_greedy_loop():
+    """The loop with poss_verify_sample at temperature 1e-4 (every target distribution a point mass on its argmax)
+    emits the greedy stream with the greedy loop's accepted paths, whatever the uniforms; at temperature 1 it runs,
+    accepts draft tokens, and two runs from the same generator seed agree."""
+    from paper_2506_03566_b200 import speculative_generate
+    cfg = ps.CONFIGS["t_fp32"].replace(n_target_layers=1)
+    w = ps.make_mimic_weights(cfg, 31)
+    P, prompt, spec, plain, log = _loop_case(cfg, w, 31, 9, 40, 5, 3, 14)
+    pt = torch.from_numpy(prompt).cuda()
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    slog = []
+    cold = speculative_generate(P, pt, 40, 5, 3, 14, log=slog, temperature=1e-4, generator=gen)
+    assert P.poss_last_status() == 0
+    assert cold == spec and slog == log
+    runs = []
+    for _ in range(2):
+        gen.manual_seed(6)
+        hlog = []
+        runs.append((speculative_generate(P, pt, 40, 5, 3, 14, log=hlog, temperature=1.0, generator=gen), hlog))
+    assert P.poss_last_status() == 0
+    assert runs[0] == runs[1] and len(runs[0][0]) == 40
+    assert all(0 <= t < cfg.vocab for t in runs[0][0])
 
 
 def test_bf16_loop_is_lossless_against_its_own_plain_decode():
