@@ -104,12 +104,12 @@ def test_tree_attention_matches_oracle(name, rows, P_len, Hq, Hkv, d):
 
 @pytest.mark.parametrize("rows,P_len,Hq,Hkv", [
     (1, 0, 8, 8), (16, 0, 8, 2), (5, 123, 8, 1), (5, 124, 8, 1), (61, 195, 16, 4), (61, 196, 16, 4),
-    (128, 128, 4, 1), (40, 1987, 8, 2), (61, 1987, 8, 8), (61, 1988, 8, 2),
+    (128, 128, 4, 1), (128, 64, 8, 1), (40, 1987, 8, 2), (61, 1987, 8, 8), (61, 1988, 8, 2),
 ])
 def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv):
     """Head dimension 128 (the tcgen05 kernel): key counts of 1 and 16, around the 128-key groups (128 / 129), the
     256-key blocks of a CTA (256 / 257) and the 2048-key limit (2027, 2048; at 2049 the split-KV kernels take the
-    call); GQA groups of 1, 4 and 8; one and several query tiles; one and two mask words."""
+    call); GQA groups of 1, 4 and 8; one to eight query tiles; one and two mask words."""
     d = 128
     cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
     P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
