@@ -72,6 +72,7 @@ struct poss_ctx {
   int last_depth, last_topk, last_nodes;
   TcGemmPlanCache* tc;
   bool attn_tc;          // tree attention on the tcgen05 kernel where it covers the call
+  bool swiglu_in_kernel; // gate/up product finished by the GEMM's own SwiGLU epilogue instead of the consumer kernel
   int prof_mode;         // 0 off, 1 = LM-head launches of the draft steps, 2 = every stage kind of the draft steps
   int prof_n;
   int prof_kind[1024];   // kind of each bracketed launch
@@ -447,10 +448,12 @@ void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const voi
   if (tc_gemm_supported(sg, K, K, M)) {
     TcEpilogue ep;
     ep.mode = TC_EPI_SWIGLU; ep.out_bf = act; ep.ldo_bf = F;
-    // few rows: the last CTA of each tile finishes it in the kernel; many rows (the target pass): that
-    // tail grows with the row count, so the partials are left to a consumer kernel spread over all SMs
+    // The tile segments are left as partials and a consumer kernel spread over all SMs finishes them: the
+    // in-kernel finish by the last CTA of each tile is a tail that grows with the row count and, measured, loses
+    // even at 10 rows (48.0 vs 46.1 us for the product, 10 us per draft round).  The kernel's own SwiGLU epilogue
+    // remains for products whose partials do not fit the scratch.
     SplitKView v;
-    if (M > 16 && F % 4 == 0) ep.view = &v;
+    if (F % 4 == 0 && !c->swiglu_in_kernel) ep.view = &v;
     launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
     if (ep.view && v.deferred) launch_splitk_swiglu<bf16>(L, v, M, F, act);
     return;
@@ -536,6 +539,8 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   c->tc = tc_plan_cache_create();
   c->attn_tc = true;
   if (const char* e = getenv("POSS_ATTN_TC")) c->attn_tc = atoi(e) != 0;
+  c->swiglu_in_kernel = false;
+  if (const char* e = getenv("POSS_SWIGLU_IN_KERNEL")) c->swiglu_in_kernel = atoi(e) != 0;
   cudaStream_t st = S(stream);
   bool ok = cudaMemsetAsync(workspace, 0, bp.off, st) == cudaSuccess;
   double inv[64];

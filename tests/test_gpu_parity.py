@@ -352,6 +352,31 @@ def test_draft_round_matches_oracle(name, over, n_new, seed, require_exact):
     assert np.array_equal(trace["step_features"], trace2["step_features"])
 
 
+def test_alternative_kernel_paths_give_the_same_round_bitwise(monkeypatch):
+    """Two kernels exist for two stages and the library picks one per call; the choice must not show in the
+    result.  The gate/up product finished by the GEMM's own SwiGLU epilogue (POSS_SWIGLU_IN_KERNEL=1) against the
+    consumer kernel over the parked partials: both add a tile's partials in range order and apply the same SiLU,
+    so a whole draft round is equal bit for bit wherever both cut the product into the same CTA ranges, i.e. with
+    more tiles than half the grid (ffn 4864 = 76 tiles here, 224 at full size; with fewer tiles the parked-partials
+    path trims its grid to a multiple of the tile count and the two agree to rounding only).  (The two attention
+    kernels group their sums differently and agree to a bf16 unit: they are compared with the oracle in the
+    attention tests.)"""
+    cfg = ps.CONFIGS["m_bf16"].replace(ffn=4864)
+    w = ps.make_weights(cfg, 12)
+    cap = cfg.prefix + 8 + cfg.tree_slots
+    tok, feat = ps.make_round_inputs(cfg, 12, 3)
+    outs = []
+    for flag in ("0", "1"):
+        monkeypatch.setenv("POSS_SWIGLU_IN_KERNEL", flag)
+        P = make_poss(cfg, w, cap)
+        dkv = dev(ps.make_draft_kv(cfg, 12, cap))
+        out = P.poss_draft_round(dkv, cfg.prefix, torch.from_numpy(tok).cuda(), dev(feat), cfg.depth, cfg.topk, cfg.total)
+        assert P.poss_last_status() == 0
+        outs.append({k: v.cpu().numpy().copy() for k, v in out.items()} | {"kv": pu.np_of(dkv)})
+    for k in outs[0]:
+        assert np.array_equal(outs[0][k], outs[1][k]), k
+
+
 def test_aliased_specialists_equal_single_layer_bitwise():
     base = ps.CONFIGS["t_bf16"]
     tok, feat = ps.make_round_inputs(base, 21, 3)
