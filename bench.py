@@ -288,6 +288,23 @@ def main():
     clocks.close()
     draft_ms = ev[2].elapsed_time(ev[3]) / args.steps
 
+    # spread of single rounds: one event pair per round, in a loop of its own (the figures above stay averages
+    # over back-to-back rounds without events in between)
+    def spread(fn, n):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        evs[0].record()
+        for i in range(n):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        t = sorted(evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(n))
+        return {"p10": t[int(0.1 * (n - 1))], "p50": t[(n - 1) // 2], "p90": t[int(0.9 * (n - 1) + 0.5)], "rounds": n}
+    n_spread = max(5, min(args.steps, 30))
+    spread_draft = spread(lambda: P.poss_draft_round(dkv, cfg.prefix, tok_d, feat_d, cfg.depth, cfg.topk, cfg.total, out=out),
+                          n_spread)
+    spread_step = spread(lambda: step(tok_d, feat_d), n_spread)
+    sync_all()
+
     # every stage kind of the draft steps in isolation (events around each stage cut the launch overlap, so
     # this loop is slower than the round above and only feeds the per-kernel table)
     P.poss_profile(2)
@@ -355,6 +372,7 @@ def main():
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "stages_us": {"draft_round": draft_ms * 1e3, "whole_step": ms * 1e3,
                           "verify_round": max(ms - draft_ms, 0.0) * 1e3},
+            "spread_us": {"draft_round": spread_draft, "whole_step": spread_step},
             "rounds_per_s": rounds_per_second(world, ms),
             "draft_round_gbs": round_bytes / (draft_ms * 1e-3) / 1e9,
             "draft_round_frac_of_hbm_peak": round_bytes / (draft_ms * 1e-3) / 1e9 / hbm_peak,
