@@ -257,6 +257,15 @@ POSS_API int poss_tree_attention_noalloc(const void* q, const void* kv, int kv_s
  * Nothing faults and the context stays usable: poss_reset clears the status. */
 POSS_API int poss_debug_lose_load(poss_ctx* ctx, int launches);
 
+/* Host-only query (no device is touched): how poss_tree_attention and the draft / target passes cut `total_keys`
+ * visible-or-masked keys for a bf16 model with head dimension 128.  The tcgen05 kernel takes up to 2048 keys:
+ * *keys_per_cta = 128 or 256 keys per CTA (groups of 128 keys at absolute positions, one or two per CTA) and
+ * *ctas_per_cluster = CTAs of one (KV head, 128 query rows), 1..8; the cut depends on total_keys alone, and group j
+ * always holds keys [128 j, 128 j + 128).  Returns POSS_OK, or POSS_E_SHAPE for a key count the kernel does not take
+ * (the split-KV kernels then run; outputs untouched), POSS_E_INVALID for NULL outputs or total_keys < 1.
+ * The paper has no counterpart. */
+POSS_API int poss_attention_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster);
+
 /* Number of kernels this context has launched so far (host counter). */
 POSS_API int64_t poss_launch_count(const poss_ctx* ctx);
 

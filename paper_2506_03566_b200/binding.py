@@ -74,6 +74,7 @@ EXPORTS = {
                                     C.c_void_p]),
     "poss_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_float)]),
+    "poss_attention_plan": (C.c_int, [C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
     "poss_debug_lose_load": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_tree_attention_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,

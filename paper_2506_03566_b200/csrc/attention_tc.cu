@@ -425,6 +425,15 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
 }  // namespace
 
 // ------------------------------------------------------------------ host side
+// The cut of the keys: a function of the key count alone.  Two 128-key groups per CTA (one when there are no more
+// than 128 keys), as many CTAs as the keys need.
+bool tree_attention_tc_plan(int total, int* cta_keys, int* n_ctas) {
+  if (total < 1 || total > MAX_SPLITS * MAX_CTA_KEYS) return false;
+  *cta_keys = total <= KG ? KG : MAX_CTA_KEYS;
+  *n_ctas = (total + *cta_keys - 1) / *cta_keys;
+  return true;
+}
+
 bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out) {
   if (a.d != D || a.Hkv < 1 || a.Hq % a.Hkv) return false;
   const int G = a.Hq / a.Hkv;
@@ -453,9 +462,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   memset(&k, 0, sizeof(k));
   k.rows = a.rows; k.Hq = a.Hq; k.G = G; k.n_q = a.rows * G;
   k.n_all = a.n_all; k.n_tree = a.n_tree; k.total = total;
-  // two 128-key groups per CTA (one when there are no more than 128 keys), as many CTAs as the keys need
-  k.cta_keys = total <= KG ? KG : MAX_CTA_KEYS;
-  k.n_splits = (total + k.cta_keys - 1) / k.cta_keys;
+  if (!tree_attention_tc_plan(total, &k.cta_keys, &k.n_splits)) return false;
   k.mask = a.mask; k.mask_words = a.mask_words;
   k.scale_log2 = a.scale * 1.4426950408889634f;
   k.part = part; k.out = out; k.status = status;

@@ -17,6 +17,7 @@ void* tc_encode_fn(TcGemmPlanCache*);
 // Tree attention on tcgen05 (bf16, head dimension 128, at most 2048 keys).  `part` holds one partial per
 // (row, head, 256 keys): rows * Hq * 8 * 132 floats at most, which the split-KV kernels' buffer always covers.
 // Returns false, having launched nothing, when the call is not covered; errors of a launch go to *status.
+bool tree_attention_tc_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster);
 bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out);
 bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
                               const bf16* vc, float* part, bf16* out, int32_t* status);

@@ -834,6 +834,15 @@ int poss_debug_lose_load(poss_ctx* c, int launches) {
   return POSS_OK;
 }
 
+int poss_attention_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster) {
+  if (!keys_per_cta || !ctas_per_cluster || total_keys < 1) return POSS_E_INVALID;
+  int k = 0, n = 0;
+  if (!tree_attention_tc_plan(total_keys, &k, &n)) return POSS_E_SHAPE;
+  *keys_per_cta = k;
+  *ctas_per_cluster = n;
+  return POSS_OK;
+}
+
 int64_t poss_launch_count(const poss_ctx* c) { return c ? c->launches : 0; }
 
 }  // extern "C"
