@@ -8,9 +8,9 @@
 //   1. TMA brings the 128 x 128 query tile and the CTA's 256 keys and values into shared memory
 //      (128-byte swizzle; rows past the last key or the last tree row arrive as zeros);
 //   2. one thread issues S = Q' K^T (tcgen05.mma, M = 128 query rows, N = 256 keys, fp32 in TMEM);
-//   3. eight warps take S out of TMEM, one thread per (query row, group): scale, ancestor mask, row
-//      maximum, p = 2^(s - m), row sum; p is written back to shared memory as an exact two-term bf16
-//      split (p = hi + lo), laid out as the A operand of the next product;
+//   3. sixteen warps take S out of TMEM, one thread per (query row, group, half of the group's keys): scale,
+//      ancestor mask, row maximum (the halves meet through shared memory), p = 2^(s - m), row sum; p is written
+//      back to shared memory as a two-term bf16 split (p = hi + lo), laid out as the A operand of the next product;
 //   4. one thread issues O_g = P_g V_g for both groups (two MMAs per 16 keys: hi and lo; V is the MN-major
 //      B operand, read as it sits in the cache: [key][d]), each group into its own TMEM accumulator;
 //   5. every CTA merges its two groups and parks (m, l) and the 128 x 128 fp32 O in global memory (one
@@ -39,8 +39,7 @@ using namespace tcptx;
 
 constexpr int D = 128;
 constexpr int QT = 128;               // query rows per CTA (UMMA M)
-constexpr int N_SOFTMAX = 256;        // eight warps: TMEM lane quarter x key group
-constexpr int N_THREADS = N_SOFTMAX + 32;
+constexpr int N_THREADS = 512;        // sixteen warps: TMEM lane quarter x key group x half of the group
 constexpr int KG = 128;               // keys per group: the unit of the softmax partials, at absolute positions
 constexpr int MAX_CTA_KEYS = 2 * KG;  // keys per CTA (UMMA N of the first product)
 constexpr int MAX_SPLITS = 8;         // portable cluster size
@@ -91,7 +90,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -129,6 +127,9 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
 }
 
 // ------------------------------------------------------------------ the kernel
+// 512 threads: warp w owns TMEM lane quarter q = w & 3 (32 query rows), key group g = (w >> 2) & 1 and half
+// hf = w >> 3 of the group's eight 16-key chunks in the softmax; column quarter cq = w >> 2 (32 output columns) when
+// the outputs are parked.  Thread 0 also issues the copies and both products.
 __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant__ CUtensorMap map_q,
                                                           const __grid_constant__ CUtensorMap map_k,
                                                           const __grid_constant__ CUtensorMap map_v, const AttnTcArgs a) {
@@ -136,7 +137,8 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   __shared__ __align__(8) uint64_t bars[5];
   __shared__ uint32_t tmem_slot;
   __shared__ int s_abort;
-  __shared__ __align__(8) float2 grp_ml[2][QT];     // (m, l) per group and query row
+  __shared__ float half_max[2][2][QT], half_sum[2][2][QT];     // [half][group][query row]
+  __shared__ float grp_m[2][QT];                               // scaled maximum per group and query row
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
@@ -158,13 +160,13 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
     return n < 0 ? 0 : (n > KG ? KG : n);
   };
 
-  if (warp == 8) {
+  if (warp == 0) {
     if (lane == 0) {
       s_abort = 0;
       mbar_init(bar_qk, 1);
       mbar_init(bar_v, 1);
       mbar_init(bar_s, 1);
-      mbar_init(bar_p, N_SOFTMAX);
+      mbar_init(bar_p, N_THREADS);
       mbar_init(bar_o, 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -186,116 +188,96 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   pdl_begin();
   pdl_sync();
 
-  if (warp == 8) {
-    if (lane == 0) {
-      // ---------------- loads and both products, in program order
-      mbar_expect_tx(bar_qk, 2u * HALF_TILE + 2u * k_half);
-      tma_load_4d(base + q_off, &map_q, bar_qk, 0, 0, kvh, qtile * (QT / a.G));
-      tma_load_4d(base + q_off + HALF_TILE, &map_q, bar_qk, 64, 0, kvh, qtile * (QT / a.G));
-      tma_load_3d(base + k_off, &map_k, bar_qk, 0, k_begin, kvh);
-      tma_load_3d(base + k_off + k_half, &map_k, bar_qk, 64, k_begin, kvh);
-      mbar_expect_tx(bar_v, 2u * k_half);
-      if (!a.inject_lost_load) {
-        tma_load_3d(base + v_off, &map_v, bar_v, 0, k_begin, kvh);
-        tma_load_3d(base + v_off + k_half, &map_v, bar_v, 64, k_begin, kvh);
-      }
-      bool ok = mbar_wait(bar_qk, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t idesc = instr_desc_bf16(QT, cta_keys);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint64_t ad = smem_desc_sw128(base + q_off + h * HALF_TILE), bd = smem_desc_sw128(base + k_off + h * k_half);
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)          // 16 bf16 = 32 bytes = 2 descriptor address units
-            umma_bf16(tmem_base, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (h | kk) ? 1u : 0u);
-        }
-        umma_commit(bar_s);
-      }
-      const bool v_ok = mbar_wait(bar_v, 0, abort_flag);
-      ok = ok && v_ok && mbar_wait(bar_p, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t idesc = instr_desc_bf16(QT, D) | (1u << 16);     // B (the values) is MN-major
-        for (int g = 0; g < ng; ++g) {
-          const int steps = (group_keys(g) + 15) / 16;
-          for (int ks = 0; ks < steps; ++ks) {
-            const int kc = g * (KG / 16) + ks;                          // 16-key step inside the CTA's keys
-            const uint32_t pa = (uint32_t)(kc >> 2) * HALF_TILE;
-            const uint64_t step = (uint64_t)(2 * (kc & 3));
-            const uint64_t ah = smem_desc_sw128(base + p_hi + pa) + step, al = smem_desc_sw128(base + p_lo + pa) + step;
-            const uint64_t bd = smem_desc_sw128_mn(base + v_off + (uint32_t)kc * 2048u, k_half);
-            const uint32_t t_o = tmem_base + o_col + (uint32_t)(g * D);
-            umma_bf16(t_o, ah, bd, idesc, ks > 0 ? 1u : 0u);
-            umma_bf16(t_o, al, bd, idesc, 1u);
-          }
-        }
-        umma_commit(bar_o);
-      }
-      if (*abort_flag) {
-        // drain: the copies this thread started must land before the CTA's shared memory goes away
-        uint64_t t0 = global_ns();
-        while (!mbar_try_wait(bar_qk, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 4) __nanosleep(64);
-        while (!mbar_try_wait(bar_v, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 2) __nanosleep(64);
-      }
+  if (threadIdx.x == 0) {
+    // ---------------- the copies and the first product
+    mbar_expect_tx(bar_qk, 2u * HALF_TILE + 2u * k_half);
+    tma_load_4d(base + q_off, &map_q, bar_qk, 0, 0, kvh, qtile * (QT / a.G));
+    tma_load_4d(base + q_off + HALF_TILE, &map_q, bar_qk, 64, 0, kvh, qtile * (QT / a.G));
+    tma_load_3d(base + k_off, &map_k, bar_qk, 0, k_begin, kvh);
+    tma_load_3d(base + k_off + k_half, &map_k, bar_qk, 64, k_begin, kvh);
+    mbar_expect_tx(bar_v, 2u * k_half);
+    if (!a.inject_lost_load) {
+      tma_load_3d(base + v_off, &map_v, bar_v, 0, k_begin, kvh);
+      tma_load_3d(base + v_off + k_half, &map_v, bar_v, 64, k_begin, kvh);
     }
-  } else {
-    // ---------------- softmax warps: TMEM lane = query row, warps 0-3 take group 0, warps 4-7 group 1
-    const int q = warp & 3, h = warp >> 2;
-    const int row = q * 32 + lane;
-    const int qi = qtile * QT + row;
-    const bool valid = qi < a.n_q;
-    const int r = valid ? qi / a.G : 0;
-    uint64_t mk0 = 0, mk1 = 0;
-    if (valid) {
-      mk0 = a.mask[(size_t)r * a.mask_words];
-      if (a.mask_words > 1) mk1 = a.mask[(size_t)r * a.mask_words + 1];
-    }
-    const int n_chunks = h < ng ? (group_keys(h) + 15) / 16 : 0;      // 16-key chunks of this warp's group
-    const int key_g = k_begin + h * KG;
-    const uint32_t t_s = tmem_base + ((uint32_t)(q * 32) << 16);
-    bool ok = mbar_wait(bar_s, 0, abort_flag);
-    tc_fence_after();
-    POSS_TRACE_POINT(1);
-    float m = NEG_BIG, lsum = 0.f;
-    if (ok && n_chunks > 0) {
-      // Two passes over the group's scores, 16 keys per TMEM load, as compact loops: a CTA runs this code
-      // once, so every instruction is fetched cold and short bodies that iterate beat straight-line code.
-      // Invisible keys become -inf: they lose every maximum and their 2^x is an exact zero.
-      auto chunk = [&](int c, uint32_t* sr) {
-        tmem_ld16_async(t_s + (uint32_t)(h * KG + c * 16), sr);
-        tmem_wait16(sr);
-        const int key0 = key_g + c * 16;
-        if (key0 + 16 > a.n_all) {                         // the chunk reaches the tree slots or the end
-          // bit j = key0 + j is visible: 16 bits cut out of (all ones below n_all | the row's ancestor mask)
-          const int t0 = key0 - a.n_all;                   // tree slot of the chunk's first key; > -16
-          uint32_t vis;
-          if (t0 >= 64) vis = t0 >= 128 ? 0u : (uint32_t)(mk1 >> (t0 - 64));
-          else if (t0 > 48) vis = (uint32_t)(mk0 >> t0) | (uint32_t)(mk1 << (64 - t0));
-          else if (t0 >= 0) vis = (uint32_t)(mk0 >> t0);
-          else vis = ((uint32_t)mk0 << (-t0)) | ((1u << (-t0)) - 1u);
-          const int n_valid = a.total - key0;              // keys of the chunk that exist
-          if (n_valid < 16) vis &= (1u << (n_valid < 0 ? 0 : n_valid)) - 1u;
+    if (mbar_wait(bar_qk, 0, abort_flag)) {
+      tc_fence_after();
+      const uint32_t idesc = instr_desc_bf16(QT, cta_keys);
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (!((vis >> j) & 1u)) sr[j] = 0xff800000u;
-        }
-      };
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      for (int h = 0; h < 2; ++h) {
+        const uint64_t ad = smem_desc_sw128(base + q_off + h * HALF_TILE), bd = smem_desc_sw128(base + k_off + h * k_half);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)          // 16 bf16 = 32 bytes = 2 descriptor address units
+          umma_bf16(tmem_base, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (h | kk) ? 1u : 0u);
+      }
+      umma_commit(bar_s);
+    }
+  }
+  __syncwarp();
+
+  // ---------------- softmax: TMEM lane = query row
+  const int q = warp & 3, g = (warp >> 2) & 1, hf = warp >> 3;
+  const int row = q * 32 + lane;
+  const int qi = qtile * QT + row;
+  const bool valid = qi < a.n_q;
+  const int r = valid ? qi / a.G : 0;
+  uint64_t mk0 = 0, mk1 = 0;
+  if (valid) {
+    mk0 = a.mask[(size_t)r * a.mask_words];
+    if (a.mask_words > 1) mk1 = a.mask[(size_t)r * a.mask_words + 1];
+  }
+  const int n_grp = g < ng ? (group_keys(g) + 15) / 16 : 0;          // 16-key chunks of this warp's group
+  const int c_lo = hf * 4 < n_grp ? hf * 4 : n_grp, c_hi = hf * 4 + 4 < n_grp ? hf * 4 + 4 : n_grp;
+  const int key_g = k_begin + g * KG;
+  const uint32_t t_s = tmem_base + ((uint32_t)(q * 32) << 16);
+  bool ok = mbar_wait(bar_s, 0, abort_flag);
+  tc_fence_after();
+  POSS_TRACE_POINT(1);
+  // Two passes over this thread's scores, 16 keys per TMEM load, as compact loops: a CTA runs this code once, so
+  // every instruction is fetched cold and short bodies that iterate beat straight-line code.  Invisible keys become
+  // -inf: they lose every maximum and their 2^x is an exact zero.
+  auto chunk = [&](int c, uint32_t* sr) {
+    tmem_ld16_async(t_s + (uint32_t)(g * KG + c * 16), sr);
+    tmem_wait16(sr);
+    const int key0 = key_g + c * 16;
+    if (key0 + 16 > a.n_all) {                         // the chunk reaches the tree slots or the end
+      // bit j = key0 + j is visible: 16 bits cut out of (all ones below n_all | the row's ancestor mask)
+      const int t0 = key0 - a.n_all;                   // tree slot of the chunk's first key; > -16
+      uint32_t vis;
+      if (t0 >= 64) vis = t0 >= 128 ? 0u : (uint32_t)(mk1 >> (t0 - 64));
+      else if (t0 > 48) vis = (uint32_t)(mk0 >> t0) | (uint32_t)(mk1 << (64 - t0));
+      else if (t0 >= 0) vis = (uint32_t)(mk0 >> t0);
+      else vis = ((uint32_t)mk0 << (-t0)) | ((1u << (-t0)) - 1u);
+      const int n_valid = a.total - key0;              // keys of the chunk that exist
+      if (n_valid < 16) vis &= (1u << (n_valid < 0 ? 0 : n_valid)) - 1u;
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (!((vis >> j) & 1u)) sr[j] = 0xff800000u;
+    }
+  };
+  {
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    if (ok) {
 #pragma unroll 1
-      for (int c = 0; c < n_chunks; ++c) {
+      for (int c = c_lo; c < c_hi; ++c) {
         uint32_t sr[16];
         chunk(c, sr);
 #pragma unroll
         for (int j = 0; j < 16; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sr[j]));
       }
-      const float mraw = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      // the scale is positive: the maximum of the scaled scores is the scaled maximum
-      const float ms = mraw == -INFINITY ? 0.f : mraw * a.scale_log2;
-      if (mraw != -INFINITY) m = ms;
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+    }
+    half_max[hf][g][row] = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+  }
+  __syncthreads();
+  {
+    const float mraw = fmaxf(half_max[0][g][row], half_max[1][g][row]);
+    // the scale is positive: the maximum of the scaled scores is the scaled maximum
+    const float ms = mraw == -INFINITY ? 0.f : mraw * a.scale_log2;
+    if (hf == 0) grp_m[g][row] = mraw == -INFINITY ? NEG_BIG : ms;
+    float ls[4] = {0.f, 0.f, 0.f, 0.f};
+    if (ok) {
 #pragma unroll 1
-      for (int c = 0; c < n_chunks; ++c) {
+      for (int c = c_lo; c < c_hi; ++c) {
         uint32_t sr[16];
         chunk(c, sr);
         uint32_t hi[8], lo[8];
@@ -308,7 +290,7 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
           split_pack(p0, p1, hi[j >> 1], lo[j >> 1]);
         }
         // A operand of P V: k-block of 64 keys, row = query row (128 bytes), 16-byte pieces swizzled by row
-        const int kc = h * (KG / 16) + c;
+        const int kc = g * (KG / 16) + c;
         const uint32_t line = (uint32_t)(kc >> 2) * HALF_TILE + (uint32_t)row * 128u;
         const uint32_t pc = (uint32_t)(kc & 3) * 2u, sw = (uint32_t)(row & 7);
         *reinterpret_cast<uint4*>(base_ptr + p_hi + line + ((pc ^ sw) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -316,45 +298,77 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         *reinterpret_cast<uint4*>(base_ptr + p_lo + line + ((pc ^ sw) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         *reinterpret_cast<uint4*>(base_ptr + p_lo + line + (((pc + 1) ^ sw) << 4)) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
       }
-      lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
     }
-    if (h < ng) grp_ml[h][row] = make_float2(m, lsum);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P becomes visible to the tensor core
-    mbar_arrive(bar_p);
-    POSS_TRACE_POINT(2);
-    ok = mbar_wait(bar_o, 0, abort_flag);
-    tc_fence_after();
-    POSS_TRACE_POINT(3);
-    softmax_sync();                 // both groups' (m, l) of every row are in place
-    if (ok) {
-      // park O in global memory (it stays in L2): this warp's 32 query rows, output columns [64 h, 64 h + 64),
-      // the CTA's groups merged in key order (a group without keys accumulated nothing: it is left out, its
-      // TMEM columns are not read)
-      const bool two = ng == 2 && group_keys(1) > 0;
-      const float2 ml0 = grp_ml[0][row], ml1 = two ? grp_ml[1][row] : make_float2(NEG_BIG, 0.f);
-      const float ms = fmaxf(ml0.x, ml1.x);
-      const float c0 = ex2(ml0.x - ms), c1 = two ? ex2(ml1.x - ms) : 0.f;
-      const uint32_t t_o = t_s + o_col + (uint32_t)(h * 64);
-      float* dst = a.part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * a.n_splits + split) * O_LD;
-      if (valid && h == 0) *reinterpret_cast<float2*>(dst + D) = make_float2(ms, ml0.y * c0 + ml1.y * c1);
+    half_sum[hf][g][row] = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P becomes visible to the tensor core
+  mbar_arrive(bar_p);
+  POSS_TRACE_POINT(2);
+
+  if (threadIdx.x == 0) {
+    // ---------------- the second product, once the values and all of P are in shared memory
+    const bool v_ok = mbar_wait(bar_v, 0, abort_flag);
+    if (v_ok && mbar_wait(bar_p, 0, abort_flag) && *abort_flag == 0) {
+      tc_fence_after();
+      const uint32_t idesc = instr_desc_bf16(QT, D) | (1u << 16);     // B (the values) is MN-major
+      for (int gg = 0; gg < ng; ++gg) {
+        const int steps = (group_keys(gg) + 15) / 16;
+        for (int ks = 0; ks < steps; ++ks) {
+          const int kc = gg * (KG / 16) + ks;                         // 16-key step inside the CTA's keys
+          const uint32_t pa = (uint32_t)(kc >> 2) * HALF_TILE;
+          const uint64_t step = (uint64_t)(2 * (kc & 3));
+          const uint64_t ah = smem_desc_sw128(base + p_hi + pa) + step, al = smem_desc_sw128(base + p_lo + pa) + step;
+          const uint64_t bd = smem_desc_sw128_mn(base + v_off + (uint32_t)kc * 2048u, k_half);
+          const uint32_t t_o = tmem_base + o_col + (uint32_t)(gg * D);
+          umma_bf16(t_o, ah, bd, idesc, ks > 0 ? 1u : 0u);
+          umma_bf16(t_o, al, bd, idesc, 1u);
+        }
+      }
+      umma_commit(bar_o);
+    }
+    if (*abort_flag) {
+      // drain: the copies this thread started must land before the CTA's shared memory goes away
+      uint64_t t0 = global_ns();
+      while (!mbar_try_wait(bar_qk, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 4) __nanosleep(64);
+      while (!mbar_try_wait(bar_v, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 2) __nanosleep(64);
+    }
+  }
+  __syncwarp();
+  ok = mbar_wait(bar_o, 0, abort_flag);
+  tc_fence_after();
+  POSS_TRACE_POINT(3);
+  __syncthreads();                  // every half's sum and every group's maximum are in place
+  if (ok) {
+    // park O in global memory (it stays in L2): this warp's 32 query rows, output columns [32 cq, 32 cq + 32), the
+    // CTA's groups merged in key order (a group without keys accumulated nothing: it is left out, its TMEM columns
+    // are not read)
+    const int cq = warp >> 2;
+    const bool two = ng == 2 && group_keys(1) > 0;
+    const float m0 = grp_m[0][row], m1 = two ? grp_m[1][row] : NEG_BIG;
+    const float l0 = half_sum[0][0][row] + half_sum[1][0][row];
+    const float l1 = two ? half_sum[0][1][row] + half_sum[1][1][row] : 0.f;
+    const float ms = fmaxf(m0, m1);
+    const float c0 = ex2(m0 - ms), c1 = two ? ex2(m1 - ms) : 0.f;
+    const uint32_t t_o = t_s + o_col + (uint32_t)(cq * 32);
+    float* dst = a.part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * a.n_splits + split) * O_LD;
+    if (valid && cq == 0) *reinterpret_cast<float2*>(dst + D) = make_float2(ms, l0 * c0 + l1 * c1);
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t v0[16], v1[16];
-        tmem_ld16_async(t_o + (uint32_t)(cc * 16), v0);
-        if (two) tmem_ld16_async(t_o + (uint32_t)(D + cc * 16), v1);
-        tmem_wait16(v0);
-        if (two) tmem_wait16(v1);
-        float v[16];
+    for (int cc = 0; cc < 2; ++cc) {
+      uint32_t v0[16], v1[16];
+      tmem_ld16_async(t_o + (uint32_t)(cc * 16), v0);
+      if (two) tmem_ld16_async(t_o + (uint32_t)(D + cc * 16), v1);
+      tmem_wait16(v0);
+      if (two) tmem_wait16(v1);
+      float v[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          v[j] = __uint_as_float(v0[j]) * c0;
-          if (two) v[j] += __uint_as_float(v1[j]) * c1;
-        }
-        if (valid) {
+      for (int j = 0; j < 16; ++j) {
+        v[j] = __uint_as_float(v0[j]) * c0;
+        if (two) v[j] += __uint_as_float(v1[j]) * c1;
+      }
+      if (valid) {
 #pragma unroll
-          for (int j = 0; j < 16; j += 4)
-            __stcg(reinterpret_cast<float4*>(dst + h * 64 + cc * 16 + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
-        }
+        for (int j = 0; j < 16; j += 4)
+          __stcg(reinterpret_cast<float4*>(dst + cq * 32 + cc * 16 + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
       }
     }
   }
@@ -373,10 +387,10 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
 #pragma unroll 1
     for (int item = threadIdx.x; item < (row_hi - row_lo) * 16; item += N_THREADS) {
       const int rr = row_lo + (item >> 4), cg = (item & 15) * 8;
-      const int qi = qtile * QT + rr;
-      if (qi >= a.n_q) continue;
-      const int r = qi / a.G, g = qi - r * a.G;
-      const float* src = a.part + (((size_t)r * a.Hq + kvh * a.G + g) * ns) * O_LD;
+      const int qj = qtile * QT + rr;
+      if (qj >= a.n_q) continue;
+      const int rj = qj / a.G, gj = qj - rj * a.G;
+      const float* src = a.part + (((size_t)rj * a.Hq + kvh * a.G + gj) * ns) * O_LD;
       // every load is in flight before the first use
       float2 ml[MAX_SPLITS];
       float4 x0[MAX_SPLITS], x1[MAX_SPLITS];
@@ -411,14 +425,14 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * j] * inv, acc[2 * j + 1] * inv);
         w[j] = *reinterpret_cast<uint32_t*>(&b);
       }
-      *reinterpret_cast<uint4*>(a.out + ((size_t)r * a.Hq + kvh * a.G + g) * D + cg) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(a.out + ((size_t)rj * a.Hq + kvh * a.G + gj) * D + cg) = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 
   POSS_TRACE_POINT(5);
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tmem_base, tmem_cols);
+  if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
   if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, (int)POSS_E_TIMEOUT);
 }
 
