@@ -126,6 +126,33 @@ def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv
         assert np.abs(got - want).max() <= 2e-2
 
 
+def test_tensor_core_tree_attention_on_random_shapes():
+    """24 seeded random shapes at head dimension 128 (1..64 rows, prefix 0..1500, 1..8 KV heads, GQA 1..8, cache
+    capacity with and without slack, random trees and chains) against the oracle."""
+    rng = np.random.default_rng(2024)
+    d = 128
+    ctxs = {}
+    for trial in range(24):
+        Hkv, G = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4, 8]))
+        Hq = Hkv * G
+        rows = int(rng.integers(1, 65))
+        P_len = int(rng.integers(0, 1501))
+        cap = P_len + rows + int(rng.integers(0, 9))
+        cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
+        if (Hq, Hkv) not in ctxs:
+            ctxs[(Hq, Hkv)] = make_poss(cfg, ps.make_weights(cfg, 1), 64)
+        P = ctxs[(Hq, Hkv)]
+        q, kv = ps.make_attention_case(3000 + trial, rows, Hq, Hkv, d, P_len, cap, cfg.dtype)
+        parents = ps.random_tree_parents(4000 + trial, rows) if trial % 3 else po.chain_parents(rows)
+        mask = po.pack_mask(po.ancestor_matrix(parents))
+        scale = 1.0 / math.sqrt(d)
+        got = pu.np_of(P.poss_tree_attention(dev(q), dev(kv), P_len, torch.from_numpy(mask.view(np.int64)).cuda(), scale))
+        assert P.poss_last_status() == 0
+        want = po.tree_attention(q, kv, P_len, parents, scale, pu.oracle_num(cfg))
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= 2e-2, (trial, rows, P_len, Hq, Hkv)
+
+
 def test_tree_root_row_equals_its_single_row_decode_bitwise():
     """The property the lossless loop rests on: a token whose visible keys are the prefix and itself gets the same
     attention output, bit for bit, as the root of a 61-row tree pass and as a single decoded row, also where the
