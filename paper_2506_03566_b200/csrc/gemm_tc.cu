@@ -619,7 +619,7 @@ struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
   int inject = 0;          // launches left whose first activation tile is withheld (wait-expiry test hook)
-  int grid = 0, stages = 0, w_policy = 1, smem_kb = 150, align_ranges = 1, split_topk = 0;
+  int grid = 0, stages = 0, w_policy = 1, smem_kb = 0, align_ranges = 1, split_topk = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -774,7 +774,11 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
   if (ep.mode == TC_EPI_TOPK && !argmax) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
-  int stages = cache->stages ? cache->stages : (int)(((size_t)cache->smem_kb * 1024u - extra - 1024u) / stage_bytes);
+  // Ring size (measured on the c2 round; POSS_TC_SMEM_KB overrides): 170 KB = nine 18 KB stages for up to 16 rows
+  // (150 KB: +12 us per draft round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass;
+  // 176 and 220 KB: +18 us per pass)
+  const int smem_kb = cache->smem_kb ? cache->smem_kb : (a.Npad <= 16 ? 170 : 200);
+  int stages = cache->stages ? cache->stages : (int)(((size_t)smem_kb * 1024u - extra - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
