@@ -12,7 +12,9 @@
  *
  * Conventions
  *   - Every function returns a poss_status; nothing throws, aborts or traps.
- *   - Pointers are DEVICE pointers owned by the caller unless the name starts with h_.
+ *   - Pointers are DEVICE pointers owned by the caller unless the name starts with h_.  Tensors (weights,
+ *     caches, q, features, outputs) start on a 16-byte boundary; a misaligned one is POSS_E_INVALID where the
+ *     call can see it on the host.
  *   - The library allocates no device memory: all scratch lives in the workspace the caller
  *     hands to poss_init (size from poss_workspace_bytes) and must outlive the context.
  *   - All work is enqueued on the stream argument and is asynchronous; no call synchronises
@@ -125,20 +127,15 @@ POSS_API int poss_draft_round(poss_ctx* ctx, void* draft_kv, int prefix_len,
                      int32_t* out_depth, uint64_t* out_anc_mask, int32_t* out_n_nodes,
                      poss_stream stream);
 
-/* Copies the last draft round's intermediate state out of the workspace (any pointer may be NULL):
- * cand_* [topk + (depth-1)*topk^2] every candidate in creation order (parent = flat index of the
- * parent candidate, -1 = root); frontier int32[depth-1][topk] flat candidate indices expanded at
- * steps 1..depth-1, best first; step_features float[depth][topk][H] the specialist features of the
- * rows expanded at each step (step 0 uses row 0 only); selected int32[n_nodes-1] flat indices kept
- * by the rerank, ascending. */
-POSS_API int poss_draft_trace(poss_ctx* ctx, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores,
-                     int32_t* frontier, float* step_features, int32_t* selected, poss_stream stream);
-
-/* Tree-masked attention (the verification pass's attention; also used by every draft step).
+/* Tree-masked attention: every draft token attends to the committed context and to its own path in the draft
+ * tree only, which is what lets the target check all draft tokens in one parallel pass (Section 2.1, the
+ * verification phase) and lets a draft step extend every frontier node at once (Eq. 2: a prediction conditions
+ * on its own previously generated features and tokens).  Used by the target pass and by every draft step.
  * q, out [rows][n_q_heads][head_dim]; kv [2][n_kv_heads][kv_slots][head_dim] with the rows' own
  * keys/values already at slots prefix_len+r.  Row r sees slots [0, prefix_len) and slot
  * prefix_len+j for every bit j set in anc_mask[r] (uint64[rows][ceil(rows/64)]).
- * Query head h reads KV head h / (n_q_heads / n_kv_heads).  rows <= POSS_MAX_ROWS. */
+ * Query head h reads KV head h / (n_q_heads / n_kv_heads).  rows <= POSS_MAX_ROWS.
+ * q, kv and out 16-byte aligned (else POSS_E_INVALID). */
 POSS_API int poss_tree_attention(poss_ctx* ctx, const void* q, const void* kv, int kv_slots, int prefix_len,
                         int rows, const uint64_t* anc_mask, float scale, void* out, poss_stream stream);
 
@@ -173,7 +170,9 @@ POSS_API int poss_verify_sample(poss_ctx* ctx, const float* target_logits, const
                        int32_t* out_new_tokens, void* out_new_features, int32_t* out_uniforms_used,
                        poss_stream stream);
 
-/* Target model over `rows` tree rows: row r holds tokens[r], sits at rotary position
+/* The verification phase's forward pass (Section 2.1: the target evaluates all draft tokens in parallel in a
+ * single forward pass; Section 3.1 uses its per-position greedy tokens to decide acceptance).
+ * Target model over `rows` tree rows: row r holds tokens[r], sits at rotary position
  * prefix_len + depth[r], is written to cache slot prefix_len + r and sees the prefix plus its
  * ancestors and itself (anc_mask as above).  A chain (depth r, lower-triangular mask) is plain
  * causal decoding / prefill.  target_kv [layers][2][n_kv_heads][target_kv_slots][head_dim].
@@ -182,13 +181,22 @@ POSS_API int poss_verify_sample(poss_ctx* ctx, const float* target_logits, const
 POSS_API int poss_target_forward(poss_ctx* ctx, void* target_kv, int prefix_len, const int32_t* tokens,
                         const int32_t* depth, const uint64_t* anc_mask, int rows,
                         void* out_features, int32_t* out_argmax, float* out_logits, poss_stream stream);
+/* The same pass under the name of its role in a round: tree verification without the logits
+ * (poss_target_forward with out_logits = NULL). */
+POSS_API int poss_target_verify(poss_ctx* ctx, void* target_kv, int prefix_len, const int32_t* tokens,
+                       const int32_t* depth, const uint64_t* anc_mask, int rows,
+                       void* out_features, int32_t* out_argmax, poss_stream stream);
 
-/* Causal prefill of n prompt tokens from position `start` (chunks of POSS_MAX_ROWS rows).
+/* The target's pass over the prompt, which leaves the features f_j and the cache the first round starts from
+ * (Section 2.1: the draft model conditions on the target's features of the committed tokens, Eq. 1).
+ * Causal prefill of n prompt tokens from position `start` (chunks of POSS_MAX_ROWS rows).
  * out_features [n][H], out_argmax int32[n] (may be NULL). */
 POSS_API int poss_target_prefill(poss_ctx* ctx, void* target_kv, int start, const int32_t* tokens, int n,
                         void* out_features, int32_t* out_argmax, poss_stream stream);
 
-/* After acceptance: in every target layer move tree slot prefix_len + path[k] to prefix_len + k
+/* Commit of a round (Section 2.1: accepted tokens join the context of the next round; Section 3.3: the caches
+ * hold previously verified tokens): the accepted path's cache entries become contiguous behind the prefix.
+ * After acceptance: in every target layer move tree slot prefix_len + path[k] to prefix_len + k
  * for k = 1..*n_accepted (path and n_accepted are the device outputs of poss_verify_accept). */
 POSS_API int poss_kv_compact(poss_ctx* ctx, void* target_kv, int prefix_len, const int32_t* path,
                     const int32_t* n_accepted, poss_stream stream);
@@ -216,19 +224,6 @@ POSS_API int poss_linear(poss_ctx* ctx, const void* x, int M, const void* w, int
 POSS_API int poss_lm_head_topk(poss_ctx* ctx, const void* features, int rows, int topk,
                       int32_t* out_ids, float* out_logp, float* out_logits, poss_stream stream);
 
-/* Device-time bracketing of the draft steps' stages, for roofline reporting.  mode 0: off; mode 1: the LM-head
- * matrix product (the dominant kernel) of every draft step sits between two CUDA events on the launching stream;
- * mode 2: so does every stage kind below (the launches between the two events are the product's kernel, plus the
- * combine kernel for POSS_PROF_ATTENTION and the in-kernel or consumer-side SwiGLU for POSS_PROF_GATE_UP).  The
- * events cut the overlap between neighbouring launches, so mode 2 times each stage in isolation and lengthens the
- * round; at most 1024 brackets between reads.  poss_profile_read SYNCHRONISES on the last event, returns per kind
- * how many launches were bracketed since the previous read and their summed device time in ms (arrays of
- * POSS_PROF_KINDS entries), and starts over.  The target pass is never bracketed. */
-enum { POSS_PROF_FC = 0, POSS_PROF_QKV = 1, POSS_PROF_ATTENTION = 2, POSS_PROF_O = 3, POSS_PROF_GATE_UP = 4,
-       POSS_PROF_DOWN = 5, POSS_PROF_LM_HEAD = 6, POSS_PROF_KINDS = 7 };
-POSS_API int poss_profile(poss_ctx* ctx, int mode);
-POSS_API int poss_profile_read(poss_ctx* ctx, int* h_launches, float* h_total_ms);
-
 /* Tree-masked attention for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a packaging variant of poss_tree_attention).
  * Who needs it: code that is handed device pointers but may not call cudaMalloc -- an engine whose
@@ -249,14 +244,6 @@ POSS_API int poss_tree_attention_noalloc(const void* q, const void* kv, int kv_s
                                          int rows, int n_q_heads, int n_kv_heads, int head_dim, int dtype,
                                          const uint64_t* anc_mask, float scale, void* out, poss_stream stream);
 
-/* Failure-detection test hook (the paper has no counterpart).  The next `launches` tensor-core launches of this
- * context (matrix products and tcgen05 tree attention alike) withhold one tile from their own pipeline (a product:
- * one activation tile; attention: the value tiles), so the bounded wait on that tile runs out (after about one
- * second): every CTA stops issuing work, waits (bounded) for its copies in flight, frees its tensor memory and
- * returns; the device status word becomes POSS_E_TIMEOUT (poss_last_status) and the launch's results are undefined.
- * Nothing faults and the context stays usable: poss_reset clears the status. */
-POSS_API int poss_debug_lose_load(poss_ctx* ctx, int launches);
-
 /* Host-only query (no device is touched): how poss_tree_attention and the draft / target passes cut `total_keys`
  * visible-or-masked keys for a bf16 model with head dimension 128.  The tcgen05 kernel takes up to 2048 keys:
  * *keys_per_cta = 128 or 256 keys per CTA (groups of 128 keys at absolute positions, one or two per CTA) and
@@ -265,9 +252,6 @@ POSS_API int poss_debug_lose_load(poss_ctx* ctx, int launches);
  * (the split-KV kernels then run; outputs untouched), POSS_E_INVALID for NULL outputs or total_keys < 1.
  * The paper has no counterpart. */
 POSS_API int poss_attention_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster);
-
-/* Number of kernels this context has launched so far (host counter). */
-POSS_API int64_t poss_launch_count(const poss_ctx* ctx);
 
 #ifdef __cplusplus
 }

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(HERE, "libposs.so")
 POSS_FP32, POSS_BF16 = 0, 1
 POSS_MAX_ROWS, POSS_MAX_TOPK, POSS_MAX_DEPTH = 128, 16, 16
 PROF_KINDS = ("fc", "qkv", "attention", "o", "gate_up", "down", "lm_head")
+POSS_OPT_ATTENTION_TCGEN05, POSS_OPT_SWIGLU_IN_KERNEL = 0, 1
 STATUS = {0: "POSS_OK", 1: "POSS_E_INVALID", 2: "POSS_E_SHAPE", 3: "POSS_E_CAPACITY", 4: "POSS_E_WORKSPACE",
           5: "POSS_E_CUDA", 6: "POSS_E_TIMEOUT"}
 
@@ -63,6 +64,8 @@ EXPORTS = {
     "poss_verify_sample": (C.c_int, [C.c_void_p] * 5 + [C.c_int, C.c_float, C.c_void_p, C.c_int] + [C.c_void_p] * 7),
     "poss_target_forward": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "poss_target_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                     C.c_void_p, C.c_void_p, C.c_void_p]),
     "poss_target_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
     "poss_kv_compact": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -77,6 +80,7 @@ EXPORTS = {
     "poss_attention_plan": (C.c_int, [C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
     "poss_debug_lose_load": (C.c_int, [C.c_void_p, C.c_int]),
+    "poss_debug_option": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "poss_tree_attention_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                               C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
 }
@@ -288,6 +292,15 @@ class Poss:
                "poss_target_forward")
         return feats, arg, logits
 
+    def poss_target_verify(self, target_kv, prefix_len, tokens, depth, anc_mask, rows):
+        c = self.config
+        feats = torch.empty((rows, c.hidden), dtype=self.dtype, device="cuda")
+        arg = torch.empty(rows, dtype=torch.int32, device="cuda")
+        _check(self.lib.poss_target_verify(self.ctx, _ptr(target_kv), prefix_len, _ptr(tokens), _ptr(depth),
+                                           _ptr(anc_mask), rows, _ptr(feats), _ptr(arg), _stream()),
+               "poss_target_verify")
+        return feats, arg
+
     def poss_target_prefill(self, target_kv, start, tokens):
         n = int(tokens.numel())
         feats = torch.empty((n, self.config.hidden), dtype=self.dtype, device="cuda")
@@ -338,6 +351,9 @@ class Poss:
 
     def poss_debug_lose_load(self, launches: int):
         _check(self.lib.poss_debug_lose_load(self.ctx, int(launches)), "poss_debug_lose_load")
+
+    def poss_debug_option(self, option: int, value: int):
+        _check(self.lib.poss_debug_option(self.ctx, int(option), int(value)), "poss_debug_option")
 
     def poss_launch_count(self) -> int:
         return int(self.lib.poss_launch_count(self.ctx))

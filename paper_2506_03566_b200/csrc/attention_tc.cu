@@ -513,10 +513,12 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
+  // the shared-memory opt-in is a per-device property of the kernel
+  static PerDeviceFlags attr_done;
+  bool* attr = attr_done.current();
+  if (!attr || !*attr) {
     if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return false;
-    attr_done = true;
+    if (attr) *attr = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
@@ -535,11 +537,12 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   cfg.numAttrs = 2;
   // A cluster shape the device does not take is reported at launch, before anything runs: remember it and
   // leave the call to the split-KV kernels.
-  static bool refused[MAX_SPLITS + 1] = {};
-  if (refused[k.n_splits]) return false;
+  static PerDeviceFlags refused[MAX_SPLITS + 1];
+  bool* ref = refused[k.n_splits].current();
+  if (ref && *ref) return false;
   if (cudaLaunchKernelEx(&cfg, k_attn_tc, mq, mk, mv, k) != cudaSuccess) {
     cudaGetLastError();
-    refused[k.n_splits] = true;
+    if (ref) *ref = true;
     return false;
   }
   ++*L.launches;

@@ -64,7 +64,7 @@ constexpr int XCH_STRIDE = 17;
 struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
-  int n_tiles, kb_total, gran, w_policy, slots, pair_tiles;
+  int n_tiles, kb_total, gran, slots, pair_tiles;
   int inject_lost_load;   // test hook: the producer leaves out the activation tile of its first stage
   const bf16* bias;
   const float* residual;
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   if (warp == 0) {
     if (lane == 0 && n_kb > 0) {
       // ---------------- TMA producer
-      const uint64_t pol_w = a.w_policy ? policy_evict_first() : policy_evict_normal(), pol_x = policy_evict_last();
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();   // weights pass through L2 once
       // position of the next k-block to load, advanced without divisions
       struct Cursor { int tile, kb, seg, lt; };
       auto cursor_at = [&](long long u) {
@@ -619,7 +619,7 @@ struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
   int inject = 0;          // launches left whose first activation tile is withheld (wait-expiry test hook)
-  int grid = 0, stages = 0, w_policy = 1, smem_kb = 0, align_ranges = 1, split_topk = 0;
+  int grid = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -630,16 +630,8 @@ TcGemmPlanCache* tc_plan_cache_create() {
   if (sms < 1) sms = 148;
   // The grid is a property of the device, not of a call: the work split (and with it the order in
   // which a tile's partial sums are added) must not change from call to call.
-  int per_sm = 1;
-  if (const char* e = getenv("POSS_TC_CTAS_PER_SM")) { int v = atoi(e); if (v >= 1 && v <= 2) per_sm = v; }
-  c->grid = sms * per_sm;
+  c->grid = sms;                       // one persistent CTA per SM
   if (c->grid > TC_MAX_GRID) c->grid = TC_MAX_GRID;
-  c->stages = 0;
-  if (const char* e = getenv("POSS_TC_STAGES")) { int v = atoi(e); if (v >= 2 && v <= MAX_STAGES) c->stages = v; }
-  if (const char* e = getenv("POSS_TC_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 220) c->smem_kb = v; }
-  if (const char* e = getenv("POSS_TC_SPLIT_TOPK")) { int v = atoi(e); if (v >= 0 && v <= 1) c->split_topk = v; }
-  if (const char* e = getenv("POSS_TC_ALIGN")) { int v = atoi(e); if (v >= 0 && v <= 1) c->align_ranges = v; }
-  if (const char* e = getenv("POSS_TC_W_POLICY")) { int v = atoi(e); if (v >= 0 && v <= 1) c->w_policy = v; }
   return c;
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
@@ -650,6 +642,12 @@ bool tc_take_injection(TcGemmPlanCache* c) {
   return true;
 }
 size_t tc_gemm_scratch_bytes() { return SCRATCH_PARTIAL_BYTES + N_COUNTERS * sizeof(int); }
+// The per-tile arrival counters return to zero by themselves after every launch that ran to its end; a launch
+// whose bounded wait ran out may leave some behind.
+bool tc_gemm_clear_counters(void* scratch, cudaStream_t stream) {
+  return cudaMemsetAsync(reinterpret_cast<char*>(scratch) + SCRATCH_PARTIAL_BYTES, 0, N_COUNTERS * sizeof(int),
+                         stream) == cudaSuccess;
+}
 
 void* tc_encode_fn(TcGemmPlanCache* c) {
   if (!c->tried) {
@@ -740,13 +738,12 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
       ep.view->ld = ep.ldo;
     }
   }
-  // whole tiles per CTA for the argmax epilogue (its state lives in registers and only the whole-tile path
-  // feeds it), and whenever the partial buffers or the tile counters could not hold the split.  The top-k
-  // epilogue takes split tiles like any other: a CTA meets its tiles in increasing order either way, so
-  // "a later equal value loses" still means "the lower id wins".
+  // whole tiles per CTA for the LM-head epilogues (the argmax state lives in registers and only the whole-tile
+  // path feeds it; the top-k lists measured slower with split tiles), and whenever the partial buffers or the
+  // tile counters could not hold the split.
   const bool argmax = ep.mode == TC_EPI_TOPK && ep.argmax_only && ep.topk == 1 && a.Npad <= 64;
   size_t part_bytes = (size_t)cache->grid * 2 * a.Npad * TILE_N * sizeof(float);
-  bool no_split = argmax || (a.mode == TC_EPI_TOPK && !cache->split_topk) || part_bytes > SCRATCH_PARTIAL_BYTES ||
+  bool no_split = argmax || a.mode == TC_EPI_TOPK || part_bytes > SCRATCH_PARTIAL_BYTES ||
                   n_tiles > N_COUNTERS;
   a.gran = no_split ? a.kb_total : 1;
   // never more CTAs than ranges to hand out: every CTA of the grid owns at least one k-block
@@ -755,7 +752,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   // Partials left to the consumer: a grid that is a whole multiple of the tile count gives every tile the
   // same number of equal ranges, none straddling two tiles, so each CTA parks one segment and the
   // consumer adds grid/tiles partials instead of one or two more.
-  if (a.mode == TC_EPI_PARTIAL && cache->align_ranges && n_tiles * 2 <= G) {
+  if (a.mode == TC_EPI_PARTIAL && n_tiles * 2 <= G) {
     int per_tile = G / n_tiles;
     if (per_tile > a.kb_total) per_tile = a.kb_total;
     G = per_tile * n_tiles;
@@ -774,15 +771,14 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
   if (ep.mode == TC_EPI_TOPK && !argmax) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
-  // Ring size (measured on the c2 round; POSS_TC_SMEM_KB overrides): 170 KB = nine 18 KB stages for up to 16 rows
-  // (150 KB: +12 us per draft round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass;
-  // 176 and 220 KB: +18 us per pass)
-  const int smem_kb = cache->smem_kb ? cache->smem_kb : (a.Npad <= 16 ? 170 : 200);
-  int stages = cache->stages ? cache->stages : (int)(((size_t)smem_kb * 1024u - extra - 1024u) / stage_bytes);
+  // Ring size (measured on the c2 round): 170 KB = nine 18 KB stages for up to 16 rows (150 KB: +12 us per draft
+  // round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass; 176 and 220 KB: +18 us
+  // per pass)
+  const int smem_kb = a.Npad <= 16 ? 170 : 200;
+  int stages = (int)(((size_t)smem_kb * 1024u - extra - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
-  a.w_policy = cache->w_policy;
   a.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;

@@ -11,6 +11,8 @@ void tc_inject_lost_load(TcGemmPlanCache*, int launches);
 // consumes one pending injection (true when this launch has to withhold its tile)
 bool tc_take_injection(TcGemmPlanCache*);
 size_t tc_gemm_scratch_bytes();
+// zeroes the per-tile arrival counters inside the scratch (after a launch that gave up on a wait)
+bool tc_gemm_clear_counters(void* scratch, cudaStream_t stream);
 // the driver's tensor-map encoder (cuTensorMapEncodeTiled), resolved once; NULL when it cannot be had
 void* tc_encode_fn(TcGemmPlanCache*);
 

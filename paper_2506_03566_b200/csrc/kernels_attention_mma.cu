@@ -333,13 +333,14 @@ __global__ void __launch_bounds__(128) k_attn_combine_bf16(int n_splits, int n_r
 template <int D, int NW>
 void launch_dn(Launcher& L, const AttnArgs& a, const bf16* q, const bf16* kc, const bf16* vc, float* part, bf16* out) {
   constexpr size_t smem = (size_t)2 * 2 * CHUNK * (D + 8) * sizeof(bf16);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceFlags attr_done;             // one per instantiation; the opt-in is per device
+  bool* attr = attr_done.current();
+  if (!attr || !*attr) {
     if (cudaFuncSetAttribute(k_attn_mma<D, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
-    attr_done = true;
+    if (attr) *attr = true;
   }
   int G = a.Hq / a.Hkv;
   int q_tiles = (a.rows * G + 16 * NW - 1) / (16 * NW);

@@ -18,7 +18,6 @@ static __device__ __align__(256) float g_noalloc_scratch[NOALLOC_SCRATCH_FLOATS]
 constexpr int MAX_DEVICES = 64;
 float* g_scratch_ptr[MAX_DEVICES] = {nullptr};
 std::mutex g_setup_mutex;
-int64_t g_launches = 0;
 
 // The array's name is only a host-side handle; the kernels need its device address, which differs
 // per device.  Looked up once per device, with that device current.
@@ -47,6 +46,10 @@ extern "C" POSS_API int poss_tree_attention_noalloc(const void* q, const void* k
   if (head_dim != 32 && head_dim != 64 && head_dim != 128) return POSS_E_SHAPE;
   int g = n_q_heads / n_kv_heads;
   if (!(g == 1 || g == 2 || g == 3 || g == 4 || g == 8)) return POSS_E_SHAPE;
+  // the kernels move keys, values and outputs in 16-byte pieces
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kv) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return POSS_E_INVALID;
+  if (((size_t)kv_slots * head_dim * (dtype == POSS_BF16 ? 2 : 4)) & 15) return POSS_E_INVALID;
   if (rows == 0) return POSS_OK;
   if (rows > POSS_MAX_ROWS || prefix_len + rows > kv_slots) return POSS_E_CAPACITY;
   // the fixed scratch bounds the problem: at least one split must fit
@@ -64,7 +67,8 @@ extern "C" POSS_API int poss_tree_attention_noalloc(const void* q, const void* k
   a.n_all = prefix_len; a.n_tree = rows; a.mask = anc_mask; a.mask_words = (rows + 63) / 64; a.scale = scale;
   Launcher L;
   L.stream = reinterpret_cast<cudaStream_t>(stream);
-  L.launches = &g_launches;
+  int64_t launches = 0;                     // this call's own count: nothing is shared between callers but the scratch
+  L.launches = &launches;
   L.err = POSS_OK;
   size_t half = (size_t)n_kv_heads * kv_slots * head_dim;
   // Nothing in the scratch has to start at zero: every partial that the combine step reads was

@@ -538,9 +538,7 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   layout(*cfg, bp, c->b, &c->n_chunks, &c->n_cand_max);
   c->tc = tc_plan_cache_create();
   c->attn_tc = true;
-  if (const char* e = getenv("POSS_ATTN_TC")) c->attn_tc = atoi(e) != 0;
   c->swiglu_in_kernel = false;
-  if (const char* e = getenv("POSS_SWIGLU_IN_KERNEL")) c->swiglu_in_kernel = atoi(e) != 0;
   cudaStream_t st = S(stream);
   bool ok = cudaMemsetAsync(workspace, 0, bp.off, st) == cudaSuccess;
   double inv[64];
@@ -572,6 +570,10 @@ int poss_reset(poss_ctx* c, poss_stream stream) {
   if (cudaMemsetAsync(c->b.counters, 0, sizeof(unsigned long long) * (POSS_MAX_DEPTH + 2), S(stream)) != cudaSuccess)
     return POSS_E_CUDA;
   if (cudaMemsetAsync(c->b.status, 0, sizeof(int32_t) * 64, S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  // what a launch that gave up on a wait may have left behind: arrival counters of the matrix product's tiles
+  // and of the top-k merge's blocks (both return to zero by themselves after a launch that ran to its end)
+  if (!tc_gemm_clear_counters(c->b.tc_scratch, S(stream))) return POSS_E_CUDA;
+  if (cudaMemsetAsync(c->b.merge_done, 0, sizeof(int) * 64, S(stream)) != cudaSuccess) return POSS_E_CUDA;
   return POSS_OK;
 }
 
@@ -627,6 +629,10 @@ int poss_draft_trace(poss_ctx* c, int32_t* cand_tokens, int32_t* cand_parents, f
 int poss_tree_attention(poss_ctx* c, const void* q, const void* kv, int kv_slots, int prefix_len, int rows,
                         const uint64_t* anc_mask, float scale, void* out, poss_stream stream) {
   if (!c || !q || !kv || !anc_mask || !out || prefix_len < 0 || rows < 0 || kv_slots < 1) return POSS_E_INVALID;
+  // the kernels move keys, values and outputs in 16-byte pieces
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kv) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return POSS_E_INVALID;
+  if (((size_t)kv_slots * c->cfg.head_dim * c->esize) & 15) return POSS_E_INVALID;
   if (rows == 0) return POSS_OK;
   if (rows > R) return POSS_E_CAPACITY;
   if (prefix_len + rows > kv_slots) return POSS_E_CAPACITY;
@@ -705,6 +711,13 @@ int poss_target_forward(poss_ctx* c, void* target_kv, int prefix_len, const int3
   if (prefix_len + rows > c->cfg.target_kv_slots) return POSS_E_CAPACITY;
   return DISPATCH(c, stream, target_forward(target_kv, prefix_len, tokens, depth, anc_mask, (rows + 63) / 64, rows,
                                             out_features, out_argmax, out_logits));
+}
+
+int poss_target_verify(poss_ctx* c, void* target_kv, int prefix_len, const int32_t* tokens, const int32_t* depth,
+                       const uint64_t* anc_mask, int rows, void* out_features, int32_t* out_argmax,
+                       poss_stream stream) {
+  return poss_target_forward(c, target_kv, prefix_len, tokens, depth, anc_mask, rows, out_features, out_argmax,
+                             nullptr, stream);
 }
 
 int poss_target_prefill(poss_ctx* c, void* target_kv, int start, const int32_t* tokens, int n, void* out_features,
@@ -831,6 +844,14 @@ int poss_profile_read(poss_ctx* c, int* h_launches, float* h_total_ms) {
 int poss_debug_lose_load(poss_ctx* c, int launches) {
   if (!c || launches < 0) return POSS_E_INVALID;
   tc_inject_lost_load(c->tc, launches);
+  return POSS_OK;
+}
+
+int poss_debug_option(poss_ctx* c, int option, int value) {
+  if (!c || (value != 0 && value != 1)) return POSS_E_INVALID;
+  if (option == POSS_OPT_ATTENTION_TCGEN05) c->attn_tc = value != 0;
+  else if (option == POSS_OPT_SWIGLU_IN_KERNEL) c->swiglu_in_kernel = value != 0;
+  else return POSS_E_INVALID;
   return POSS_OK;
 }
 

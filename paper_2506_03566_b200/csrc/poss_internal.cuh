@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include "../../include/poss.h"
+#include "../../include/poss_debug.h"
 
 typedef __nv_bfloat16 bf16;
 
@@ -109,6 +110,20 @@ inline void launch_pdl(Launcher& L, void (*kernel)(KArgs...), dim3 grid, dim3 bl
   ++*L.launches;
   if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) L.err = POSS_E_CUDA;
 }
+
+// Per-device "already done" flags for set-up that CUDA keeps per device (a kernel's shared-memory opt-in, a
+// cluster shape the device refused): a process may hold contexts on several devices, so the flag is indexed
+// by the current device's ordinal.  Devices past the table share its last entry's fate of "never cached".
+struct PerDeviceFlags {
+  static constexpr int MAX_DEVICES = 64;
+  bool done[MAX_DEVICES] = {};
+  // the flag of the current device, or NULL when the ordinal cannot be had or does not fit the table
+  bool* current() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    return &done[dev];
+  }
+};
 
 // ------------------------------------------------------------------ split-K results left for the consumer
 // The tensor-core GEMM cuts the (tile, k-block) sequence of a product into one contiguous range per

@@ -18,7 +18,8 @@ Workload recipes (shapes follow the paper's experiment setup: Llama-3-8B-Instruc
 and Llama-2-13B-chat geometry, tree width 10, total tokens 60/80, depth 6/8;
 Section 4.1 "Implementations" and Appendix C of the paper):
 
-* every weight matrix, embedding and LM head ~ N(0, 0.02); norm gains = 1;
+* every weight matrix, embedding and LM head ~ N(0, 0.02); RMSNorm gains ~ 1 + N(0, 0.1)
+  (non-trivial, so that a dropped, misplaced or shifted gain shows in every comparison);
   fc bias ~ N(0, 0.02);
 * prefix KV of every specialist ~ N(0, 1); features ~ N(0, 1); token ids uniform.
 """
@@ -55,6 +56,7 @@ class PossConfig:
     prefix: int             # P: committed prefix length for drafter-only workloads
     n_target_layers: int = 0
     fc_bias: bool = True
+    norm_in: bool = True    # False: the draft layers carry no input norm (their "norm_in" is None)
 
     def replace(self, **kw) -> "PossConfig":
         return dataclasses.replace(self, **kw)
@@ -128,6 +130,14 @@ def ones(shape, dtype: str) -> np.ndarray:
     return np.full(shape, 0x3F80, dtype=np.uint16)
 
 
+def gain(seed: int, name: str, shape, dtype: str, spread: float = 0.1) -> np.ndarray:
+    """RMSNorm gain 1 + N(0, spread), same storage conventions as normal()."""
+    shape = tuple(int(s) for s in np.atleast_1d(shape))
+    g = np.random.Generator(np.random.Philox(key=_key(seed, name, 0)))
+    x = np.float32(1.0) + np.float32(spread) * g.standard_normal(shape, dtype=np.float32)
+    return x if dtype == "fp32" else _to_bf16_bits(x.ravel()).reshape(shape)
+
+
 def tokens(seed: int, name: str, count: int, vocab: int) -> np.ndarray:
     g = np.random.Generator(np.random.Philox(key=_key(seed, name, 0)))
     return g.integers(0, vocab, size=count, dtype=np.int64).astype(np.int32)
@@ -142,12 +152,12 @@ def layer_weights(cfg: PossConfig, seed: int, tag: str, with_fc: bool) -> dict:
         # columns [0,H) multiply the token embedding, [H,2H) the feature
         w["fc_w"] = normal(seed, f"{tag}.fc_w", (H, 2 * H), 0.02, dt)
         w["fc_b"] = normal(seed, f"{tag}.fc_b", (H,), 0.02, dt) if cfg.fc_bias else None
-    w["norm_in"] = ones((H,), dt)
+    w["norm_in"] = gain(seed, f"{tag}.norm_in", (H,), dt) if (cfg.norm_in or not with_fc) else None
     w["wq"] = normal(seed, f"{tag}.wq", (qd, H), 0.02, dt)
     w["wk"] = normal(seed, f"{tag}.wk", (kd, H), 0.02, dt)
     w["wv"] = normal(seed, f"{tag}.wv", (kd, H), 0.02, dt)
     w["wo"] = normal(seed, f"{tag}.wo", (H, qd), 0.02, dt)
-    w["norm_post"] = ones((H,), dt)
+    w["norm_post"] = gain(seed, f"{tag}.norm_post", (H,), dt)
     w["w_gate"] = normal(seed, f"{tag}.w_gate", (F, H), 0.02, dt)
     w["w_up"] = normal(seed, f"{tag}.w_up", (F, H), 0.02, dt)
     w["w_down"] = normal(seed, f"{tag}.w_down", (H, F), 0.02, dt)
@@ -170,7 +180,7 @@ def make_weights(cfg: PossConfig, seed: int, alias_specialists: bool = False) ->
     else:
         w["spec"] = [layer_weights(cfg, seed, f"spec{j}", True) for j in range(cfg.S)]
     w["target"] = [layer_weights(cfg, seed, f"tgt{j}", False) for j in range(cfg.n_target_layers)]
-    w["final_norm"] = ones((cfg.hidden,), cfg.dtype)
+    w["final_norm"] = gain(seed, "final_norm", (cfg.hidden,), cfg.dtype)
     return w
 
 

@@ -63,3 +63,23 @@ def test_the_attention_kernel_reports_a_wait_that_runs_out_and_the_context_stays
     again = pu.np_of(P.poss_tree_attention(qd, kvd, P_len, mask, scale))
     assert P.poss_last_status() == 0
     assert np.array_equal(again, good)
+
+
+def test_a_wait_that_runs_out_in_a_counted_product_leaves_no_stale_tile_counters():
+    """The LM head with its logits stored runs the matrix product whose split tiles are finished by the last CTA to
+    arrive (per-tile arrival counters).  A launch that gives up on a wait may leave counters behind; poss_reset
+    clears them, and the same call then reproduces its earlier result bit for bit."""
+    from paper_2506_03566_b200 import Poss, make_config, to_device
+    cfg = ps.CONFIGS["m_bf16"].replace(S=1, n_target_layers=0)
+    P = Poss(make_config(cfg.replace(topk=16, total=16, depth=2), 64), ps.make_weights(cfg, 2))
+    f = to_device(ps.normal(4, "f", (10, cfg.hidden), 1.5, "bf16"))
+    ids0, logp0, lg0 = P.poss_lm_head_topk(f, 10, want_logits=True)
+    assert P.poss_last_status() == 0
+    P.poss_debug_lose_load(1)
+    P.poss_lm_head_topk(f, 10, want_logits=True)       # results undefined; must neither fault nor hang
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 6
+    P.poss_reset()
+    ids1, logp1, lg1 = P.poss_lm_head_topk(f, 10, want_logits=True)
+    assert P.poss_last_status() == 0
+    assert torch.equal(ids0, ids1) and torch.equal(logp0, logp1) and torch.equal(lg0, lg1)

@@ -48,7 +48,8 @@ def test_full_size_draft_round_matches_oracle(name, n_new, seed):
     del P
     torch.cuda.empty_cache()
     num = pu.oracle_num(cfg, big=True)
-    rep = pu.compare_round(cfg, w, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, g, trace, num, False)
+    rep = pu.compare_round(cfg, w, kv, cfg.prefix, tok, feat, cfg.depth, cfg.topk, cfg.total, g, trace, num, False,
+                           noise_num=po.Num(np.float64, "bf16"))
     pu.compare_kv(cfg, dkv, rep["kv_oracle"], cfg.prefix, cfg.prefix + n_new, pu.TOL[cfg.dtype])
     print(name, {k: v for k, v in rep.items() if k != "kv_oracle"})
     assert int(g["n_nodes"][0]) == cfg.total + 1
@@ -67,7 +68,7 @@ def test_full_size_verification_attention_matches_oracle(rows, P_len):
     scale = 1.0 / math.sqrt(d)
     got = pu.np_of(P.poss_tree_attention(_dev(q), _dev(kv), P_len, torch.from_numpy(mask.view(np.int64)).cuda(), scale))
     want = po.tree_attention(q, kv, P_len, parents, scale, pu.oracle_num(cfg))
-    assert np.abs(got - want).max() <= 2e-2
+    pu.check_attention(got, want, "bf16", f"{rows}x{P_len}")
     # a node's output does not change when a non-ancestor's key/value changes
     r = rows - 1
     other = next(j for j in range(1, rows) if not po.ancestor_matrix(parents)[r, j])
@@ -154,7 +155,82 @@ def test_full_size_verify_sample_over_the_whole_vocabulary():
     print("verify_sample 61 x 128256, depths", depths, "bonus equal to the oracle's in", exact, "of 12, us per call", round(e0.elapsed_time(e1) * 50, 1))
 
 
-def test_c5_full_loop_matches_plain_greedy_decode():
+@pytest.fixture(scope="module")
+def c5_weights():
+    """The 32-layer target + six specialists of config c5 (about 17 GB of bf16 on the host), drawn once."""
+    return ps.make_weights(ps.CONFIGS["c5"], 105)
+
+
+def test_c5_target_tree_pass_matches_oracle(c5_weights):
+    """The verification pass at its full size, element by element: 61 tree rows through the 32-layer
+    Llama-3-8B-shaped target behind a 512-slot prefix (prefix keys/values ~ N(0,1) as in the drafter workloads, the
+    same bits on both sides), against the oracle in fp32 arithmetic under the bf16 contract.  Through 32 layers two
+    correct bf16 implementations drift apart by flipped roundings, so the bound is measured in the same test: the
+    oracle is run a second time in fp64 arithmetic and the CUDA path must be as close to the fp32 oracle as that
+    (maximum and RMS of the difference within 3 x the oracle-to-oracle distance, never below the 2e-2 of the one-layer
+    cases).  The greedy tokens must be the oracle's wherever its top-two margin exceeds the same bound."""
+    from paper_2506_03566_b200 import Poss, make_config
+    cfg, w = ps.CONFIGS["c5"], c5_weights
+    rows, P_len = cfg.total + 1, cfg.prefix
+    slots = P_len + rows + 3
+    kv_bits = np.zeros((cfg.n_target_layers, 2, cfg.n_kv_heads, slots, cfg.head_dim), dtype=np.uint16)
+    kv_bits[:, :, :, :P_len] = ps.normal(106, "target_kv", (cfg.n_target_layers, 2, cfg.n_kv_heads, P_len, cfg.head_dim),
+                                        1.0, "bf16")
+    parents = ps.random_tree_parents(107, rows, max_children=10)
+    depth = np.zeros(rows, dtype=np.int32)
+    for r in range(1, rows):
+        depth[r] = depth[parents[r]] + 1
+    toks = ps.tokens(108, "tree_tokens", rows, cfg.vocab)
+    mask = po.pack_mask(po.ancestor_matrix(parents))
+
+    P = Poss(make_config(cfg, 64 + cfg.tree_slots, slots), w)
+    tkv = _dev(kv_bits)
+    tf, targ, tl = P.poss_target_forward(tkv, P_len, torch.from_numpy(toks).cuda(), torch.from_numpy(depth).cuda(),
+                                         torch.from_numpy(mask.view(np.int64)).cuda(), rows, want_logits=True)
+    # the production form of the same pass (fused argmax epilogue, no logits stored) must pick the same tokens
+    tf2, targ2 = P.poss_target_verify(tkv, P_len, torch.from_numpy(toks).cuda(), torch.from_numpy(depth).cuda(),
+                                      torch.from_numpy(mask.view(np.int64)).cuda(), rows)
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 0
+    got_f, got_arg, got_l = pu.np_of(tf), targ.cpu().numpy(), tl.cpu().numpy()
+    assert np.array_equal(pu.np_of(tf2), got_f) and np.array_equal(targ2.cpu().numpy(), got_arg)
+    P.close()
+    del P, tkv
+    torch.cuda.empty_cache()
+
+    outs = {}
+    for name, num in (("fp32", po.Num(np.float32, "bf16")), ("fp64", po.Num(np.float64, "bf16"))):
+        kv_o = po.widen(kv_bits, num.dtype).copy()
+        outs[name] = po.target_forward(cfg, w, kv_o, P_len, toks, P_len + depth, parents, num)
+    f_o, l_o = outs["fp32"]
+    f_n, l_n = outs["fp64"]
+
+    def dist(a, b):
+        d = np.abs(np.asarray(a, dtype=np.float64) - np.asarray(b, dtype=np.float64))
+        return float(d.max()), float(np.sqrt(np.mean(d * d)))
+
+    report = {}
+    for what, got, want, other in (("features", got_f, f_o, f_n), ("logits", got_l, l_o, l_n)):
+        e_max, e_rms = dist(got, want)
+        n_max, n_rms = dist(other, want)
+        rms = float(np.sqrt(np.mean(np.square(np.asarray(want, dtype=np.float64)))))
+        report[what] = {"rms": round(rms, 3), "err_max": round(e_max, 4), "err_rms": round(e_rms, 5),
+                        "oracle_noise_max": round(n_max, 4), "oracle_noise_rms": round(n_rms, 5)}
+        assert e_max <= max(2e-2, 3.0 * n_max), (what, report)
+        assert e_rms <= max(2e-3, 3.0 * n_rms), (what, report)
+    bound = max(pu.MARGIN, 3.0 * report["logits"]["oracle_noise_max"])
+    want_arg = po.argmax_rows(l_o)
+    differ = 0
+    for r in range(rows):
+        if got_arg[r] != want_arg[r]:
+            differ += 1
+            srt = np.sort(l_o[r])[::-1]
+            assert srt[0] - srt[1] < bound, f"row {r}: greedy token differs at a margin of {srt[0] - srt[1]}"
+    report["argmax_rows_differing_at_a_near_tie"] = differ
+    print("c5 target pass, 61 rows x 32 layers:", report)
+
+
+def test_c5_full_loop_matches_plain_greedy_decode(c5_weights):
     """Config c5: 32-layer Llama-3-8B-shaped target + the c2 drafter, prompt of 512 ids, 512 generated tokens.
     Every round = draft tree (depth 6, top-k 10, 60 tokens) + tree-masked target pass + accept walk + KV
     compaction.  The speculative stream must equal the plain greedy decode of the same target token for
@@ -166,7 +242,7 @@ def test_c5_full_loop_matches_plain_greedy_decode():
     the oracle on a short prompt."""
     from paper_2506_03566_b200 import Poss, make_config, speculative_generate, plain_generate
     cfg = ps.CONFIGS["c5"]
-    w = ps.make_weights(cfg, 105)
+    w = c5_weights
     n_prompt, n_gen = cfg.prefix, 512
     slots = n_prompt + n_gen + cfg.total + cfg.depth + 4
     P = Poss(make_config(cfg, slots + cfg.tree_slots, slots), w)
@@ -175,18 +251,27 @@ def test_c5_full_loop_matches_plain_greedy_decode():
 
     # the plain decode against the oracle's definition, on a short prompt (a full-length one is minutes of CPU)
     short = prompt[:6]
-    got = plain_generate(P, torch.from_numpy(short).cuda(), 4)
-    kv_o = po.new_target_kv(cfg, 16, num)
+    n_pin = 16
+    got = plain_generate(P, torch.from_numpy(short).cuda(), n_pin)
+    kv_o = po.new_target_kv(cfg, 6 + n_pin + 1, num)
     stream = list(short)
-    for k in range(4):
+    for k in range(n_pin):
         n = len(stream)
         if k == 0:
             _, lg = po.target_forward(cfg, w, kv_o, 0, np.array(stream, dtype=np.int32), np.arange(n), po.chain_parents(n), num)
         else:
             _, lg = po.target_forward(cfg, w, kv_o, n - 1, [stream[-1]], [n - 1], po.chain_parents(1), num)
-        srt = np.sort(lg[-1])[::-1]
         want = int(po.argmax_rows(lg[-1:])[0])
-        assert got[k] == want or srt[0] - srt[1] < pu.MARGIN, f"plain decode differs from the oracle at token {k}"
+        if got[k] != want:
+            # explained only by a near-tie: the gap must be below the margin, or below 3 x the distance between the
+            # oracle's own fp32 and fp64 evaluations of this very position (32 layers of flipped bf16 roundings)
+            num64 = po.Num(np.float64, "bf16")
+            kv64 = po.new_target_kv(cfg, n + 1, num64)
+            _, lg64 = po.target_forward(cfg, w, kv64, 0, np.array(stream, dtype=np.int32), np.arange(n), po.chain_parents(n), num64)
+            noise = float(np.abs(lg64[-1] - lg[-1]).max())
+            gap = float(lg[-1][want] - lg[-1][got[k]])
+            print(f"plain decode token {k}: GPU {got[k]}, oracle {want}, gap {gap:.4f}, oracle fp32/fp64 distance {noise:.4f}")
+            assert gap < max(pu.MARGIN, 3.0 * noise), f"plain decode differs from the oracle at token {k}"
         stream.append(int(got[k]))
 
     cur = prompt
@@ -220,11 +305,9 @@ def test_c5_full_loop_matches_plain_greedy_decode():
             gap = abs(float(lg[-1][spec[i]]) - float(lg[-1][plain[i]]))
             rms = float(np.sqrt(np.mean(np.square(lg[-1]))))
             where = "oracle logits"
-        # Two bf16 paths through L layers differ by about one rounding (2^-9 relative) at each of the ~4 rounding
-        # points of a layer, adding up like a random walk: 2^-9 * sqrt(4 L) of the logits' RMS (2.2 % at L = 32).
-        # A parting is explained when the gap is within twice that, and never needs to be below the 1e-2 of the
-        # shallow cases.
-        bound = max(pu.MARGIN, 2.0 * 2.0 ** -9 * math.sqrt(4.0 * cfg.n_target_layers) * rms)
+        # The tree pass and the single-row decode sum a token's attention in the same grouping, so the streams are
+        # expected not to part at all; a parting is tolerated only at a near-tie under the margin of every other test.
+        bound = pu.MARGIN
         assert gap < bound, f"streams part at generated token {n_gen - left + i} without a near-tie ({gap} >= {bound} in the {where})"
         partings.append((n_gen - left + i, round(gap, 5), round(rms, 2), where))
         cur = np.concatenate([common, np.array([plain[i]], dtype=np.int32)])

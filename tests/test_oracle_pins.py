@@ -42,7 +42,11 @@ def hf_model(cfg, w, layers):
         sd[p + "mlp.gate_proj.weight"] = _t(l["w_gate"])
         sd[p + "mlp.up_proj.weight"] = _t(l["w_up"])
         sd[p + "mlp.down_proj.weight"] = _t(l["w_down"])
-        sd[p + "input_layernorm.weight"] = _t(l["norm_in"])
+        if l["norm_in"] is None:
+            # a layer without an input norm: the library layer with that module taken out
+            m.model.layers[i].input_layernorm = torch.nn.Identity()
+        else:
+            sd[p + "input_layernorm.weight"] = _t(l["norm_in"])
         sd[p + "post_attention_layernorm.weight"] = _t(l["norm_post"])
     missing = m.load_state_dict(sd, strict=False)
     assert not missing.missing_keys and not missing.unexpected_keys
@@ -272,6 +276,49 @@ def test_chain_draft_equals_eq9_with_library_layers(S, n):
     assert list(res.parents) == [-1, 0, 1, 2, 3, 4]
     assert np.abs(res.scores[1:] - np.cumsum(want_logp)).max() < 1e-6
     assert list(res.depth) == [0, 1, 2, 3, 4, 5]
+
+
+def test_synthetic_gains_are_not_trivial():
+    """Every RMSNorm gain of the synthetic recipe differs from 1 (fp32 and bf16 storage alike), element by
+    element differently, so that the pins below and every GPU comparison see the gain path."""
+    for name in ("t_fp32", "t_bf16"):
+        cfg = ps.CONFIGS[name]
+        w = ps.make_weights(cfg, 2)
+        gains = [w["final_norm"]] + [l[k] for l in w["spec"] + w["target"] for k in ("norm_in", "norm_post")]
+        for g in gains:
+            g = po.widen(g, np.float64)
+            assert g.shape == (cfg.hidden,)
+            assert 0.05 < g.std() < 0.2 and abs(g.mean() - 1.0) < 0.05
+            assert np.abs(g - np.roll(g, 1)).mean() > 0.05        # a gain read one column off is a different gain
+    assert not np.array_equal(w["spec"][0]["norm_in"], w["spec"][1]["norm_in"])
+    assert not np.array_equal(w["spec"][0]["norm_in"], w["spec"][0]["norm_post"])
+
+
+def test_rmsnorm_matches_torch_rms_norm_with_a_gain():
+    g = np.random.default_rng(7)
+    x = g.standard_normal((5, 48)) * 3.0
+    gn = 1.0 + 0.3 * g.standard_normal(48)
+    want = torch.nn.functional.rms_norm(torch.from_numpy(x), (48,), torch.from_numpy(gn), 1e-5).numpy()
+    assert np.abs(po.rmsnorm(x, gn, 1e-5, NUM) - want).max() < 1e-12
+    assert po.rmsnorm(x, None, 1e-5, NUM) is x                    # no norm at all, not a norm with gain 1
+
+
+@pytest.mark.parametrize("S,n", [(3, 2), (1, 5)])
+def test_chain_draft_without_input_norm_equals_the_library_layer_without_it(S, n):
+    """Draft layers with norm_in absent: the attention reads fc's output as it is (no normalisation, no gain);
+    the library layer with its input_layernorm module removed is the definition."""
+    cfg = ps.CONFIGS["t_fp32"].replace(S=S, n=n, depth=5, topk=1, total=5, norm_in=False)
+    w = ps.make_weights(cfg, 5)
+    assert all(l["norm_in"] is None for l in w["spec"]) and all(l["norm_in"] is not None for l in w["target"])
+    toks, feats = ps.make_round_inputs(cfg, 5, n_new=4)
+    res = po.draft_round(cfg, w, fresh_draft_kv(cfg, 5, 4, prefix=0), 0, toks, feats, 5, 1, 5, NUM)
+    want_tok, want_logp = drafter_chain_by_library(cfg, w, toks, feats, 5)
+    assert list(res.tokens[1:]) == want_tok
+    assert np.abs(res.scores[1:] - np.cumsum(want_logp)).max() < 1e-6
+    # and it is a different function from the normed layer
+    w2 = ps.make_weights(cfg.replace(norm_in=True), 5)
+    res2 = po.draft_round(cfg, w2, fresh_draft_kv(cfg, 5, 4, prefix=0), 0, toks, feats, 5, 1, 5, NUM)
+    assert np.abs(res2.scores[1:] - res.scores[1:]).max() > 1e-4
 
 
 def test_prefix_cache_equals_recomputing_the_prefix():
@@ -656,3 +703,43 @@ def test_pins_catch_a_wrong_specialist_schedule(monkeypatch):
     monkeypatch.setattr(po, "specialist_for_position", lambda i, n, S: max(1, min(math.ceil(i / n), S)))
     res = po.draft_round(cfg, w, fresh_draft_kv(cfg, 5, 4, prefix=0), 0, toks, feats, 5, 1, 5, NUM)
     assert np.abs(res.scores[1:] - np.cumsum(want_logp)).max() > 1e-6
+
+
+@pytest.mark.parametrize("mistake", ["dropped", "before_the_normalisation", "shifted", "none_means_unit_gain_norm"])
+def test_pins_catch_a_wrong_rmsnorm_gain(monkeypatch, mistake):
+    """The library pins must go red for a norm that drops its gain, applies it on the wrong side of the
+    normalisation, reads it one column off, or treats an absent norm as a norm with gain 1."""
+    def wrong(x, g, eps, num):
+        x = np.asarray(x, dtype=num.dtype)
+        if g is None:
+            if mistake == "none_means_unit_gain_norm":
+                return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+            return x
+        gw = num.w(g)
+        if mistake == "dropped":
+            return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+        if mistake == "before_the_normalisation":
+            y = x * gw
+            return y / np.sqrt(np.mean(y * y, axis=-1, keepdims=True) + eps)
+        if mistake == "shifted":
+            return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps) * np.roll(gw, 1)
+        return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps) * gw
+    monkeypatch.setattr(po, "rmsnorm", wrong)
+    if mistake == "none_means_unit_gain_norm":
+        cfg = ps.CONFIGS["t_fp32"].replace(S=3, n=2, depth=5, topk=1, total=5, norm_in=False)
+        w = ps.make_weights(cfg, 5)
+        toks, feats = ps.make_round_inputs(cfg, 5, n_new=4)
+        want_tok, want_logp = drafter_chain_by_library(cfg, w, toks, feats, 5)
+        res = po.draft_round(cfg, w, fresh_draft_kv(cfg, 5, 4, prefix=0), 0, toks, feats, 5, 1, 5, NUM)
+        assert np.abs(res.scores[1:] - np.cumsum(want_logp)).max() > 1e-4
+        return
+    cfg = ps.CONFIGS["t_fp32"]
+    w = ps.make_weights(cfg, 2)
+    m = hf_model(cfg, w, w["target"])
+    prompt = ps.make_prompt(cfg, 2, 23)
+    with torch.no_grad():
+        out = m(torch.from_numpy(prompt.astype(np.int64))[None], output_hidden_states=True)
+    kv = po.new_target_kv(cfg, 64, NUM)
+    feat, logits = po.target_forward(cfg, w, kv, 0, prompt, np.arange(23), po.chain_parents(23), NUM)
+    assert np.abs(out.logits[0].numpy() - logits).max() > 1e-3
+    assert np.abs(out.hidden_states[-1][0].numpy() - feat).max() > 1e-3
