@@ -26,6 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "poss_draft_round_us_60tok_depth6"
+# DRAM bytes (read + written) of one LM-head launch of k_gemm_tc at the Llama-3-8B shape, from the ncu capture whose
+# summary is the named file (None once the kernel has changed since the capture)
+TRAFFIC = {"bytes": None, "workloads": ("c2", "c4", "c5"),
+           "source": "profiles/k_gemm_tc_c2_m10_gateup_down_lmhead.md, third captured launch (-s 9 -c 3: the LM head)"}
 
 
 def algorithmic_bytes(cfg):
@@ -101,6 +105,38 @@ def rounds_per_second(world: int, ms_per_step: float) -> float:
     return world * 1e3 / ms_per_step
 
 
+def workload_name(cfg) -> str:
+    """The drafter workload, worded identically by both arms."""
+    shape = "Llama-3-8B" if cfg.hidden == 4096 else "Llama-2-13B" if cfg.hidden == 5120 else "test"
+    return (f"{cfg.name}: drafter H={cfg.hidden} F={cfg.ffn} V={cfg.vocab} ({shape}-shaped), {cfg.S} specialists x {cfg.n} "
+            f"positions, depth {cfg.depth}, top-k {cfg.topk}, {cfg.total} tokens, prefix {cfg.prefix}")
+
+
+def chain_spans(records):
+    """Timeline records [(kernel name, ns)] in time order -> {phase: {kernel: [launches, summed span in us]}}.
+    A record is the instant a launch's wait for its predecessor returned; the span of a launch inside the chain is
+    the time to the next record.  Phases: a draft round runs from its first gather_x to its rerank, a target pass
+    from embed_rows to the accept walk; the last record of a phase has no successor inside it and is left out."""
+    out = {"draft": {}, "target": {}}
+    phase = None
+    for i, (name, t) in enumerate(records):
+        if name == "gather_x" and phase != "draft":
+            phase = "draft"
+        elif name == "embed_rows":
+            phase = "target"
+        if phase is None or i + 1 >= len(records):
+            continue
+        nxt_name, nxt_t = records[i + 1]
+        ends = (phase == "draft" and name == "rerank") or (phase == "target" and name == "accept_walk")
+        if not ends:
+            cell = out[phase].setdefault(name, [0, 0.0])
+            cell[0] += 1
+            cell[1] += (nxt_t - t) / 1e3
+        if ends:
+            phase = None
+    return out
+
+
 def run_reference(args, cfg):
     """The oracle, as it stands, on the host cores: one full draft round per step."""
     import poss_synth as ps
@@ -126,8 +162,7 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: drafter H={cfg.hidden} F={cfg.ffn} V={cfg.vocab}, {cfg.S} specialists x {cfg.n} "
-                                   f"positions, depth {cfg.depth}, top-k {cfg.topk}, {cfg.total} tokens, prefix {cfg.prefix}"},
+            "config": {"workload": workload_name(cfg), "step": "one draft round (the metric's quantity)"},
             "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
                              "sample": "one full draft round (numpy fp32, bf16 rounding contract); verify stages not included"},
             "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -202,11 +237,13 @@ def main():
         def dev_normal(*shape, std=0.02):
             return (torch.randn(*shape, device="cuda", generator=gen) * std).to(torch.bfloat16)
 
-        ones = torch.ones(H, device="cuda", dtype=torch.bfloat16)
-        w["target"] = [{"norm_in": ones, "wq": dev_normal(qd, H), "wk": dev_normal(kd, H), "wv": dev_normal(kd, H),
-                        "wo": dev_normal(H, qd), "norm_post": ones, "w_gate": dev_normal(F, H),
+        def dev_gain():
+            return (1.0 + 0.1 * torch.randn(H, device="cuda", generator=gen)).to(torch.bfloat16)
+
+        w["target"] = [{"norm_in": dev_gain(), "wq": dev_normal(qd, H), "wk": dev_normal(kd, H), "wv": dev_normal(kd, H),
+                        "wo": dev_normal(H, qd), "norm_post": dev_gain(), "w_gate": dev_normal(F, H),
                         "w_up": dev_normal(F, H), "w_down": dev_normal(H, F)} for _ in range(n_layers)]
-        w["final_norm"] = ones
+        w["final_norm"] = dev_gain()
     P = Poss(make_config(cfg.replace(n_target_layers=n_layers), cap, tcap), w)
     dkv = to_device(ps.make_draft_kv(cfg, seed, cap))
     tok_h, feat_h = ps.make_round_inputs(cfg, seed, 1)
@@ -314,6 +351,16 @@ def main():
     P.poss_profile(0)
     sync_all()
 
+    # the same stages INSIDE the chain of dependent launches: every launch records the device time at which its wait
+    # for its predecessor returned; a launch's span is the time to the next record (overlap included, nothing cut)
+    P.poss_profile(3)
+    n_chain = min(args.steps, 10)
+    for _ in range(n_chain):
+        step(tok_d, feat_d)
+    chain = chain_spans(P.poss_timeline_read())
+    P.poss_profile(0)
+    sync_all()
+
     # ---------------- timed region 2: end to end through the C ABI with host buffers (host-timed)
     # (a) the metric's own quantity: pinned-host inputs -> device, draft round, tree back to pinned host
     res_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
@@ -362,12 +409,10 @@ def main():
             "metric": METRIC, "value": draft_ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: drafter H={cfg.hidden} F={cfg.ffn} V={cfg.vocab} "
-                                   f"({'Llama-3-8B' if cfg.hidden == 4096 else 'Llama-2-13B' if cfg.hidden == 5120 else 'test'}-shaped), "
-                                   f"{cfg.S} specialists x {cfg.n} positions, depth {cfg.depth}, top-k {cfg.topk}, "
-                                   f"{cfg.total} tokens, prefix {cfg.prefix}; step = draft round + " +
-                                   (f"61-row tree-masked pass of a {n_layers}-layer Llama-3-8B-shaped target + accept walk + KV compaction"
-                                    if with_target else "61-row verification attention + logits argmax + accept walk"),
+            "config": {"workload": workload_name(cfg),
+                       "step": "draft round (the metric's quantity) + " +
+                               (f"{rows}-row tree-masked pass of a {n_layers}-layer target of the same shape + accept walk + KV compaction"
+                                if with_target else f"{rows}-row verification attention + logits argmax + accept walk"),
                        "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "stages_us": {"draft_round": draft_ms * 1e3, "whole_step": ms * 1e3,
@@ -386,7 +431,8 @@ def main():
                          "frac": achieved / hbm_peak if achieved else None,
                          # dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch, from the ncu capture
                          # summarised in profiles/k_gemm_tc_c2_m10_gateup_down_lmhead.md (c2 shapes only)
-                         "traffic": 1050838000 + 8038144 if cfg.name in ("c2", "c4", "c5") else None,
+                         "traffic": TRAFFIC["bytes"] if cfg.name in TRAFFIC["workloads"] else None,
+                         "traffic_source": TRAFFIC["source"] if cfg.name in TRAFFIC["workloads"] else None,
                          "launches_timed": n_lm, "avg_launch_us": lm_dur * 1e3,
                          "algorithmic_bytes_per_launch": lm_bytes},
         }
@@ -399,8 +445,27 @@ def main():
             k: {"launches": n, "avg_us": t / n * 1e3, "algorithmic_bytes": kind_bytes[k],
                 "gbs": kind_bytes[k] / (t / n * 1e-3) / 1e9, "frac_of_hbm_peak": kind_bytes[k] / (t / n * 1e-3) / 1e9 / hbm_peak}
             for k, (n, t) in per_kind.items() if n}
-        line["kernels_note"] = ("each stage of the draft steps between two CUDA events of its own (isolated: no overlap with its "
-                                "neighbours); gate_up includes the SwiGLU, attention its combine kernel; bytes = weights (or K/V) only")
+        # in-chain spans of the same stages (a product's span is its GEMM launch; gate_up adds the SwiGLU consumer)
+        d = chain["draft"]
+        span = lambda *names: sum(d[n][1] for n in names if n in d) / max(max((d[n][0] for n in names if n in d), default=1), 1)
+        chain_kind = {"fc": ("gemm_fc",), "qkv": ("gemm_qkv",), "attention": ("attn_tc", "attn_mma", "attn_combine_bf16"),
+                      "o": ("gemm_o",), "gate_up": ("gemm_gate_up", "splitk_swiglu"), "down": ("gemm_down",),
+                      "lm_head": ("gemm_lm_head",)}
+        for k, names in chain_kind.items():
+            if k in line["kernels"] and any(n in d for n in names):
+                us = span(*names)
+                line["kernels"][k]["in_chain_us"] = us
+                line["kernels"][k]["in_chain_frac_of_hbm_peak"] = kind_bytes[k] / (us * 1e-6) / 1e9 / hbm_peak
+        line["chain_us_per_launch"] = {ph: {n: round(c[1] / c[0], 2) for n, c in sorted(v.items())} for ph, v in chain.items()}
+        if with_target and chain["target"]:
+            t = chain["target"]
+            per_layer = ("gemm_qkv", "rope_append", "attn_tc", "attn_mma", "attn_combine_bf16", "gemm_o", "reduce_norm",
+                         "gemm_gate_up", "splitk_swiglu", "gemm_down")
+            line["target_layer_in_chain_us"] = sum(t[n][1] for n in per_layer if n in t) / (n_chain * n_layers)
+        line["kernels_note"] = ("avg_us: each stage of the draft steps between two CUDA events of its own (isolated: no overlap "
+                                "with its neighbours); in_chain_us: the same stage inside the chain of dependent launches, from "
+                                "device timestamps taken when each launch's wait for its predecessor returns (span to the next "
+                                "launch's); gate_up includes the SwiGLU, attention its combine kernel; bytes = weights (or K/V) only")
         if not args.no_cpu_baseline and world == 1:
             from oracle import poss_oracle as po
             wr = ps.make_weights(cfg, seed)

@@ -24,7 +24,8 @@ extern "C" {
 POSS_API int poss_draft_trace(poss_ctx* ctx, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores,
                      int32_t* frontier, float* step_features, int32_t* selected, poss_stream stream);
 
-/* Device-time bracketing of the draft steps' stages, for roofline reporting.  mode 0: off; mode 1: the LM-head
+/* Device-time bracketing of the draft steps' stages, for roofline reporting.  mode 0: off (also switches the timeline
+ * recording below off); mode 1: the LM-head
  * matrix product (the dominant kernel) of every draft step sits between two CUDA events on the launching stream;
  * mode 2: so does every stage kind below (the launches between the two events are the product's kernel, plus the
  * combine kernel for POSS_PROF_ATTENTION and the in-kernel or consumer-side SwiGLU for POSS_PROF_GATE_UP).  The
@@ -36,6 +37,26 @@ enum { POSS_PROF_FC = 0, POSS_PROF_QKV = 1, POSS_PROF_ATTENTION = 2, POSS_PROF_O
        POSS_PROF_DOWN = 5, POSS_PROF_LM_HEAD = 6, POSS_PROF_KINDS = 7 };
 POSS_API int poss_profile(poss_ctx* ctx, int mode);
 POSS_API int poss_profile_read(poss_ctx* ctx, int* h_launches, float* h_total_ms);
+
+/* Timeline of the chain of dependent launches (poss_profile mode 3).  Every launch of the library on the current
+ * device -- draft steps and target pass alike -- records which kernel it is and the device time (ns, the GPU's global
+ * timer) at which its wait for its predecessor returned, i.e. at which the predecessor grid had completed.  The
+ * difference between two consecutive records is the earlier kernel's span INSIDE the chain, overlap with its
+ * neighbours included (mode 2 cuts that overlap).  Recording adds one store per launch and leaves the chain as it is.
+ * It is a property of the device, not of the context: switch it on for one context at a time; poss_profile(ctx, 0)
+ * switches it off.  poss_timeline_read SYNCHRONISES the stream, copies up to `capacity` records in launch order
+ * (h_kernel[i] a POSS_K_* value, h_time_ns[i]) to the host, stores their number in *h_count and starts over; at most
+ * 8192 records are kept between reads.  A matrix product's id tells which product it is. */
+enum { POSS_K_OTHER = 0, POSS_K_GATHER_X = 1, POSS_K_EMBED_ROWS = 2, POSS_K_RMSNORM = 3, POSS_K_REDUCE_NORM = 4,
+       POSS_K_ROPE_APPEND = 5, POSS_K_ATTN_TC = 6, POSS_K_ATTN_MMA = 7, POSS_K_ATTN_COMBINE_BF16 = 8,
+       POSS_K_ATTN_PARTIAL = 9, POSS_K_ATTN_COMBINE = 10, POSS_K_SPLITK_REDUCE = 11, POSS_K_SPLITK_SWIGLU = 12,
+       POSS_K_SILU_MUL = 13, POSS_K_CAST = 14, POSS_K_GEMM_SIMT = 15, POSS_K_TOPK_PARTIAL = 16, POSS_K_TOPK_MERGE =
+       17, POSS_K_TOPK_MERGE_EXPAND = 18, POSS_K_ARGMAX_PARTIAL = 19, POSS_K_RERANK = 20, POSS_K_ACCEPT_WALK = 21,
+       POSS_K_SAMPLE_WALK = 22, POSS_K_KV_COMPACT = 23, POSS_K_CHAIN_MASK = 24, POSS_K_TILE_CONTRIB = 25,
+       POSS_K_GEMM_FC = 32, POSS_K_GEMM_QKV = 33, POSS_K_GEMM_O = 34, POSS_K_GEMM_GATE_UP = 35, POSS_K_GEMM_DOWN =
+       36,        POSS_K_GEMM_LM_HEAD = 37, POSS_K_GEMM_OTHER = 38, POSS_K_COUNT = 39 };
+POSS_API int poss_timeline_read(poss_ctx* ctx, int capacity, int32_t* h_kernel, int64_t* h_time_ns, int* h_count,
+                       poss_stream stream);
 
 /* Failure-detection test hook (the paper has no counterpart).  The next `launches` tensor-core launches of this
  * context (matrix products and tcgen05 tree attention alike) withhold one tile from their own pipeline (a product:

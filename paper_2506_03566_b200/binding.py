@@ -18,6 +18,13 @@ POSS_FP32, POSS_BF16 = 0, 1
 POSS_MAX_ROWS, POSS_MAX_TOPK, POSS_MAX_DEPTH = 128, 16, 16
 PROF_KINDS = ("fc", "qkv", "attention", "o", "gate_up", "down", "lm_head")
 POSS_OPT_ATTENTION_TCGEN05, POSS_OPT_SWIGLU_IN_KERNEL = 0, 1
+KERNEL_NAMES = {0: "other", 1: "gather_x", 2: "embed_rows", 3: "rmsnorm", 4: "reduce_norm", 5: "rope_append",
+                6: "attn_tc", 7: "attn_mma", 8: "attn_combine_bf16", 9: "attn_partial", 10: "attn_combine",
+                11: "splitk_reduce", 12: "splitk_swiglu", 13: "silu_mul", 14: "cast", 15: "gemm_simt",
+                16: "topk_partial", 17: "topk_merge", 18: "topk_merge_expand", 19: "argmax_partial", 20: "rerank",
+                21: "accept_walk", 22: "sample_walk", 23: "kv_compact", 24: "chain_mask", 25: "tile_contrib",
+                32: "gemm_fc", 33: "gemm_qkv", 34: "gemm_o", 35: "gemm_gate_up", 36: "gemm_down", 37: "gemm_lm_head",
+                38: "gemm_other"}
 STATUS = {0: "POSS_OK", 1: "POSS_E_INVALID", 2: "POSS_E_SHAPE", 3: "POSS_E_CAPACITY", 4: "POSS_E_WORKSPACE",
           5: "POSS_E_CUDA", 6: "POSS_E_TIMEOUT"}
 
@@ -77,6 +84,8 @@ EXPORTS = {
                                     C.c_void_p]),
     "poss_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "poss_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_float)]),
+    "poss_timeline_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int64),
+                                     C.POINTER(C.c_int), C.c_void_p]),
     "poss_attention_plan": (C.c_int, [C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "poss_launch_count": (C.c_int64, [C.c_void_p]),
     "poss_debug_lose_load": (C.c_int, [C.c_void_p, C.c_int]),
@@ -348,6 +357,15 @@ class Poss:
         ms = (C.c_float * len(PROF_KINDS))()
         _check(self.lib.poss_profile_read(self.ctx, n, ms), "poss_profile_read")
         return {k: (int(n[i]), float(ms[i])) for i, k in enumerate(PROF_KINDS)}
+
+    def poss_timeline_read(self, capacity: int = 8192):
+        """-> list of (kernel name, device time in ns) in time order (poss_profile mode 3)."""
+        k = (C.c_int32 * capacity)()
+        t = (C.c_int64 * capacity)()
+        n = C.c_int()
+        _check(self.lib.poss_timeline_read(self.ctx, capacity, k, t, C.byref(n), _stream()), "poss_timeline_read")
+        rec = sorted(((int(t[i]), int(k[i])) for i in range(n.value)))
+        return [(KERNEL_NAMES.get(kk, str(kk)), tt) for tt, kk in rec]
 
     def poss_debug_lose_load(self, launches: int):
         _check(self.lib.poss_debug_lose_load(self.ctx, int(launches)), "poss_debug_lose_load")

@@ -33,6 +33,8 @@
 #include "tc_ptx.cuh"
 #include <string.h>
 
+POSS_TRACE_REGISTER()
+
 namespace {
 
 using namespace tcptx;
@@ -186,7 +188,7 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   // The successor may start only now that this CTA holds its TMEM columns: a successor's CTA that took
   // columns on this SM first would keep them until this grid has finished, which then could not happen.
   pdl_begin();
-  pdl_sync();
+  pdl_sync(POSS_K_ATTN_TC);
 
   if (threadIdx.x == 0) {
     // ---------------- the copies and the first product

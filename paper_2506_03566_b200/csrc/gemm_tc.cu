@@ -42,6 +42,8 @@
 #include <stdlib.h>
 #include <math.h>
 
+POSS_TRACE_REGISTER()
+
 #define LAUNCH_CHECK(L)                                         \
   do {                                                          \
     ++*(L).launches;                                            \
@@ -66,6 +68,7 @@ struct TcArgs {
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
   int n_tiles, kb_total, gran, slots, pair_tiles;
   int inject_lost_load;   // test hook: the producer leaves out the activation tile of its first stage
+  int trace_tag;          // kernel id for the timeline recording (POSS_K_GEMM_*)
   const bf16* bias;
   const float* residual;
   int ldr;
@@ -195,7 +198,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         load_w(cw, it);
         advance(cw);
       }
-      pdl_sync();
+      pdl_sync(a.trace_tag);
       for (int it = 0; it < pre; ++it) { if (!(a.inject_lost_load && it == 0)) load_x(cx, it); advance(cx); }
       int issued = pre, s = 0;
       uint32_t phase = 0;                     // parity of the "empty" completion that frees stage s next
@@ -249,7 +252,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     }
   } else {
     // ---------------- epilogue warps: TMEM lane = weight row
-    pdl_sync();
+    pdl_sync(-1);
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int t = q * 32 + lane;                  // row inside the tile
     const int K = a.topk;
@@ -780,6 +783,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (stages < 2) stages = 2;
   a.n_stages = stages;
   a.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
+  a.trace_tag = ep.trace_tag;
   a.bias = ep.bias; a.residual = ep.residual; a.ldr = ep.ldr; a.out = ep.out; a.ldo = ep.ldo;
   a.out_bf = ep.out_bf; a.ldo_bf = ep.ldo_bf;
   a.scratch = reinterpret_cast<float*>(scratch);

@@ -58,6 +58,7 @@ struct TcEpilogue {
   int32_t* pidx = nullptr;
   int* n_lists = nullptr;
   SplitKView* view = nullptr;
+  int trace_tag = POSS_K_GEMM_OTHER;   // which product this is, for the timeline recording
 };
 
 void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx, int M, const GemmSegs& segs, int K,

@@ -9,6 +9,8 @@
 // result does not depend on scheduling.
 #include "poss_internal.cuh"
 
+POSS_TRACE_REGISTER()
+
 #define NEG_BIG (-1.0e30f)
 
 template <typename T, int D> struct KeyLoad;
@@ -55,7 +57,7 @@ __global__ void __launch_bounds__(128) k_attn_partial(AttnArgs a, const T* q,
   __shared__ float qs[G * D];
   __shared__ float sm_m[4][G], sm_l[4][G];
   __shared__ float sm_o[4][G][D];
-  pdl_enter();
+  pdl_enter(POSS_K_ATTN_PARTIAL);
   int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < G * D; i += 128)
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(128) k_attn_partial(AttnArgs a, const T* q,
 
 template <typename T, int D>
 __global__ void k_attn_combine(int n_splits, const float* part, T* out) {
-  pdl_enter();
+  pdl_enter(POSS_K_ATTN_COMBINE);
   int rh = blockIdx.x;       // row * Hq + head
   int e = threadIdx.x;
   const float* pp = part + (size_t)rh * n_splits * (D + 2);

@@ -18,6 +18,8 @@
 #include "poss_internal.cuh"
 #include <string.h>
 
+POSS_TRACE_REGISTER()
+
 namespace {
 
 constexpr float NEG_BIG = -1.0e30f;
@@ -69,7 +71,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
   bf16* Ks = reinterpret_cast<bf16*>(smem_attn);  // [2][CHUNK][LD]
   bf16* Vs = Ks + 2 * CHUNK * LD;                 // [2][CHUNK][LD]
 
-  pdl_enter();
+  pdl_enter(POSS_K_ATTN_MMA);
 
   const int split = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnArgs a, const bf16* q,
 template <int D>
 __global__ void __launch_bounds__(128) k_attn_combine_bf16(int n_splits, int n_rh, const float* part, bf16* out) {
   constexpr int NP = D / 64;             // pairs per lane
-  pdl_enter();
+  pdl_enter(POSS_K_ATTN_COMBINE_BF16);
   const int lane = threadIdx.x & 31;
   const int rh = blockIdx.x * 4 + (threadIdx.x >> 5);       // row * Hq + head
   if (rh >= n_rh) return;

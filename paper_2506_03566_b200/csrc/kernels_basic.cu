@@ -1,6 +1,8 @@
 // Element-wise stages and the SIMT skinny matrix product (check mode and odd shapes).
 #include "poss_internal.cuh"
 
+POSS_TRACE_REGISTER()
+
 // ------------------------------------------------------------------ SIMT skinny GEMM
 // out[m][n] = sum_k X[m][k] * W[n][k] (+ bias[n]) (+ residual[m][n]).  One warp per output column n,
 // eight rows of X at a time in registers.  The reduction order of an output element depends only on
@@ -28,7 +30,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const T* X, int ldx, int M, G
                                                    int K, const T* bias,
                                                    const float* residual, int ldr,
                                                    float* out, int ldo) {
-  pdl_enter();
+  pdl_enter(POSS_K_GEMM_SIMT);
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int n = blockIdx.x * 8 + warp;
   if (n >= N) return;
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(256) k_gather_x(StepRows s, const int32_t* new
                                                   const int32_t* node_prow, int Kmax,
                                                   const T* fb, const T* embed, int H,
                                                   T* X) {
-  pdl_enter();
+  pdl_enter(POSS_K_GATHER_X);
   int m = blockIdx.x;
   RowInfo r = row_info(s, m);
   int tok;
@@ -139,7 +141,7 @@ template void launch_gather_x<bf16>(Launcher&, StepRows, const int32_t*, const b
 template <typename T>
 __global__ void k_embed_rows(const int32_t* tokens, const T* embed, int H,
                              float* out) {
-  pdl_enter();
+  pdl_enter(POSS_K_EMBED_ROWS);
   int m = blockIdx.x;
   const T* e = embed + (size_t)tokens[m] * H;
   for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)m * H + i] = to_f(e[i]);
@@ -158,7 +160,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* x, int H, const T*
                                                  float eps, T* out) {
   __shared__ float red[8];
   __shared__ float inv_s;
-  pdl_enter();
+  pdl_enter(POSS_K_RMSNORM);
   const float* xr = x + (size_t)blockIdx.x * H;
   T* o = out + (size_t)blockIdx.x * H;
   if (gain == nullptr) {
@@ -210,7 +212,7 @@ template void launch_rmsnorm<bf16>(Launcher&, const float*, int, int, const bf16
 
 template <typename T>
 __global__ void k_cast(const float* x, size_t n, T* out) {
-  pdl_enter();
+  pdl_enter(POSS_K_CAST);
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = from_f<T>(x[i]);
 }
@@ -225,7 +227,7 @@ template void launch_cast_rows<bf16>(Launcher&, const float*, size_t, bf16*);
 // act = T(silu(gate) * up), gate/up stored side by side: gu[row][0..F) gate, [F..2F) up
 template <typename T>
 __global__ void k_silu_mul(const float* gu, int F, T* out) {
-  pdl_enter();
+  pdl_enter(POSS_K_SILU_MUL);
   int row = blockIdx.y;
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= F) return;
@@ -331,7 +333,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_reduce_norm(SplitKView prod, i
     }
   }
   __syncthreads();
-  pdl_sync();
+  pdl_sync(POSS_K_REDUCE_NORM);
   POSS_TRACE_POINT(1);
   float ss = 0.f;
   // value of one group of four columns: product + (residual + bias), stored to h, squares added to ss
@@ -432,7 +434,7 @@ template void launch_reduce_norm<bf16>(Launcher&, const SplitKView&, int, int, c
 template <typename T>
 __global__ void __launch_bounds__(256) k_splitk_reduce(SplitKView prod, int N, const T* bias, const float* residual,
                                                        int ldr, float* out, int ldo, T* out_act) {
-  pdl_enter();
+  pdl_enter(POSS_K_SPLITK_REDUCE);
   const int m = blockIdx.y;
   const int n = (blockIdx.x * 256 + threadIdx.x) * 4;
   if (n >= N) return;
@@ -481,7 +483,7 @@ __global__ void __launch_bounds__(256) k_splitk_swiglu(SplitKView prod, int M, i
   const int l0 = m0 < M ? m0 : M - 1, l1 = m1 < M ? m1 : M - 1;      // rows loaded (clamped), stored if < M
   const int off[4] = {l0 * 128 + cg, l0 * 128 + cg + 64, l1 * 128 + cg, l1 * 128 + cg + 64};
   const bool vec = (F & 3) == 0 && (reinterpret_cast<uintptr_t>(act) & 15) == 0;
-  pdl_sync();
+  pdl_sync(POSS_K_SPLITK_SWIGLU);
   if (f >= F || m0 >= M) return;
   float4 x[4];
   splitk_sum<4>(prod, tc, off, x);
@@ -561,7 +563,7 @@ __global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, Spl
   }
   const bool vec = aligned16(kcache) && aligned16(vcache) && (a.q_rows == 0 || aligned16(qout));
   __syncthreads();
-  pdl_sync();
+  pdl_sync(POSS_K_ROPE_APPEND);
   int slot, pos;
   if (a.mode == 0) {
     RowInfo r = row_info(a.s, m);
@@ -642,7 +644,7 @@ template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKV
 
 // chain mask / depth for causal prefill chunks: row r sees rows 0..r of its chunk
 __global__ void k_chain_mask(uint64_t* mask, int32_t* depth, int rows) {
-  pdl_enter();
+  pdl_enter(POSS_K_CHAIN_MASK);
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= rows) return;
   depth[r] = r;

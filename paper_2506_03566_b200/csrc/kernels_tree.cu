@@ -4,6 +4,8 @@
 #include <math.h>
 #include <string.h>
 
+POSS_TRACE_REGISTER()
+
 #define NEG_INF (-INFINITY)
 
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
@@ -26,7 +28,7 @@ __global__ void __launch_bounds__(256) k_topk_partial(const float* logits, int V
   __shared__ float wv[8];
   __shared__ int wi[8];
   __shared__ float s_max;
-  pdl_enter();
+  pdl_enter(POSS_K_TOPK_PARTIAL);
   int chunk = blockIdx.x, row = blockIdx.y;
   int lo = chunk * POSS_TOPK_CHUNK;
   int n = min(POSS_TOPK_CHUNK, V - lo);
@@ -104,7 +106,7 @@ __global__ void __launch_bounds__(256) k_argmax_partial(const T* logits, int V, 
                                                         int32_t* pidx, int n_chunks) {
   __shared__ float wv[8];
   __shared__ int wi[8];
-  pdl_enter();
+  pdl_enter(POSS_K_ARGMAX_PARTIAL);
   const int chunk = blockIdx.x, row = blockIdx.y;
   const int lo = chunk * POSS_ARGMAX_CHUNK;
   const int n = min(POSS_ARGMAX_CHUNK, V - lo);
@@ -232,7 +234,7 @@ __global__ void __launch_bounds__(128) k_topk_merge(int K, int n_lists, const fl
   __shared__ float red[4];
   __shared__ float s_gm, s_lse;
   __shared__ int s_is_last;
-  pdl_enter();
+  pdl_enter(POSS_K_TOPK_MERGE);
   const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* rmax = pmax + (size_t)row * n_lists;
   const float* rsum = psum + (size_t)row * n_lists;
@@ -335,7 +337,7 @@ __global__ void __launch_bounds__(1024) k_topk_merge_expand(int rows, int K, int
   float* smax = reinterpret_cast<float*>(idxs + total4);         // [rows][n_lists]
   float* ssum = smax + rows * n_lists;                           // [rows][n_lists]
   int* heads = reinterpret_cast<int*>(ssum + rows * n_lists);    // [rows][n_lists]
-  pdl_enter();
+  pdl_enter(POSS_K_TOPK_MERGE_EXPAND);
   {
     const int n4 = total / 4;
     const float4* pv4 = reinterpret_cast<const float4*>(pval);
@@ -512,7 +514,7 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
                                                  uint64_t* out_mask, int32_t* out_n_nodes) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ int wtot[32];
-  pdl_enter();
+  pdl_enter(POSS_K_RERANK);
   float* sc = reinterpret_cast<float*>(smem_raw);               // [n_cand]
   int* newidx = reinterpret_cast<int*>(sc + n_cand);            // [n_cand] node index or 0 if dropped
   int* par = newidx + n_cand;                                   // [n_cand] parent candidate
@@ -606,7 +608,7 @@ __global__ void __launch_bounds__(256) k_accept_walk(const int32_t* g, const T* 
   __shared__ int s_tok[256], s_par[256], s_g[256];
   __shared__ int path[POSS_MAX_DEPTH + 1];
   __shared__ int s_a;
-  pdl_enter();
+  pdl_enter(POSS_K_ACCEPT_WALK);
   for (int i = threadIdx.x; i < rows; i += blockDim.x) { s_tok[i] = tokens[i]; s_par[i] = parents[i]; s_g[i] = g[i]; }
   __syncthreads();
   const int lane = threadIdx.x & 31;
@@ -692,7 +694,7 @@ __global__ void __launch_bounds__(SW_THREADS) k_sample_walk(const float* logits,
   __shared__ float s_m, s_z, s_rem, s_thr;
   __shared__ int s_next, s_nrem, s_used, s_a, s_bonus, s_warp;
   __shared__ float s_before;
-  pdl_enter();
+  pdl_enter(POSS_K_SAMPLE_WALK);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < rows; i += SW_THREADS) { s_tok[i] = tokens[i]; s_par[i] = parents[i]; }
   if (threadIdx.x == 0) { path[0] = 0; s_used = 0; }
@@ -837,7 +839,7 @@ template <typename T>
 __global__ void __launch_bounds__(128) k_kv_compact(T* kv, int Hkv, int cap, int d, int prefix_len,
                                                     const int32_t* path,
                                                     const int32_t* n_accepted) {
-  pdl_enter();
+  pdl_enter(POSS_K_KV_COMPACT);
   int a = n_accepted[0];
   T* base = kv + ((size_t)blockIdx.x * Hkv + blockIdx.y) * (size_t)cap * d;
   for (int k = 1; k <= a; ++k) {

@@ -54,6 +54,7 @@ struct Buffers {
   int* merge_done;       // [1] block counter of the top-k merge kernel
   double* rope_inv;      // [head_dim / 2] inverse rotary frequencies
   void* tc_scratch;      // split-K partials + tile counters of the tensor-core GEMM
+  unsigned long long* timeline;   // records of the timeline mode: header + (kernel id, time) rows
   TreeState ts;
 };
 
@@ -73,7 +74,8 @@ struct poss_ctx {
   TcGemmPlanCache* tc;
   bool attn_tc;          // tree attention on the tcgen05 kernel where it covers the call
   bool swiglu_in_kernel; // gate/up product finished by the GEMM's own SwiGLU epilogue instead of the consumer kernel
-  int prof_mode;         // 0 off, 1 = LM-head launches of the draft steps, 2 = every stage kind of the draft steps
+  int prof_mode;         // 0 off, 1 = LM-head launches of the draft steps, 2 = every stage kind of the draft steps,
+                         // 3 = timeline records written by the kernels themselves
   int prof_n;
   int prof_kind[1024];   // kind of each bracketed launch
   cudaEvent_t* prof_ev;   // 2 * PROF_MAX events, created on first enable
@@ -148,6 +150,7 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.merge_done = bp.take<int>(64, 4);
   b.rope_inv = bp.take<double>(64, 8);
   b.tc_scratch = bp.take<void>(tc_gemm_scratch_bytes(), 1);
+  b.timeline = bp.take<unsigned long long>(poss_trace::HEADER_WORDS + poss_trace::ROW_WORDS * poss_trace::MAX_ROWS, 8);
   b.ts.cand_tok = bp.take<int32_t>(*n_cand_max, 4);
   b.ts.cand_parent = bp.take<int32_t>(*n_cand_max, 4);
   b.ts.cand_score = bp.take<float>(*n_cand_max, 4);
@@ -170,7 +173,7 @@ struct Impl {
 
   // brackets the launches issued between begin and end with two events (profiling only)
   int prof_begin(int kind) {
-    if (!c->prof_mode || !in_draft || c->prof_n >= PROF_MAX) return -1;
+    if (!c->prof_mode || c->prof_mode == 3 || !in_draft || c->prof_n >= PROF_MAX) return -1;
     if (c->prof_mode == 1 && kind != POSS_PROF_LM_HEAD) return -1;
     int i = c->prof_n++;
     c->prof_kind[i] = kind;
@@ -186,10 +189,12 @@ struct Impl {
   // out[M][N] = x . segs^T (+bias) (+residual); picks the tensor-core kernel when it applies
   // out_act (optional, [M][ldo]) receives the same values in the context dtype
   void gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual, int ldr,
-            float* out, int ldo, int impl = 0, T* out_act = nullptr);
+            float* out, int ldo, int impl = 0, T* out_act = nullptr, int tag = POSS_K_GEMM_OTHER);
   // x . segs^T handed to a consumer kernel: split-K partials when the tensor-core kernel can leave them,
   // else the plain product in tmp[M][ldo]
-  SplitKView gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo);
+  // tag: which product this is (POSS_K_GEMM_*), for the timeline recording
+  SplitKView gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo,
+                       int tag = POSS_K_GEMM_OTHER);
   // act[M][F] = T(silu(x . gate^T) * (x . up^T))
   void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
   // tree-masked attention: the tcgen05 kernel where it covers the call (bf16, head dimension 128, at most
@@ -207,7 +212,7 @@ struct Impl {
     int pr = expand != nullptr ? prof_begin(POSS_PROF_LM_HEAD) : -1;   // the draft steps' launches only
     int n_lists = 0;
     bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists, !need_logp && K == 1);
-    if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab);
+    if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab, 0, nullptr, POSS_K_GEMM_LM_HEAD);
     prof_end(pr);
     if (!fused) {
       launch_topk_partial(L, lg, rows, g.vocab, K, c->b.pmax, c->b.psum, c->b.pval, c->b.pidx, c->n_chunks);
@@ -226,13 +231,13 @@ struct Impl {
     launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), W(c->embed), H, A(b.X));
     GemmSegs fc; fc.n = 1; fc.w[0] = lw.fc_w; fc.rows[0] = H;
     int pr = prof_begin(POSS_PROF_FC);
-    SplitKView v_fc = gemm_view(A(b.X), 2 * H, s.M, fc, 2 * H, b.ptmp, H);
+    SplitKView v_fc = gemm_view(A(b.X), 2 * H, s.M, fc, 2 * H, b.ptmp, H, POSS_K_GEMM_FC);
     prof_end(pr);
     launch_reduce_norm<T>(L, v_fc, s.M, H, W(lw.fc_b), nullptr, W(lw.norm_in), g.rms_eps, b.h0, A(b.xn));
     GemmSegs qkv; qkv.n = 3;
     qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
     pr = prof_begin(POSS_PROF_QKV);
-    SplitKView v_qkv = gemm_view(A(b.xn), H, s.M, qkv, H, b.ptmp, qd + 2 * kd);
+    SplitKView v_qkv = gemm_view(A(b.xn), H, s.M, qkv, H, b.ptmp, qd + 2 * kd, POSS_K_GEMM_QKV);
     prof_end(pr);
     RopeArgs ra;
     ra.inv_freq = b.rope_inv;
@@ -251,7 +256,7 @@ struct Impl {
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, F = g.ffn;
     GemmSegs so; so.n = 1; so.w[0] = lw.wo; so.rows[0] = H;
     int pr = prof_begin(POSS_PROF_O);
-    SplitKView v_o = gemm_view(A(b.o), qd, rows, so, qd, b.ptmp, H);
+    SplitKView v_o = gemm_view(A(b.o), qd, rows, so, qd, b.ptmp, H, POSS_K_GEMM_O);
     prof_end(pr);
     launch_reduce_norm<T>(L, v_o, rows, H, nullptr, x0, W(lw.norm_post), g.rms_eps, b.h1, A(b.u));
     pr = prof_begin(POSS_PROF_GATE_UP);
@@ -259,7 +264,7 @@ struct Impl {
     prof_end(pr);
     GemmSegs sd; sd.n = 1; sd.w[0] = lw.w_down; sd.rows[0] = H;
     pr = prof_begin(POSS_PROF_DOWN);
-    SplitKView v_d = gemm_view(A(b.act), F, rows, sd, F, b.ptmp, H);
+    SplitKView v_d = gemm_view(A(b.act), F, rows, sd, F, b.ptmp, H, POSS_K_GEMM_DOWN);
     prof_end(pr);
     if (next_gain) launch_reduce_norm<T>(L, v_d, rows, H, nullptr, b.h1, next_gain, g.rms_eps, out, out_act);
     else launch_splitk_reduce<T>(L, v_d, rows, H, nullptr, b.h1, H, out, H, out_act);
@@ -366,7 +371,7 @@ struct Impl {
       T* vc = kc + per_layer / 2;
       GemmSegs qkv; qkv.n = 3;
       qkv.w[0] = lw.wq; qkv.rows[0] = qd; qkv.w[1] = lw.wk; qkv.rows[1] = kd; qkv.w[2] = lw.wv; qkv.rows[2] = kd;
-      SplitKView v_qkv = gemm_view(A(b.xn), H, rows, qkv, H, b.ptmp, qd + 2 * kd);
+      SplitKView v_qkv = gemm_view(A(b.xn), H, rows, qkv, H, b.ptmp, qd + 2 * kd, POSS_K_GEMM_QKV);
       RopeArgs ra;
       ra.inv_freq = b.rope_inv;
       ra.mode = 1; ra.base = prefix_len; ra.depth = depth; ra.rows = rows; ra.q_rows = rows;
@@ -393,19 +398,19 @@ struct Impl {
 
 template <typename T>
 void Impl<T>::gemm(const T* x, int ldx, int M, const GemmSegs& segs, int K, const T* bias, const float* residual,
-                   int ldr, float* out, int ldo, int impl, T* out_act) {
+                   int ldr, float* out, int ldo, int impl, T* out_act, int) {
   launch_gemm_simt<T>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
   if (out_act) launch_cast_rows<T>(L, out, (size_t)M * ldo, out_act);
 }
 template <>
 void Impl<bf16>::gemm(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, const bf16* bias,
-                      const float* residual, int ldr, float* out, int ldo, int impl, bf16* out_act) {
+                      const float* residual, int ldr, float* out, int ldo, int impl, bf16* out_act, int tag) {
   bool can_tc = tc_gemm_supported(segs, K, ldx, M);
   if (impl == 2 && !can_tc) { L.err = POSS_E_SHAPE; return; }
   if (impl != 1 && can_tc) {
     TcEpilogue ep;
     ep.mode = TC_EPI_STORE; ep.bias = bias; ep.residual = residual; ep.ldr = ldr; ep.out = out; ep.ldo = ldo;
-    ep.out_bf = out_act; ep.ldo_bf = ldo;
+    ep.out_bf = out_act; ep.ldo_bf = ldo; ep.trace_tag = tag;
     launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, ep, c->b.tc_scratch, c->b.status);
   } else {
     launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, bias, residual, ldr, out, ldo);
@@ -414,7 +419,7 @@ void Impl<bf16>::gemm(const bf16* x, int ldx, int M, const GemmSegs& segs, int K
 }
 
 template <typename T>
-SplitKView Impl<T>::gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo) {
+SplitKView Impl<T>::gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo, int) {
   launch_gemm_simt<T>(L, x, ldx, M, segs, K, nullptr, nullptr, 0, tmp, ldo);
   SplitKView v;
   memset(&v, 0, sizeof(v));
@@ -422,13 +427,14 @@ SplitKView Impl<T>::gemm_view(const T* x, int ldx, int M, const GemmSegs& segs, 
   return v;
 }
 template <>
-SplitKView Impl<bf16>::gemm_view(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo) {
+SplitKView Impl<bf16>::gemm_view(const bf16* x, int ldx, int M, const GemmSegs& segs, int K, float* tmp, int ldo,
+                                 int tag) {
   SplitKView v;
   memset(&v, 0, sizeof(v));
   v.direct = tmp; v.ld = ldo;
   if (tc_gemm_supported(segs, K, ldx, M)) {
     TcEpilogue ep;
-    ep.mode = TC_EPI_STORE; ep.out = tmp; ep.ldo = ldo; ep.view = &v;
+    ep.mode = TC_EPI_STORE; ep.out = tmp; ep.ldo = ldo; ep.view = &v; ep.trace_tag = tag;
     launch_gemm_tc(L, c->tc, x, ldx, M, segs, K, ep, c->b.tc_scratch, c->b.status);
   } else {
     launch_gemm_simt<bf16>(L, x, ldx, M, segs, K, nullptr, nullptr, 0, tmp, ldo);
@@ -447,7 +453,7 @@ void Impl<bf16>::gemm_swiglu(const bf16* x, int M, const void* w_gate, const voi
   GemmSegs sg; sg.n = 2; sg.w[0] = w_gate; sg.rows[0] = F; sg.w[1] = w_up; sg.rows[1] = F;
   if (tc_gemm_supported(sg, K, K, M)) {
     TcEpilogue ep;
-    ep.mode = TC_EPI_SWIGLU; ep.out_bf = act; ep.ldo_bf = F;
+    ep.mode = TC_EPI_SWIGLU; ep.out_bf = act; ep.ldo_bf = F; ep.trace_tag = POSS_K_GEMM_GATE_UP;
     // The tile segments are left as partials and a consumer kernel spread over all SMs finishes them: the
     // in-kernel finish by the last CTA of each tile is a tail that grows with the row count and, measured, loses
     // even at 10 rows (48.0 vs 46.1 us for the product, 10 us per draft round).  The kernel's own SwiGLU epilogue
@@ -479,11 +485,30 @@ bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* 
   GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = c->cfg.vocab;
   if (!tc_gemm_supported(sg, K, K, M)) return false;
   TcEpilogue ep;
-  ep.mode = TC_EPI_TOPK; ep.topk = topk; ep.argmax_only = argmax_only;
+  ep.mode = TC_EPI_TOPK; ep.topk = topk; ep.argmax_only = argmax_only; ep.trace_tag = POSS_K_GEMM_LM_HEAD;
   ep.pmax = c->b.pmax; ep.psum = c->b.psum; ep.pval = c->b.pval; ep.pidx = c->b.pidx; ep.n_lists = n_lists;
   launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
   return true;
 }
+
+}  // namespace
+
+// ------------------------------------------------------------------ timeline recording: per-translation-unit setters
+namespace poss_trace {
+namespace {
+constexpr int MAX_UNITS = 16;
+SetFn& setter(int i) { static SetFn fns[MAX_UNITS] = {}; return fns[i]; }
+int& n_setters() { static int n = 0; return n; }
+}  // namespace
+void register_setter(SetFn fn) { if (n_setters() < MAX_UNITS) setter(n_setters()++) = fn; }
+bool set_all(unsigned long long* device_buf) {
+  bool ok = true;
+  for (int i = 0; i < n_setters(); ++i) ok = setter(i)(device_buf) && ok;
+  return ok;
+}
+}  // namespace poss_trace
+
+namespace {
 
 #define DISPATCH(ctx, stream, call)                         \
   ((ctx)->cfg.dtype == POSS_BF16 ? Impl<bf16>(ctx, stream).call : Impl<float>(ctx, stream).call)
@@ -554,6 +579,7 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
 
 int poss_destroy(poss_ctx* c) {
   if (!c) return POSS_E_INVALID;
+  if (c->prof_mode == 3) poss_trace::set_all(nullptr);
   tc_plan_cache_destroy(c->tc);
   if (c->prof_ev) {
     for (int i = 0; i < 2 * PROF_MAX; ++i) cudaEventDestroy(c->prof_ev[i]);
@@ -814,8 +840,16 @@ int poss_lm_head_topk(poss_ctx* c, const void* features, int rows, int topk, int
 }
 
 int poss_profile(poss_ctx* c, int mode) {
-  if (!c || mode < 0 || mode > 2) return POSS_E_INVALID;
-  if (mode && !c->prof_ev) {
+  if (!c || mode < 0 || mode > 3) return POSS_E_INVALID;
+  // the kernels' record pointer: the context's buffer in mode 3, nothing otherwise (synchronous host calls)
+  if (mode == 3) {
+    if (cudaMemset(c->b.timeline, 0, sizeof(unsigned long long) * poss_trace::HEADER_WORDS) != cudaSuccess)
+      return POSS_E_CUDA;
+    if (!poss_trace::set_all(c->b.timeline)) return POSS_E_CUDA;
+  } else if (c->prof_mode == 3) {
+    if (!poss_trace::set_all(nullptr)) return POSS_E_CUDA;
+  }
+  if (mode && mode != 3 && !c->prof_ev) {
     c->prof_ev = (cudaEvent_t*)malloc(sizeof(cudaEvent_t) * 2 * PROF_MAX);
     if (!c->prof_ev) return POSS_E_INVALID;
     for (int i = 0; i < 2 * PROF_MAX; ++i)
@@ -838,6 +872,36 @@ int poss_profile_read(poss_ctx* c, int* h_launches, float* h_total_ms) {
     h_total_ms[c->prof_kind[i]] += ms;
   }
   c->prof_n = 0;
+  return POSS_OK;
+}
+
+int poss_timeline_read(poss_ctx* c, int capacity, int32_t* h_kernel, int64_t* h_time_ns, int* h_count,
+                       poss_stream stream) {
+  if (!c || !h_kernel || !h_time_ns || !h_count || capacity < 0) return POSS_E_INVALID;
+  *h_count = 0;
+  cudaStream_t st = S(stream);
+  unsigned long long n = 0;
+  if (cudaMemcpyAsync(&n, c->b.timeline, sizeof(n), cudaMemcpyDeviceToHost, st) != cudaSuccess) return POSS_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return POSS_E_CUDA;
+  if (n > (unsigned long long)poss_trace::MAX_ROWS) n = poss_trace::MAX_ROWS;
+  if (n > (unsigned long long)capacity) n = capacity;
+  if (n) {
+    unsigned long long* rows = (unsigned long long*)malloc(sizeof(unsigned long long) * poss_trace::ROW_WORDS * n);
+    if (!rows) return POSS_E_INVALID;
+    bool ok = cudaMemcpyAsync(rows, c->b.timeline + poss_trace::HEADER_WORDS,
+                              sizeof(unsigned long long) * poss_trace::ROW_WORDS * n, cudaMemcpyDeviceToHost,
+                              st) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
+    // launches overlap (programmatic dependent launch), so the appends are not strictly in time order
+    for (unsigned long long i = 0; ok && i < n; ++i) {
+      h_kernel[i] = (int32_t)rows[poss_trace::ROW_WORDS * i];
+      h_time_ns[i] = (int64_t)rows[poss_trace::ROW_WORDS * i + 1];
+    }
+    free(rows);
+    if (!ok) return POSS_E_CUDA;
+  }
+  if (cudaMemsetAsync(c->b.timeline, 0, sizeof(unsigned long long) * poss_trace::HEADER_WORDS, st) != cudaSuccess)
+    return POSS_E_CUDA;
+  *h_count = (int)n;
   return POSS_OK;
 }
 

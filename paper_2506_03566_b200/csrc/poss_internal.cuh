@@ -81,14 +81,60 @@ struct Launcher {
 // through the read-only data path.  Pointers to activations, indices and caches therefore carry no
 // `const __restrict__` pair (the compiler would turn their loads into non-coherent ones and could hoist
 // them above the wait); only weights, which no kernel writes, may.
-__device__ __forceinline__ void pdl_enter() {
+//
+// Timeline recording (poss_profile mode 3).  While it is switched on, thread 0 of block (0,0,0) of every launch
+// appends (kernel id, device time at which its wait for the predecessor returned) to a buffer of the context.
+// The predecessor grid has completed at that instant, so the difference between two consecutive records is the
+// time the earlier kernel held the chain: its span *inside* the chain of dependent launches, overlap with its
+// neighbours included.  The buffer pointer is a per-device global of each translation unit (set on the host by
+// trace_set_all); when it is NULL, the cost is one predicated load in one thread per launch.
+namespace poss_trace {
+constexpr int HEADER_WORDS = 8, ROW_WORDS = 2, MAX_ROWS = 8192;
+static __device__ unsigned long long* g_buf = nullptr;
+typedef bool (*SetFn)(unsigned long long*);
+void register_setter(SetFn fn);                      // poss_api.cu: one entry per translation unit with kernels
+bool set_all(unsigned long long* device_buf);        // points every translation unit's g_buf at the buffer (or NULL)
+// internal linkage on purpose: every translation unit sets its own copy of g_buf
+static bool set_local(unsigned long long* p) {
+  return cudaMemcpyToSymbol(g_buf, &p, sizeof(p)) == cudaSuccess;
+}
+}  // namespace poss_trace
+// a translation unit that defines kernels places this once at file scope (the type lives in the unit's own
+// anonymous namespace, so that each unit registers its own setter)
+#define POSS_TRACE_REGISTER()                                                                  \
+  namespace {                                                                                  \
+  struct PossTraceRegistrar {                                                                  \
+    PossTraceRegistrar() { poss_trace::register_setter(&poss_trace::set_local); }              \
+  } g_poss_trace_registrar;                                                                    \
+  }
+
+__device__ __forceinline__ void pdl_trace(int kernel_id) {
+  if (kernel_id >= 0 && threadIdx.x == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) {
+    unsigned long long* buf = poss_trace::g_buf;
+    if (buf) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      const unsigned long long i = atomicAdd(buf, 1ull);
+      if (i < (unsigned long long)poss_trace::MAX_ROWS) {
+        buf[poss_trace::HEADER_WORDS + poss_trace::ROW_WORDS * i] = (unsigned long long)kernel_id;
+        buf[poss_trace::HEADER_WORDS + poss_trace::ROW_WORDS * i + 1] = t;
+      }
+    }
+  }
+}
+// kernel_id: a POSS_K_* value (poss_debug.h); -1 = a second wait inside a kernel whose first one records
+__device__ __forceinline__ void pdl_enter(int kernel_id) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  pdl_trace(kernel_id);
 }
 // The two halves, for kernels with work that needs nothing from a predecessor (index arithmetic on the
 // launch parameters, loads of weights): pdl_begin(), that work, pdl_sync(), then everything else.
 __device__ __forceinline__ void pdl_begin() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_sync(int kernel_id) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  pdl_trace(kernel_id);
+}
 
 // hook for a timeline-recording build; empty in the library
 #ifndef POSS_TRACE_POINT
