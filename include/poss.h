@@ -245,13 +245,14 @@ POSS_API int poss_tree_attention_noalloc(const void* q, const void* kv, int kv_s
                                          const uint64_t* anc_mask, float scale, void* out, poss_stream stream);
 
 /* Host-only query (no device is touched): how poss_tree_attention and the draft / target passes cut `total_keys`
- * visible-or-masked keys for a bf16 model with head dimension 128.  The tcgen05 kernel takes up to 2048 keys:
- * *keys_per_cta = 128 or 256 keys per CTA (groups of 128 keys at absolute positions, one or two per CTA) and
- * *ctas_per_cluster = CTAs of one (KV head, 128 query rows), 1..8; the cut depends on total_keys alone, and group j
- * always holds keys [128 j, 128 j + 128).  Returns POSS_OK, or POSS_E_SHAPE for a key count the kernel does not take
- * (the split-KV kernels then run; outputs untouched), POSS_E_INVALID for NULL outputs or total_keys < 1.
- * The paper has no counterpart. */
-POSS_API int poss_attention_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster);
+ * visible-or-masked keys for a bf16 model with head dimension 128.  The tcgen05 kernel takes up to 10240 keys:
+ * groups of 128 keys at absolute positions (group j always holds keys [128 j, 128 j + 128)), two consecutive groups
+ * per unit, one partial result per unit, all units merged in key order in one pass.  *keys_per_unit = 128 (one group,
+ * at most 128 keys in all) or 256, *n_units = units that hold keys; the cut depends on total_keys alone, never on the
+ * rows, the heads or the number of CTAs that share the units.  Returns POSS_OK, or POSS_E_SHAPE for a key count the
+ * kernel does not take (the split-KV kernels then run; outputs untouched), POSS_E_INVALID for NULL outputs or
+ * total_keys < 1.  The paper has no counterpart. */
+POSS_API int poss_attention_plan(int total_keys, int* keys_per_unit, int* n_units);
 
 #ifdef __cplusplus
 }

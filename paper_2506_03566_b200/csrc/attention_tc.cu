@@ -1,34 +1,41 @@
 // Tree-masked attention on the 5th-generation tensor cores (bf16, head dimension 128): the kernel of every
-// draft step and target layer whenever the key count fits one pass (at most 2048 keys).
+// draft step and target layer, from one key up to 10240 keys (prefix 8192 + tree and beyond).
 //
 // Geometry.  For one KV head the G = Hq/Hkv query heads of all tree rows form one matrix Q' of rows*G
 // query rows (query row qi = r*G + g).  The keys are cut into groups of 128 at absolute positions
-// (group j = keys [128 j, 128 j + 128)); a CTA owns two consecutive groups, one KV head and 128 query
-// rows.  The CTAs of one (KV head, query tile) form one thread-block cluster (1 to 8 of them):
-//   1. TMA brings the 128 x 128 query tile and the CTA's 256 keys and values into shared memory
-//      (128-byte swizzle; rows past the last key or the last tree row arrive as zeros);
-//   2. one thread issues S = Q' K^T (tcgen05.mma, M = 128 query rows, N = 256 keys, fp32 in TMEM);
-//   3. sixteen warps take S out of TMEM, one thread per (query row, group, half of the group's keys): scale,
-//      ancestor mask, row maximum (the halves meet through shared memory), p = 2^(s - m), row sum; p is written
-//      back to shared memory as a two-term bf16 split (p = hi + lo), laid out as the A operand of the next product;
-//   4. one thread issues O_g = P_g V_g for both groups (two MMAs per 16 keys: hi and lo; V is the MN-major
-//      B operand, read as it sits in the cache: [key][d]), each group into its own TMEM accumulator;
-//   5. every CTA merges its two groups and parks (m, l) and the 128 x 128 fp32 O in global memory (one
-//      short-lived partial per CTA, read back out of L2); after a cluster barrier CTA j merges its share of
-//      the query rows over the cluster's CTAs, in key order, and writes the bf16 result.  (Reading the
-//      peers' shared memory instead was measured: the SM-to-SM path moved these rows at a quarter of L2's
-//      rate.)
+// (group j = keys [128 j, 128 j + 128)) and two consecutive groups form a unit of 256 keys.  The units of one
+// (KV head, 128 query rows) are dealt round-robin to the CTAs that walk them (unit u goes to walker
+// u mod n_walk); a walker pipelines its groups:
+//   * one thread (warp 16) issues every copy and every product.  TMA brings the query tile once and, per group,
+//     128 keys (one stage: a group's keys are free again as soon as its scores exist) and 128 values (two
+//     stages), 128-byte swizzle, rows past the last key or the last tree row arriving as zeros.  S_g = Q' K_g^T
+//     (tcgen05.mma, M = 128 query rows, N = 128 keys, fp32 in TMEM) runs two groups ahead into one of two score
+//     buffers; O_g = P_g V_g (two MMAs per 16 keys: hi and lo; V is the MN-major B operand, read as it sits in
+//     the cache: [key][d]) goes into one of two output accumulators, one per group of the unit;
+//   * sixteen warps do the softmax of one group at a time, one thread per (query row, quarter of the group's
+//     keys): scores out of TMEM once (32 registers), ancestor mask, row maximum (the quarters meet through shared
+//     memory), p = 2^(s - m), row sum; p is written to shared memory as a two-term bf16 split (p = hi + lo), laid
+//     out as the A operand of the second product;
+//   * when a unit's groups are done the same warps merge the two accumulators and park (m, l) and the 128 x 128
+//     fp32 O of the unit in global memory (short-lived, read back out of L2).
+// The walkers of one (KV head, query tile) form one or more thread-block clusters of up to 8 CTAs.  After a
+// cluster barrier the CTA of cluster rank j merges its share of the query rows over ALL units in key order and
+// writes the bf16 result.  With several clusters, the rank-j CTAs count their arrivals per (KV head, query tile,
+// rank) after their own cluster's barrier, and the one that arrives last does rank j's merge: nobody waits for
+// another cluster.
 //
-// The groups sit at absolute key positions and a query row's arithmetic does not depend on where in the
-// tile it sits, nor on keys it does not see (a masked key enters every sum as an exact zero): a token whose
-// visible keys are the prefix and itself gets the same bit pattern whether it is verified as the root of a
-// 61-row tree or decoded alone.
+// The groups and units sit at absolute key positions, every unit is parked on its own and the final merge is
+// one flat pass over the units in key order, so a query row's arithmetic depends neither on how many walkers
+// there are, nor on where in the tile the row sits, nor on keys it does not see (a masked key enters every sum
+// as an exact zero): a token whose visible keys are the prefix and itself gets the same bit pattern whether it
+// is verified as the root of a 61-row tree or decoded alone.
 //
 // Visibility.  Keys [0, n_all) are seen by every row; key n_all + t is seen by row r iff bit t of the
 // row's packed ancestor mask is set.
 //
-// Every wait on an mbarrier is bounded (wall time); on expiry the CTA raises POSS_E_TIMEOUT, skips its
-// remaining work, still meets its cluster at the barrier, frees its TMEM and returns.
+// Every wait on an mbarrier is bounded (wall time); on expiry the CTA raises POSS_E_TIMEOUT; every later wait
+// then returns at once, the CTA runs through the rest of its (bounded) walk without meaning, still meets its
+// cluster at the barrier, keeps the arrival counters consistent, frees its TMEM and returns.
 #include "gemm_tc.cuh"
 #include "tc_ptx.cuh"
 #include <string.h>
@@ -41,24 +48,34 @@ using namespace tcptx;
 
 constexpr int D = 128;
 constexpr int QT = 128;               // query rows per CTA (UMMA M)
-constexpr int N_THREADS = 512;        // sixteen warps: TMEM lane quarter x key group x half of the group
-constexpr int KG = 128;               // keys per group: the unit of the softmax partials, at absolute positions
-constexpr int MAX_CTA_KEYS = 2 * KG;  // keys per CTA (UMMA N of the first product)
-constexpr int MAX_SPLITS = 8;         // portable cluster size
+constexpr int KG = 128;               // keys per group: the unit of the softmax, at absolute positions
+constexpr int UNIT_KEYS = 2 * KG;     // keys per parked partial
+constexpr int N_SOFTMAX = 512;        // sixteen softmax warps: TMEM lane quarter x quarter of the group's keys
+constexpr int N_THREADS = N_SOFTMAX + 32;   // + the warp whose first lane issues copies and products
+constexpr int MAX_CLUSTER = 8;        // portable cluster size
+constexpr int MAX_UNITS = 40;         // 10240 keys
+constexpr int MAX_ARRIVAL_SETS = 512; // (KV head, query tile) pairs that can run with several clusters
 constexpr int O_LD = D + 4;           // floats per parked partial: 128 outputs, m, l, padding to 16 bytes
-constexpr int HALF_TILE = QT * 128;   // bytes of a [128 rows][64 bf16] tile
+constexpr int TILE = 128 * 128;       // bytes of a [128 rows][64 bf16] tile
 constexpr float NEG_BIG = -1.0e30f;
+// shared memory: query tile (two 64-column halves), one key stage, two value stages, P as hi and lo (two 64-key
+// blocks each)
+constexpr uint32_t Q_OFF = 0, K_OFF = 2 * TILE, V_OFF = 4 * TILE, P_HI = 8 * TILE, P_LO = 10 * TILE;
+constexpr uint32_t SMEM_TILES = 12 * TILE;                // 192 KB
+constexpr uint32_t TMEM_COLS = 512;                       // S0 | S1 | O0 | O1, 128 columns each
 
 struct AttnTcArgs {
   int rows, Hq, G, n_q;               // n_q = rows * G query rows per KV head
   int n_all, n_tree, total;
-  int cta_keys, n_splits;             // keys per CTA (128 or 256); CTAs per cluster
-  uint32_t region_a_bytes;            // Q + K, later P (hi, lo); V sits behind it
+  int n_units;                        // 256-key units of the call
+  int n_walk;                         // CTAs that share the units of one (KV head, query tile)
+  int cluster, n_clusters;            // n_walk = cluster * n_clusters
   const uint64_t* mask;
   int mask_words;
   float scale_log2;                   // softmax scale times log2(e)
   int inject_lost_load;               // test hook: the value tiles are never requested
-  float* part;                        // [rows][Hq][n_splits][O_LD]: a CTA's merged partial, 128 outputs then (m, l)
+  float* part;                        // [rows][Hq][n_units][O_LD]: a unit's partial, 128 outputs then (m, l)
+  int* arrivals;                      // [Hkv * query tiles][MAX_CLUSTER], zero between launches
   bf16* out;
   int32_t* status;
 };
@@ -101,6 +118,8 @@ __device__ __forceinline__ uint32_t cluster_rank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
+// barrier among the sixteen softmax warps only
+__device__ __forceinline__ void softmax_sync(int id) { asm volatile("bar.sync %0, 512;" ::"r"(id) : "memory"); }
 // 16 TMEM columns of this thread's lane into registers, without waiting; tmem_wait16 is the matching wait (it
 // names the registers, so nothing that reads them can be scheduled ahead of it)
 __device__ __forceinline__ void tmem_ld16_async(uint32_t taddr, uint32_t* r) {
@@ -129,47 +148,51 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
 }
 
 // ------------------------------------------------------------------ the kernel
-// 512 threads: warp w owns TMEM lane quarter q = w & 3 (32 query rows), key group g = (w >> 2) & 1 and half
-// hf = w >> 3 of the group's eight 16-key chunks in the softmax; column quarter cq = w >> 2 (32 output columns) when
-// the outputs are parked.  Thread 0 also issues the copies and both products.
+// 544 threads.  Softmax warp w (0..15) owns TMEM lane quarter q = w & 3 (32 query rows) and quarter cq = w >> 2 of
+// a group's eight 16-key chunks; when a unit is parked the same thread owns output columns [32 cq, 32 cq + 32).
+// Lane 0 of warp 16 issues the copies and both products.
 __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant__ CUtensorMap map_q,
                                                           const __grid_constant__ CUtensorMap map_k,
                                                           const __grid_constant__ CUtensorMap map_v, const AttnTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[5];
+  __shared__ __align__(8) uint64_t bars[9];
   __shared__ uint32_t tmem_slot;
-  __shared__ int s_abort;
-  __shared__ float half_max[2][2][QT], half_sum[2][2][QT];     // [half][group][query row]
-  __shared__ float grp_m[2][QT];                               // scaled maximum per group and query row
+  __shared__ int s_abort, s_last;
+  __shared__ float x_max[4][QT], x_sum[4][QT];                 // [key quarter][query row]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
+  const int walker = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const int cta_keys = a.cta_keys, ng = cta_keys / KG;
-  const uint32_t k_half = (uint32_t)cta_keys * 128u;            // bytes of [cta_keys][64 bf16]
-  const uint32_t q_off = 0, k_off = 2 * HALF_TILE;              // region A, first life
-  const uint32_t p_hi = 0, p_lo = (uint32_t)(cta_keys / 64) * HALF_TILE;   // region A, second life
-  const uint32_t v_off = a.region_a_bytes;
-  const uint32_t bar_qk = smem_u32(&bars[0]), bar_v = smem_u32(&bars[1]), bar_s = smem_u32(&bars[2]),
-                 bar_p = smem_u32(&bars[3]), bar_o = smem_u32(&bars[4]);
-  const uint32_t o_col = (uint32_t)cta_keys;                    // S at column 0, O of group g at o_col + 128 g
-  const uint32_t tmem_cols = 2u * (uint32_t)cta_keys;
-  const int k_begin = split * cta_keys;
-  // keys of group g that exist at all (the rest of the group, if any, is zero fill)
-  auto group_keys = [&](int g) {
-    int n = a.total - (k_begin + g * KG);
+  const uint32_t bar_q = smem_u32(&bars[0]), bar_k = smem_u32(&bars[1]), bar_p = smem_u32(&bars[6]),
+                 bar_pv = smem_u32(&bars[7]), bar_of = smem_u32(&bars[8]);
+  auto bar_v = [&](int st) { return smem_u32(&bars[2 + st]); };
+  auto bar_s = [&](int b) { return smem_u32(&bars[4 + b]); };
+
+  // this walker's groups, in the order it meets them: its units walker, walker + n_walk, ...; a unit's second
+  // group exists when it holds at least one key
+  const int n_my_units = walker < a.n_units ? (a.n_units - 1 - walker) / a.n_walk + 1 : 0;
+  auto group_of = [&](int gi) { return 2 * (walker + (gi >> 1) * a.n_walk) + (gi & 1); };
+  auto keys_of = [&](int grp) {
+    int n = a.total - grp * KG;
     return n < 0 ? 0 : (n > KG ? KG : n);
   };
+  int n_g = 2 * n_my_units;
+  if (n_g > 0 && keys_of(group_of(n_g - 1)) == 0) --n_g;
 
   if (warp == 0) {
     if (lane == 0) {
       s_abort = 0;
-      mbar_init(bar_qk, 1);
-      mbar_init(bar_v, 1);
-      mbar_init(bar_s, 1);
-      mbar_init(bar_p, N_THREADS);
-      mbar_init(bar_o, 1);
+      s_last = 0;
+      mbar_init(bar_q, 1);
+      mbar_init(bar_k, 1);
+      mbar_init(bar_v(0), 1);
+      mbar_init(bar_v(1), 1);
+      mbar_init(bar_s(0), 1);
+      mbar_init(bar_s(1), 1);
+      mbar_init(bar_p, N_SOFTMAX);
+      mbar_init(bar_pv, 1);
+      mbar_init(bar_of, N_SOFTMAX);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       prefetch_tensormap(&map_q);
@@ -177,7 +200,7 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
       prefetch_tensormap(&map_v);
     }
     __syncwarp();
-    tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    tmem_alloc(smem_u32(&tmem_slot), TMEM_COLS);
   }
   tc_fence_before();
   __syncthreads();
@@ -190,189 +213,257 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   pdl_begin();
   pdl_sync(POSS_K_ATTN_TC);
 
-  if (threadIdx.x == 0) {
-    // ---------------- the copies and the first product
-    mbar_expect_tx(bar_qk, 2u * HALF_TILE + 2u * k_half);
-    tma_load_4d(base + q_off, &map_q, bar_qk, 0, 0, kvh, qtile * (QT / a.G));
-    tma_load_4d(base + q_off + HALF_TILE, &map_q, bar_qk, 64, 0, kvh, qtile * (QT / a.G));
-    tma_load_3d(base + k_off, &map_k, bar_qk, 0, k_begin, kvh);
-    tma_load_3d(base + k_off + k_half, &map_k, bar_qk, 64, k_begin, kvh);
-    mbar_expect_tx(bar_v, 2u * k_half);
-    if (!a.inject_lost_load) {
-      tma_load_3d(base + v_off, &map_v, bar_v, 0, k_begin, kvh);
-      tma_load_3d(base + v_off + k_half, &map_v, bar_v, 64, k_begin, kvh);
-    }
-    if (mbar_wait(bar_qk, 0, abort_flag)) {
-      tc_fence_after();
-      const uint32_t idesc = instr_desc_bf16(QT, cta_keys);
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const uint64_t ad = smem_desc_sw128(base + q_off + h * HALF_TILE), bd = smem_desc_sw128(base + k_off + h * k_half);
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)          // 16 bf16 = 32 bytes = 2 descriptor address units
-          umma_bf16(tmem_base, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (h | kk) ? 1u : 0u);
-      }
-      umma_commit(bar_s);
-    }
-  }
-  __syncwarp();
-
-  // ---------------- softmax: TMEM lane = query row
-  const int q = warp & 3, g = (warp >> 2) & 1, hf = warp >> 3;
-  const int row = q * 32 + lane;
-  const int qi = qtile * QT + row;
-  const bool valid = qi < a.n_q;
-  const int r = valid ? qi / a.G : 0;
-  uint64_t mk0 = 0, mk1 = 0;
-  if (valid) {
-    mk0 = a.mask[(size_t)r * a.mask_words];
-    if (a.mask_words > 1) mk1 = a.mask[(size_t)r * a.mask_words + 1];
-  }
-  const int n_grp = g < ng ? (group_keys(g) + 15) / 16 : 0;          // 16-key chunks of this warp's group
-  const int c_lo = hf * 4 < n_grp ? hf * 4 : n_grp, c_hi = hf * 4 + 4 < n_grp ? hf * 4 + 4 : n_grp;
-  const int key_g = k_begin + g * KG;
-  const uint32_t t_s = tmem_base + ((uint32_t)(q * 32) << 16);
-  bool ok = mbar_wait(bar_s, 0, abort_flag);
-  tc_fence_after();
-  POSS_TRACE_POINT(1);
-  // Two passes over this thread's scores, 16 keys per TMEM load, as compact loops: a CTA runs this code once, so
-  // every instruction is fetched cold and short bodies that iterate beat straight-line code.  Invisible keys become
-  // -inf: they lose every maximum and their 2^x is an exact zero.
-  auto chunk = [&](int c, uint32_t* sr) {
-    tmem_ld16_async(t_s + (uint32_t)(g * KG + c * 16), sr);
-    tmem_wait16(sr);
-    const int key0 = key_g + c * 16;
-    if (key0 + 16 > a.n_all) {                         // the chunk reaches the tree slots or the end
-      // bit j = key0 + j is visible: 16 bits cut out of (all ones below n_all | the row's ancestor mask)
-      const int t0 = key0 - a.n_all;                   // tree slot of the chunk's first key; > -16
-      uint32_t vis;
-      if (t0 >= 64) vis = t0 >= 128 ? 0u : (uint32_t)(mk1 >> (t0 - 64));
-      else if (t0 > 48) vis = (uint32_t)(mk0 >> t0) | (uint32_t)(mk1 << (64 - t0));
-      else if (t0 >= 0) vis = (uint32_t)(mk0 >> t0);
-      else vis = ((uint32_t)mk0 << (-t0)) | ((1u << (-t0)) - 1u);
-      const int n_valid = a.total - key0;              // keys of the chunk that exist
-      if (n_valid < 16) vis &= (1u << (n_valid < 0 ? 0 : n_valid)) - 1u;
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (!((vis >> j) & 1u)) sr[j] = 0xff800000u;
-    }
-  };
-  {
-    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    if (ok) {
-#pragma unroll 1
-      for (int c = c_lo; c < c_hi; ++c) {
-        uint32_t sr[16];
-        chunk(c, sr);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sr[j]));
-      }
-    }
-    half_max[hf][g][row] = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-  }
-  __syncthreads();
-  {
-    const float mraw = fmaxf(half_max[0][g][row], half_max[1][g][row]);
-    // the scale is positive: the maximum of the scaled scores is the scaled maximum
-    const float ms = mraw == -INFINITY ? 0.f : mraw * a.scale_log2;
-    if (hf == 0) grp_m[g][row] = mraw == -INFINITY ? NEG_BIG : ms;
-    float ls[4] = {0.f, 0.f, 0.f, 0.f};
-    if (ok) {
-#pragma unroll 1
-      for (int c = c_lo; c < c_hi; ++c) {
-        uint32_t sr[16];
-        chunk(c, sr);
-        uint32_t hi[8], lo[8];
-#pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(sr[j]), a.scale_log2, -ms));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[j + 1]), a.scale_log2, -ms));
-          ls[j & 3] += p0;
-          ls[(j & 3) + 1] += p1;
-          split_pack(p0, p1, hi[j >> 1], lo[j >> 1]);
+  if (warp == 16) {
+    if (lane == 0 && n_g > 0) {
+      // ---------------- copies and products
+      int k_loads = 0, v_loads0 = 0, v_loads1 = 0;
+      auto load_k = [&](int gi) {
+        const int key0 = group_of(gi) * KG;
+        mbar_expect_tx(bar_k, 2u * TILE);
+        tma_load_3d(base + K_OFF, &map_k, bar_k, 0, key0, kvh);
+        tma_load_3d(base + K_OFF + TILE, &map_k, bar_k, 64, key0, kvh);
+        ++k_loads;
+      };
+      auto load_v = [&](int gi) {
+        const int key0 = group_of(gi) * KG, st = gi & 1;
+        mbar_expect_tx(bar_v(st), 2u * TILE);
+        if (!a.inject_lost_load) {
+          tma_load_3d(base + V_OFF + st * 2u * TILE, &map_v, bar_v(st), 0, key0, kvh);
+          tma_load_3d(base + V_OFF + st * 2u * TILE + TILE, &map_v, bar_v(st), 64, key0, kvh);
         }
-        // A operand of P V: k-block of 64 keys, row = query row (128 bytes), 16-byte pieces swizzled by row
-        const int kc = g * (KG / 16) + c;
-        const uint32_t line = (uint32_t)(kc >> 2) * HALF_TILE + (uint32_t)row * 128u;
-        const uint32_t pc = (uint32_t)(kc & 3) * 2u, sw = (uint32_t)(row & 7);
-        *reinterpret_cast<uint4*>(base_ptr + p_hi + line + ((pc ^ sw) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(base_ptr + p_hi + line + (((pc + 1) ^ sw) << 4)) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-        *reinterpret_cast<uint4*>(base_ptr + p_lo + line + ((pc ^ sw) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        *reinterpret_cast<uint4*>(base_ptr + p_lo + line + (((pc + 1) ^ sw) << 4)) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-      }
-    }
-    half_sum[hf][g][row] = (ls[0] + ls[1]) + (ls[2] + ls[3]);
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P becomes visible to the tensor core
-  mbar_arrive(bar_p);
-  POSS_TRACE_POINT(2);
-
-  if (threadIdx.x == 0) {
-    // ---------------- the second product, once the values and all of P are in shared memory
-    const bool v_ok = mbar_wait(bar_v, 0, abort_flag);
-    if (v_ok && mbar_wait(bar_p, 0, abort_flag) && *abort_flag == 0) {
-      tc_fence_after();
-      const uint32_t idesc = instr_desc_bf16(QT, D) | (1u << 16);     // B (the values) is MN-major
-      for (int gg = 0; gg < ng; ++gg) {
-        const int steps = (group_keys(gg) + 15) / 16;
+        if (st) ++v_loads1; else ++v_loads0;
+      };
+      const uint32_t idesc_s = instr_desc_bf16(QT, KG);
+      const uint32_t idesc_o = instr_desc_bf16(QT, D) | (1u << 16);     // B (the values) is MN-major
+      auto issue_s = [&](int gi) {
+        const uint32_t t_s = tmem_base + (uint32_t)((gi & 1) * KG);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint64_t ad = smem_desc_sw128(base + Q_OFF + h * TILE), bd = smem_desc_sw128(base + K_OFF + h * TILE);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)          // 16 bf16 = 32 bytes = 2 descriptor address units
+            umma_bf16(t_s, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc_s, (h | kk) ? 1u : 0u);
+        }
+        umma_commit(bar_s(gi & 1));
+      };
+      auto issue_pv = [&](int gi) {
+        const int steps = (keys_of(group_of(gi)) + 15) / 16;
+        const uint32_t t_o = tmem_base + 2u * KG + (uint32_t)((gi & 1) * D);
+        const uint32_t v_base = base + V_OFF + (uint32_t)(gi & 1) * 2u * TILE;
         for (int ks = 0; ks < steps; ++ks) {
-          const int kc = gg * (KG / 16) + ks;                         // 16-key step inside the CTA's keys
-          const uint32_t pa = (uint32_t)(kc >> 2) * HALF_TILE;
-          const uint64_t step = (uint64_t)(2 * (kc & 3));
-          const uint64_t ah = smem_desc_sw128(base + p_hi + pa) + step, al = smem_desc_sw128(base + p_lo + pa) + step;
-          const uint64_t bd = smem_desc_sw128_mn(base + v_off + (uint32_t)kc * 2048u, k_half);
-          const uint32_t t_o = tmem_base + o_col + (uint32_t)(gg * D);
-          umma_bf16(t_o, ah, bd, idesc, ks > 0 ? 1u : 0u);
-          umma_bf16(t_o, al, bd, idesc, 1u);
+          const uint32_t pa = (uint32_t)(ks >> 2) * TILE;
+          const uint64_t step = (uint64_t)(2 * (ks & 3));
+          const uint64_t ah = smem_desc_sw128(base + P_HI + pa) + step, al = smem_desc_sw128(base + P_LO + pa) + step;
+          const uint64_t bd = smem_desc_sw128_mn(v_base + (uint32_t)ks * 2048u, TILE);
+          umma_bf16(t_o, ah, bd, idesc_o, ks > 0 ? 1u : 0u);
+          umma_bf16(t_o, al, bd, idesc_o, 1u);
+        }
+        umma_commit(bar_pv);
+      };
+
+      mbar_expect_tx(bar_q, 2u * TILE);
+      tma_load_4d(base + Q_OFF, &map_q, bar_q, 0, 0, kvh, qtile * (QT / a.G));
+      tma_load_4d(base + Q_OFF + TILE, &map_q, bar_q, 64, 0, kvh, qtile * (QT / a.G));
+      load_k(0);
+      load_v(0);
+      if (n_g > 1) load_v(1);
+      bool ok = mbar_wait(bar_q, 0, abort_flag) && mbar_wait(bar_k, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0);
+      }
+      if (ok && n_g > 1) {
+        ok = mbar_wait(bar_s(0), 0, abort_flag);              // the first group's scores exist: its keys may go
+        if (ok) {
+          load_k(1);
+          ok = mbar_wait(bar_k, 1, abort_flag);
+        }
+        if (ok) {
+          tc_fence_after();
+          issue_s(1);
+          if (n_g > 2) {
+            ok = mbar_wait(bar_s(1), 0, abort_flag);
+            if (ok) load_k(2);
+          }
         }
       }
-      umma_commit(bar_o);
+      for (int gi = 0; gi < n_g && ok; ++gi) {
+        ok = mbar_wait(bar_p, (uint32_t)(gi & 1), abort_flag) &&                      // P of this group is written
+             mbar_wait(bar_v(gi & 1), (uint32_t)((gi >> 1) & 1), abort_flag);         // its values have landed
+        // a unit's accumulators are free again once the previous unit has been read out of them
+        if (ok && (gi & 1) == 0 && gi >= 2) ok = mbar_wait(bar_of, (uint32_t)(((gi >> 1) - 1) & 1), abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(gi);
+        if (gi + 2 < n_g) {
+          // scores two groups ahead, into the buffer this group's softmax has just left
+          ok = mbar_wait(bar_k, (uint32_t)((gi + 2) & 1), abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(gi + 2);
+          if (gi + 3 < n_g) {
+            ok = mbar_wait(bar_s(gi & 1), (uint32_t)(((gi + 2) >> 1) & 1), abort_flag);
+            if (!ok) break;
+            load_k(gi + 3);
+          }
+          ok = mbar_wait(bar_pv, (uint32_t)(gi & 1), abort_flag);                     // this group's values may go
+          if (!ok) break;
+          load_v(gi + 2);
+        }
+      }
+      if (*abort_flag) {
+        // drain: the copies this thread started must land before the CTA's shared memory goes away
+        const uint64_t t0 = global_ns();
+        auto drain = [&](uint32_t bar, int loads) {
+          if (loads <= 0) return;
+          const uint32_t par = (uint32_t)((loads - 1) & 1);
+          while (!mbar_try_wait(bar, par) && global_ns() - t0 < WAIT_LIMIT_NS / 2) __nanosleep(64);
+        };
+        drain(bar_q, 1);
+        drain(bar_k, k_loads);
+        drain(bar_v(0), v_loads0);
+        drain(bar_v(1), v_loads1);
+      }
     }
-    if (*abort_flag) {
-      // drain: the copies this thread started must land before the CTA's shared memory goes away
-      uint64_t t0 = global_ns();
-      while (!mbar_try_wait(bar_qk, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 4) __nanosleep(64);
-      while (!mbar_try_wait(bar_v, 0) && global_ns() - t0 < WAIT_LIMIT_NS / 2) __nanosleep(64);
+  } else {
+    // ---------------- softmax and parking: TMEM lane = query row
+    const int q = warp & 3, cq = warp >> 2;
+    const int row = q * 32 + lane;
+    const int qi = qtile * QT + row;
+    const bool valid = qi < a.n_q;
+    const int r = valid ? qi / a.G : 0;
+    uint64_t mk0 = 0, mk1 = 0;
+    if (valid) {
+      mk0 = a.mask[(size_t)r * a.mask_words];
+      if (a.mask_words > 1) mk1 = a.mask[(size_t)r * a.mask_words + 1];
     }
-  }
-  __syncwarp();
-  ok = mbar_wait(bar_o, 0, abort_flag);
-  tc_fence_after();
-  POSS_TRACE_POINT(3);
-  __syncthreads();                  // every half's sum and every group's maximum are in place
-  if (ok) {
-    // park O in global memory (it stays in L2): this warp's 32 query rows, output columns [32 cq, 32 cq + 32), the
-    // CTA's groups merged in key order (a group without keys accumulated nothing: it is left out, its TMEM columns
-    // are not read)
-    const int cq = warp >> 2;
-    const bool two = ng == 2 && group_keys(1) > 0;
-    const float m0 = grp_m[0][row], m1 = two ? grp_m[1][row] : NEG_BIG;
-    const float l0 = half_sum[0][0][row] + half_sum[1][0][row];
-    const float l1 = two ? half_sum[0][1][row] + half_sum[1][1][row] : 0.f;
-    const float ms = fmaxf(m0, m1);
-    const float c0 = ex2(m0 - ms), c1 = two ? ex2(m1 - ms) : 0.f;
-    const uint32_t t_o = t_s + o_col + (uint32_t)(cq * 32);
-    float* dst = a.part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * a.n_splits + split) * O_LD;
-    if (valid && cq == 0) *reinterpret_cast<float2*>(dst + D) = make_float2(ms, l0 * c0 + l1 * c1);
+    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+    float m_g0 = NEG_BIG, m_g1 = NEG_BIG, l_g0 = 0.f, l_g1 = 0.f;   // scaled maximum / row sum of the unit's two groups
+
+    for (int gi = 0; gi < n_g; ++gi) {
+      const int grp = group_of(gi);
+      const int key_g = grp * KG;
+      const int n_ch = (keys_of(grp) + 15) / 16;               // 16-key chunks of the group that hold keys
+      mbar_wait(bar_s(gi & 1), (uint32_t)((gi >> 1) & 1), abort_flag);
+      tc_fence_after();
+      POSS_TRACE_POINT(1);
+      // this thread's two chunks of scores; invisible keys become -inf: they lose every maximum and their 2^x is
+      // an exact zero
+      uint32_t sr[2][16];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int c = 2 * cq + j;
+        if (c < n_ch) {
+          tmem_ld16_async(t_lane + (uint32_t)((gi & 1) * KG + c * 16), sr[j]);
+          tmem_wait16(sr[j]);
+          const int key0 = key_g + c * 16;
+          if (key0 + 16 > a.n_all) {                           // the chunk reaches the tree slots or the end
+            // bit i = key0 + i is visible: 16 bits cut out of (all ones below n_all | the row's ancestor mask)
+            const int t0 = key0 - a.n_all;                     // tree slot of the chunk's first key; > -16
+            uint32_t vis;
+            if (t0 >= 64) vis = t0 >= 128 ? 0u : (uint32_t)(mk1 >> (t0 - 64));
+            else if (t0 > 48) vis = (uint32_t)(mk0 >> t0) | (uint32_t)(mk1 << (64 - t0));
+            else if (t0 >= 0) vis = (uint32_t)(mk0 >> t0);
+            else vis = ((uint32_t)mk0 << (-t0)) | ((1u << (-t0)) - 1u);
+            const int n_valid = a.total - key0;                // keys of the chunk that exist
+            if (n_valid < 16) vis &= (1u << (n_valid < 0 ? 0 : n_valid)) - 1u;
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (!((vis >> i) & 1u)) sr[j][i] = 0xff800000u;
+          }
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int i = 0; i < 16; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sr[j][i]));
+          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+        }
+      }
+      x_max[cq][row] = mx;
+      softmax_sync(1);
+      const float mraw = fmaxf(fmaxf(x_max[0][row], x_max[1][row]), fmaxf(x_max[2][row], x_max[3][row]));
+      // the scale is positive: the maximum of the scaled scores is the scaled maximum
+      const float ms = mraw == -INFINITY ? 0.f : mraw * a.scale_log2;
+      // P is one buffer: the previous group's second product must have read it
+      if (gi > 0) mbar_wait(bar_pv, (uint32_t)((gi - 1) & 1), abort_flag);
+      float ls = 0.f;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int c = 2 * cq + j;
+        if (c < n_ch) {
+          uint32_t hi[8], lo[8];
+          float l4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[j][i]), a.scale_log2, -ms));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[j][i + 1]), a.scale_log2, -ms));
+            l4[i & 3] += p0;
+            l4[(i & 3) + 1] += p1;
+            split_pack(p0, p1, hi[i >> 1], lo[i >> 1]);
+          }
+          ls += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+          // A operand of P V: k-block of 64 keys, row = query row (128 bytes), 16-byte pieces swizzled by row
+          const uint32_t line = (uint32_t)(c >> 2) * TILE + (uint32_t)row * 128u;
+          const uint32_t pc = (uint32_t)(c & 3) * 2u, sw = (uint32_t)(row & 7);
+          *reinterpret_cast<uint4*>(base_ptr + P_HI + line + ((pc ^ sw) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(base_ptr + P_HI + line + (((pc + 1) ^ sw) << 4)) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          *reinterpret_cast<uint4*>(base_ptr + P_LO + line + ((pc ^ sw) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(base_ptr + P_LO + line + (((pc + 1) ^ sw) << 4)) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
+      }
+      x_sum[cq][row] = ls;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P becomes visible to the tensor core
+      tc_fence_before();
+      mbar_arrive(bar_p);
+      softmax_sync(2);
+      POSS_TRACE_POINT(2);
+      {
+        const float mg = mraw == -INFINITY ? NEG_BIG : ms;
+        const float lg = (x_sum[0][row] + x_sum[1][row]) + (x_sum[2][row] + x_sum[3][row]);
+        if (gi & 1) { m_g1 = mg; l_g1 = lg; } else { m_g0 = mg; l_g0 = lg; }
+      }
+
+      if ((gi & 1) == 1 || gi == n_g - 1) {
+        // ---- the unit is complete: merge its groups in key order and park (m, l, O) in global memory (it stays in
+        // L2).  This thread: its query row, output columns [32 cq, 32 cq + 32).  (A unit whose second group holds
+        // no key accumulated nothing there: that accumulator is not read.)
+        const bool two = (gi & 1) == 1;
+        mbar_wait(bar_pv, (uint32_t)(gi & 1), abort_flag);
+        tc_fence_after();
+        POSS_TRACE_POINT(3);
+        const float m0 = m_g0, m1 = two ? m_g1 : NEG_BIG;
+        const float l0 = l_g0, l1 = two ? l_g1 : 0.f;
+        const float mu = fmaxf(m0, m1);
+        const float c0 = ex2(m0 - mu), c1 = two ? ex2(m1 - mu) : 0.f;
+        const int unit = walker + (gi >> 1) * a.n_walk;
+        const uint32_t t_o = t_lane + 2u * KG + (uint32_t)(cq * 32);
+        float* dst = a.part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * a.n_units + unit) * O_LD;
+        if (valid && cq == 0) *reinterpret_cast<float2*>(dst + D) = make_float2(mu, l0 * c0 + l1 * c1);
 #pragma unroll 1
-    for (int cc = 0; cc < 2; ++cc) {
-      uint32_t v0[16], v1[16];
-      tmem_ld16_async(t_o + (uint32_t)(cc * 16), v0);
-      if (two) tmem_ld16_async(t_o + (uint32_t)(D + cc * 16), v1);
-      tmem_wait16(v0);
-      if (two) tmem_wait16(v1);
-      float v[16];
+        for (int cc = 0; cc < 2; ++cc) {
+          uint32_t v0[16], v1[16];
+          tmem_ld16_async(t_o + (uint32_t)(cc * 16), v0);
+          if (two) tmem_ld16_async(t_o + (uint32_t)(D + cc * 16), v1);
+          tmem_wait16(v0);
+          if (two) tmem_wait16(v1);
+          float v[16];
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        v[j] = __uint_as_float(v0[j]) * c0;
-        if (two) v[j] += __uint_as_float(v1[j]) * c1;
-      }
-      if (valid) {
+          for (int j = 0; j < 16; ++j) {
+            v[j] = __uint_as_float(v0[j]) * c0;
+            if (two) v[j] += __uint_as_float(v1[j]) * c1;
+          }
+          if (valid) {
 #pragma unroll
-        for (int j = 0; j < 16; j += 4)
-          __stcg(reinterpret_cast<float4*>(dst + cq * 32 + cc * 16 + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+            for (int j = 0; j < 16; j += 4)
+              __stcg(reinterpret_cast<float4*>(dst + cq * 32 + cc * 16 + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_of);                                   // the accumulators may take the next unit
+        m_g0 = m_g1 = NEG_BIG;
+        l_g0 = l_g1 = 0.f;
       }
     }
+    if (a.n_clusters > 1) __threadfence();                     // this thread's parked values, before the arrival count
   }
 
   tc_fence_before();
@@ -380,44 +471,68 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   cluster_sync_all();
   POSS_TRACE_POINT(4);
 
-  // ---------------- merge over the cluster's CTAs, in key order: this CTA's share of the query rows.  The
-  // partials were written before the cluster barrier (release / acquire at cluster scope) and are read past L1.
-  {
-    const int ns = a.n_splits;
-    const int rank = (int)cluster_rank();
-    const int row_lo = rank * QT / ns, row_hi = (rank + 1) * QT / ns;
+  // ---------------- merge over ALL units, in key order: this cluster rank's share of the query rows.  Within a
+  // cluster the partials were written before the cluster barrier (release / acquire at cluster scope); with several
+  // clusters the rank's last arriver merges (fence + counter), and nobody waits.  Partials are read past L1.
+  const int rank = (int)cluster_rank();
+  bool do_merge = true;
+  if (a.n_clusters > 1) {
+    if (threadIdx.x == 0) {
+      int* cnt = a.arrivals + ((size_t)(kvh * gridDim.z + qtile) * MAX_CLUSTER + rank);
+      __threadfence();
+      const int prev = atomicAdd(cnt, 1);
+      const int last = prev == a.n_clusters - 1;
+      if (last) *cnt = 0;                                      // every other arrival is in: ready for the next launch
+      __threadfence();
+      s_last = last;
+    }
+    __syncthreads();
+    do_merge = s_last != 0;
+  }
+  if (do_merge) {
+    const int nu = a.n_units;
+    const int row_lo = rank * QT / a.cluster, row_hi = (rank + 1) * QT / a.cluster;
 #pragma unroll 1
     for (int item = threadIdx.x; item < (row_hi - row_lo) * 16; item += N_THREADS) {
       const int rr = row_lo + (item >> 4), cg = (item & 15) * 8;
       const int qj = qtile * QT + rr;
       if (qj >= a.n_q) continue;
       const int rj = qj / a.G, gj = qj - rj * a.G;
-      const float* src = a.part + (((size_t)rj * a.Hq + kvh * a.G + gj) * ns) * O_LD;
-      // every load is in flight before the first use
-      float2 ml[MAX_SPLITS];
-      float4 x0[MAX_SPLITS], x1[MAX_SPLITS];
-#pragma unroll
-      for (int j = 0; j < MAX_SPLITS; ++j) {
-        if (j < ns) {
-          ml[j] = __ldcg(reinterpret_cast<const float2*>(src + (size_t)j * O_LD + D));
-          x0[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)j * O_LD + cg));
-          x1[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)j * O_LD + cg + 4));
-        }
-      }
+      const float* src = a.part + (((size_t)rj * a.Hq + kvh * a.G + gj) * nu) * O_LD;
+      // the maximum over all units first (every load in flight before the first use, in batches)
       float mm = NEG_BIG;
+#pragma unroll 1
+      for (int u0 = 0; u0 < nu; u0 += 8) {
+        float mv[8];
 #pragma unroll
-      for (int j = 0; j < MAX_SPLITS; ++j)
-        if (j < ns) mm = fmaxf(mm, ml[j].x);
+        for (int j = 0; j < 8; ++j)
+          mv[j] = u0 + j < nu ? __ldcg(src + (size_t)(u0 + j) * O_LD + D) : NEG_BIG;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mm = fmaxf(mm, mv[j]);
+      }
       float ll = 0.f, acc[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll 1
+      for (int u0 = 0; u0 < nu; u0 += 6) {
+        float2 ml[6];
+        float4 x0[6], x1[6];
 #pragma unroll
-      for (int j = 0; j < MAX_SPLITS; ++j) {
-        if (j < ns) {
-          const float c = ex2(ml[j].x - mm);
-          ll += ml[j].y * c;
-          acc[0] += x0[j].x * c; acc[1] += x0[j].y * c; acc[2] += x0[j].z * c; acc[3] += x0[j].w * c;
-          acc[4] += x1[j].x * c; acc[5] += x1[j].y * c; acc[6] += x1[j].z * c; acc[7] += x1[j].w * c;
+        for (int j = 0; j < 6; ++j) {
+          if (u0 + j < nu) {
+            ml[j] = __ldcg(reinterpret_cast<const float2*>(src + (size_t)(u0 + j) * O_LD + D));
+            x0[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg));
+            x1[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg + 4));
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 6; ++j) {
+          if (u0 + j < nu) {
+            const float c = ex2(ml[j].x - mm);
+            ll += ml[j].y * c;
+            acc[0] += x0[j].x * c; acc[1] += x0[j].y * c; acc[2] += x0[j].z * c; acc[3] += x0[j].w * c;
+            acc[4] += x1[j].x * c; acc[5] += x1[j].y * c; acc[6] += x1[j].z * c; acc[7] += x1[j].w * c;
+          }
         }
       }
       const float inv = 1.f / ll;
@@ -434,28 +549,30 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   POSS_TRACE_POINT(5);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+  if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
   if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, (int)POSS_E_TIMEOUT);
 }
 
 }  // namespace
 
 // ------------------------------------------------------------------ host side
-// The cut of the keys: a function of the key count alone.  Two 128-key groups per CTA (one when there are no more
-// than 128 keys), as many CTAs as the keys need.
-bool tree_attention_tc_plan(int total, int* cta_keys, int* n_ctas) {
-  if (total < 1 || total > MAX_SPLITS * MAX_CTA_KEYS) return false;
-  *cta_keys = total <= KG ? KG : MAX_CTA_KEYS;
-  *n_ctas = (total + *cta_keys - 1) / *cta_keys;
+// The cut of the keys: a function of the key count alone.  Groups of 128 keys from key 0 on, two per unit; one
+// partial per unit.
+bool tree_attention_tc_plan(int total, int* unit_keys, int* n_units) {
+  if (total < 1 || total > MAX_UNITS * UNIT_KEYS) return false;
+  *unit_keys = total <= KG ? KG : UNIT_KEYS;
+  *n_units = (total + UNIT_KEYS - 1) / UNIT_KEYS;
   return true;
 }
+
+size_t tree_attention_tc_arrival_ints() { return (size_t)MAX_ARRIVAL_SETS * MAX_CLUSTER; }
 
 bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out) {
   if (a.d != D || a.Hkv < 1 || a.Hq % a.Hkv) return false;
   const int G = a.Hq / a.Hkv;
   if (G > QT || QT % G) return false;
   const int total = a.n_all + a.n_tree;
-  if (a.rows < 1 || total < 1 || total > MAX_SPLITS * MAX_CTA_KEYS) return false;
+  if (a.rows < 1 || total < 1 || total > MAX_UNITS * UNIT_KEYS) return false;
   if (a.mask_words > 2 || a.n_tree > 128) return false;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |
        reinterpret_cast<uintptr_t>(out)) & 15)
@@ -468,7 +585,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
-                              const bf16* vc, float* part, bf16* out, int32_t* status) {
+                              const bf16* vc, float* part, size_t part_floats, int* arrivals, bf16* out,
+                              int32_t* status) {
   if (!tree_attention_tc_supported(a, q, kc, vc, out) || !status || !part || (reinterpret_cast<uintptr_t>(part) & 15))
     return false;
   EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(tc_encode_fn(cache));
@@ -478,20 +596,32 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   memset(&k, 0, sizeof(k));
   k.rows = a.rows; k.Hq = a.Hq; k.G = G; k.n_q = a.rows * G;
   k.n_all = a.n_all; k.n_tree = a.n_tree; k.total = total;
-  if (!tree_attention_tc_plan(total, &k.cta_keys, &k.n_splits)) return false;
+  int unit_keys = 0;
+  if (!tree_attention_tc_plan(total, &unit_keys, &k.n_units)) return false;
+  if ((size_t)a.rows * a.Hq * k.n_units * O_LD > part_floats) return false;
+  // Walkers per (KV head, query tile): as many as the units, as long as the whole grid still fits the SMs at one
+  // CTA each; more than eight of them form several clusters.  (Scheduling only: the result does not depend on it.)
+  const int q_tiles = (k.n_q + QT - 1) / QT;
+  const int sets = a.Hkv * q_tiles;
+  int walk = tc_sm_count(cache) / sets;
+  if (walk < 1) walk = 1;
+  if (walk > k.n_units) walk = k.n_units;
+  if (walk > MAX_CLUSTER && (!arrivals || sets > MAX_ARRIVAL_SETS)) walk = MAX_CLUSTER;
+  if (walk > MAX_CLUSTER) {
+    k.n_clusters = walk / MAX_CLUSTER;
+    k.cluster = MAX_CLUSTER;
+  } else {
+    k.n_clusters = 1;
+    k.cluster = walk;
+  }
+  k.n_walk = k.cluster * k.n_clusters;
   k.mask = a.mask; k.mask_words = a.mask_words;
   k.scale_log2 = a.scale * 1.4426950408889634f;
-  k.part = part; k.out = out; k.status = status;
+  k.part = part; k.arrivals = arrivals; k.out = out; k.status = status;
   k.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
-  const uint32_t k_half = (uint32_t)k.cta_keys * 128u, p_bytes = 2u * (uint32_t)(k.cta_keys / 64) * HALF_TILE;
-  uint32_t region_a = 2u * HALF_TILE + 2u * k_half;
-  if (region_a < p_bytes) region_a = p_bytes;
-  k.region_a_bytes = region_a;                       // a multiple of 1024 either way
-  size_t smem = (size_t)region_a + 2u * k_half + 1024u;
-  // At least half an SM's shared memory, so that two of these CTAs never share an SM: each holds up to all
-  // of the SM's TMEM until its whole cluster has merged, and CTAs of two clusters queued behind each other's
-  // TMEM on two SMs would wait forever.
-  if (smem < 116u * 1024u) smem = 116u * 1024u;
+  // More than half an SM's shared memory, so that two of these CTAs never share an SM: each holds all of the SM's
+  // TMEM until its whole cluster has merged.
+  const size_t smem = (size_t)SMEM_TILES + 1024u;
 
   // The maps carry the call's extents (rows, key count): rows past them are filled with zeros by the copy.
   CUtensorMap mq, mk, mv;
@@ -508,7 +638,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   for (int i = 0; i < 2; ++i) {
     cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)total, (cuuint64_t)a.Hkv};
     cuuint64_t gstr[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.cap * D * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)k.cta_keys, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)KG, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     if (encode(i ? &mv : &mk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(i ? vc : kc), gdim, gstr, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -524,7 +654,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(k.n_splits, a.Hkv, (k.n_q + QT - 1) / QT);
+  cfg.gridDim = dim3(k.n_walk, a.Hkv, q_tiles);
   cfg.blockDim = dim3(N_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = L.stream;
@@ -532,15 +662,15 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   at[1].id = cudaLaunchAttributeClusterDimension;
-  at[1].val.clusterDim.x = k.n_splits;
+  at[1].val.clusterDim.x = k.cluster;
   at[1].val.clusterDim.y = 1;
   at[1].val.clusterDim.z = 1;
   cfg.attrs = at;
   cfg.numAttrs = 2;
   // A cluster shape the device does not take is reported at launch, before anything runs: remember it and
   // leave the call to the split-KV kernels.
-  static PerDeviceFlags refused[MAX_SPLITS + 1];
-  bool* ref = refused[k.n_splits].current();
+  static PerDeviceFlags refused[MAX_CLUSTER + 1];
+  bool* ref = refused[k.cluster].current();
   if (ref && *ref) return false;
   if (cudaLaunchKernelEx(&cfg, k_attn_tc, mq, mk, mv, k) != cudaSuccess) {
     cudaGetLastError();

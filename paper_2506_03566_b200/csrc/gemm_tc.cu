@@ -622,7 +622,7 @@ struct TcGemmPlanCache {
   EncodeTiledFn encode = nullptr;
   bool tried = false, attr_set = false;
   int inject = 0;          // launches left whose first activation tile is withheld (wait-expiry test hook)
-  int grid = 0;
+  int grid = 0, sms = 0;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
 };
 
@@ -633,11 +633,13 @@ TcGemmPlanCache* tc_plan_cache_create() {
   if (sms < 1) sms = 148;
   // The grid is a property of the device, not of a call: the work split (and with it the order in
   // which a tile's partial sums are added) must not change from call to call.
+  c->sms = sms;
   c->grid = sms;                       // one persistent CTA per SM
   if (c->grid > TC_MAX_GRID) c->grid = TC_MAX_GRID;
   return c;
 }
 void tc_plan_cache_destroy(TcGemmPlanCache* p) { delete p; }
+int tc_sm_count(const TcGemmPlanCache* c) { return c->sms; }
 void tc_inject_lost_load(TcGemmPlanCache* c, int launches) { c->inject = launches < 0 ? 0 : launches; }
 bool tc_take_injection(TcGemmPlanCache* c) {
   if (c->inject <= 0) return false;

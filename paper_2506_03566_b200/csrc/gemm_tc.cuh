@@ -16,13 +16,19 @@ bool tc_gemm_clear_counters(void* scratch, cudaStream_t stream);
 // the driver's tensor-map encoder (cuTensorMapEncodeTiled), resolved once; NULL when it cannot be had
 void* tc_encode_fn(TcGemmPlanCache*);
 
-// Tree attention on tcgen05 (bf16, head dimension 128, at most 2048 keys).  `part` holds one partial per
-// (row, head, 256 keys): rows * Hq * 8 * 132 floats at most, which the split-KV kernels' buffer always covers.
+// number of SMs of the device the cache was created on (= the persistent grid of the matrix products)
+int tc_sm_count(const TcGemmPlanCache*);
+
+// Tree attention on tcgen05 (bf16, head dimension 128, at most 10240 keys).  `part` (part_floats floats) holds one
+// partial of 132 floats per (row, head, 256-key unit); `arrivals` (tree_attention_tc_arrival_ints() ints, zero
+// between launches, may be NULL) lets more than eight CTAs share one (KV head, query tile).
 // Returns false, having launched nothing, when the call is not covered; errors of a launch go to *status.
-bool tree_attention_tc_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster);
+bool tree_attention_tc_plan(int total_keys, int* keys_per_unit, int* n_units);
+size_t tree_attention_tc_arrival_ints();
 bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out);
 bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
-                              const bf16* vc, float* part, bf16* out, int32_t* status);
+                              const bf16* vc, float* part, size_t part_floats, int* arrivals, bf16* out,
+                              int32_t* status);
 
 // true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 8, ...)
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);

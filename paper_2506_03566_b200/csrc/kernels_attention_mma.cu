@@ -1,5 +1,6 @@
-// Split-KV tree attention on tensor cores (bf16): the production kernel of poss_tree_attention and of
-// every draft step and target layer.
+// Split-KV tree attention on mma.sync tensor cores (bf16): the kernel for what the tcgen05 kernel does not take
+// (head dimension 64, more than 10240 keys, callers without a context workspace) and the comparison partner of
+// the tcgen05 kernel in the tests.
 //
 // Geometry.  For one KV head the G = Hq/Hkv query heads of all tree rows form one matrix Q' of
 // rows*G query rows (query row qi = r*G + g).  A block owns (key split, KV head, 64 query rows); each of

@@ -12,7 +12,7 @@ namespace {
 
 constexpr int R = POSS_MAX_ROWS;
 constexpr int KMAX = POSS_MAX_TOPK;
-constexpr int ATTN_MAX_SPLITS = 32;
+constexpr int ATTN_MAX_SPLITS = 48;     // sizes the attention partials: 47 units of 256 keys on the tcgen05 kernel
 
 struct Bump {
   size_t off = 0;
@@ -33,6 +33,8 @@ struct Buffers {
   float* ptmp;        // [R][max(H, (Hq+2Hkv)d)] product of a GEMM that did not leave split-K partials
   void* q;            // [R][Hq d] act
   float* attn_part;
+  size_t attn_part_floats;
+  int* attn_arrivals;    // arrival counters of the tcgen05 attention (several clusters per KV head), zero between launches
   void* o;            // [R][Hq d] act
   float* h1;          // [R][H]
   void* u;            // [R][H] act
@@ -124,7 +126,9 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.qkv = bp.take<float>(R * (qd + 2 * kd), 4);
   b.ptmp = bp.take<float>(R * (H > qd + 2 * kd ? H : qd + 2 * kd), 4);
   b.q = bp.take<void>(R * qd, es);
-  b.attn_part = bp.take<float>(attn_partial_floats(R, c.n_q_heads, c.head_dim, ATTN_MAX_SPLITS), 4);
+  b.attn_part_floats = attn_partial_floats(R, c.n_q_heads, c.head_dim, ATTN_MAX_SPLITS);
+  b.attn_part = bp.take<float>(b.attn_part_floats, 4);
+  b.attn_arrivals = bp.take<int>(tree_attention_tc_arrival_ints(), 4);
   b.o = bp.take<void>(R * qd, es);
   b.h1 = bp.take<float>(R * H, 4);
   b.u = bp.take<void>(R * H, es);
@@ -474,7 +478,9 @@ void Impl<T>::attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc
 }
 template <>
 void Impl<bf16>::attention(const AttnArgs& aa, const bf16* q, const bf16* kc, const bf16* vc, bf16* out) {
-  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, q, kc, vc, c->b.attn_part, out, c->b.status)) return;
+  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, q, kc, vc, c->b.attn_part, c->b.attn_part_floats,
+                                             c->b.attn_arrivals, out, c->b.status))
+    return;
   run_tree_attention<bf16>(L, aa, ATTN_MAX_SPLITS, q, kc, vc, c->b.attn_part, out);
 }
 
@@ -600,6 +606,8 @@ int poss_reset(poss_ctx* c, poss_stream stream) {
   // and of the top-k merge's blocks (both return to zero by themselves after a launch that ran to its end)
   if (!tc_gemm_clear_counters(c->b.tc_scratch, S(stream))) return POSS_E_CUDA;
   if (cudaMemsetAsync(c->b.merge_done, 0, sizeof(int) * 64, S(stream)) != cudaSuccess) return POSS_E_CUDA;
+  if (cudaMemsetAsync(c->b.attn_arrivals, 0, sizeof(int) * tree_attention_tc_arrival_ints(), S(stream)) != cudaSuccess)
+    return POSS_E_CUDA;
   return POSS_OK;
 }
 
@@ -919,12 +927,12 @@ int poss_debug_option(poss_ctx* c, int option, int value) {
   return POSS_OK;
 }
 
-int poss_attention_plan(int total_keys, int* keys_per_cta, int* ctas_per_cluster) {
-  if (!keys_per_cta || !ctas_per_cluster || total_keys < 1) return POSS_E_INVALID;
+int poss_attention_plan(int total_keys, int* keys_per_unit, int* n_units) {
+  if (!keys_per_unit || !n_units || total_keys < 1) return POSS_E_INVALID;
   int k = 0, n = 0;
   if (!tree_attention_tc_plan(total_keys, &k, &n)) return POSS_E_SHAPE;
-  *keys_per_cta = k;
-  *ctas_per_cluster = n;
+  *keys_per_unit = k;
+  *n_units = n;
   return POSS_OK;
 }
 

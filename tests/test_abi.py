@@ -73,18 +73,17 @@ def test_workspace_grows_with_the_model(lib):
 
 
 def test_attention_key_cut_depends_on_the_key_count_alone_and_sits_at_absolute_positions(lib):
-    """The tcgen05 attention cuts its keys into 128-key groups at absolute positions, two per CTA, at most eight CTAs
-    per cluster: every key count from 1 to 2048 is covered exactly once, the keys before any position fall into the
-    same groups whatever comes after them (what makes a tree's root row equal to its single-row decode bit for bit),
-    and counts past 2048 are reported as not covered."""
+    """The tcgen05 attention cuts its keys into 128-key groups at absolute positions, two per 256-key unit, one partial
+    per unit: every key count from 1 to 10240 is covered exactly once, the keys before any position fall into the
+    same groups and units whatever comes after them (what makes a tree's root row equal to its single-row decode bit
+    for bit), and counts past 10240 are reported as not covered."""
     k, n = C.c_int(), C.c_int()
     assert lib.poss_attention_plan(0, C.byref(k), C.byref(n)) == 1
     assert lib.poss_attention_plan(5, None, C.byref(n)) == 1
-    for total in range(1, 2049):
+    for total in list(range(1, 2600)) + [4096, 4097, 8192, 8193, 8273, 10239, 10240]:
         assert lib.poss_attention_plan(total, C.byref(k), C.byref(n)) == 0
-        assert k.value in (128, 256) and 1 <= n.value <= 8
-        assert (n.value - 1) * k.value < total <= n.value * k.value      # no empty CTA, nothing left out
-        assert k.value % 128 == 0                                        # groups of 128 keys from key 0 on
+        assert k.value == (128 if total <= 128 else 256) and 1 <= n.value <= 40
+        assert (n.value - 1) * 256 < total <= n.value * 256              # no empty unit, nothing left out
     k.value, n.value = -1, -1
-    assert lib.poss_attention_plan(2049, C.byref(k), C.byref(n)) == 2     # POSS_E_SHAPE
+    assert lib.poss_attention_plan(10241, C.byref(k), C.byref(n)) == 2    # POSS_E_SHAPE
     assert (k.value, n.value) == (-1, -1)

@@ -104,11 +104,15 @@ def test_tree_attention_matches_oracle(name, rows, P_len, Hq, Hkv, d):
 @pytest.mark.parametrize("rows,P_len,Hq,Hkv", [
     (1, 0, 8, 8), (16, 0, 8, 2), (5, 123, 8, 1), (5, 124, 8, 1), (61, 195, 16, 4), (61, 196, 16, 4),
     (128, 128, 4, 1), (128, 64, 8, 1), (40, 1987, 8, 2), (61, 1987, 8, 8), (61, 1988, 8, 2),
+    (61, 4035, 8, 1), (10, 2100, 40, 40), (10, 8262, 32, 8), (10, 8262, 8, 1), (81, 8192, 8, 8), (128, 10112, 4, 4),
+    (1, 10239, 8, 8), (70, 5000, 16, 2),
 ])
 def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv):
     """Head dimension 128 (the tcgen05 kernel): key counts of 1 and 16, around the 128-key groups (128 / 129), the
-    256-key blocks of a CTA (256 / 257) and the 2048-key limit (2027, 2048; at 2049 the split-KV kernels take the
-    call); GQA groups of 1, 4 and 8; one to eight query tiles; one and two mask words."""
+    256-key units (256 / 257), 2048 / 2049 keys (where a (KV head, query tile) starts to be walked by CTAs that take
+    several units each), 4096, the long-prefix draft and target shapes (8272 / 8273 keys: more than eight walkers, i.e.
+    several clusters and the arrival counters) and the 10240-key limit; GQA groups of 1, 4 and 8; multi-head attention
+    with 40 KV heads; one to eight query tiles; one and two mask words."""
     d = 128
     cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
     P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
@@ -125,8 +129,8 @@ def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv
 
 
 def test_tensor_core_tree_attention_on_random_shapes():
-    """24 seeded random shapes at head dimension 128 (1..64 rows, prefix 0..1500, 1..8 KV heads, GQA 1..8, cache
-    capacity with and without slack, random trees and chains) against the oracle."""
+    """24 seeded random shapes at head dimension 128 (1..64 rows, prefix 0..1500 and, every fourth trial, up to 9000;
+    1..8 KV heads, GQA 1..8, cache capacity with and without slack, random trees and chains) against the oracle."""
     rng = np.random.default_rng(2024)
     d = 128
     ctxs = {}
@@ -135,6 +139,8 @@ def test_tensor_core_tree_attention_on_random_shapes():
         Hq = Hkv * G
         rows = int(rng.integers(1, 65))
         P_len = int(rng.integers(0, 1501))
+        if trial % 4 == 3:
+            P_len = int(rng.integers(1500, 9001))
         cap = P_len + rows + int(rng.integers(0, 9))
         cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
         if (Hq, Hkv) not in ctxs:
@@ -153,14 +159,15 @@ def test_tensor_core_tree_attention_on_random_shapes():
 def test_tree_root_row_equals_its_single_row_decode_bitwise():
     """The property the lossless loop rests on: a token whose visible keys are the prefix and itself gets the same
     attention output, bit for bit, as the root of a 61-row tree pass and as a single decoded row, also where the
-    two calls cut their keys into different numbers of blocks (prefix 1000: 1061 against 1001 keys)."""
+    two calls cut their keys into different numbers of units and deal them to different numbers of CTAs (prefix 1000:
+    1061 against 1001 keys; prefix 2040: 9 units on walkers that take two of them against 8 units)."""
     Hq, Hkv, d, rows = 32, 8, 128, 61
     cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
     P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
     scale = 1.0 / math.sqrt(d)
     tree = po.pack_mask(po.ancestor_matrix(ps.random_tree_parents(13, rows)))
     one = po.pack_mask(po.ancestor_matrix(po.chain_parents(1)))
-    for P_len in (0, 100, 250, 1000, 1023, 1980):
+    for P_len in (0, 100, 250, 1000, 1023, 1980, 2040, 4090, 8190):
         q, kv = ps.make_attention_case(14 + P_len, rows, Hq, Hkv, d, P_len, P_len + rows + 2, cfg.dtype)
         full = pu.np_of(P.poss_tree_attention(dev(q), dev(kv), P_len, torch.from_numpy(tree.view(np.int64)).cuda(), scale))
         single = pu.np_of(P.poss_tree_attention(dev(q[:1]), dev(kv), P_len, torch.from_numpy(one.view(np.int64)).cuda(), scale))
