@@ -57,7 +57,8 @@ enum { POSS_FP32 = 0, POSS_BF16 = 1 };
 /* Compile-time limits of the kernels. */
 enum { POSS_MAX_ROWS = 128,      /* rows of any one matrix product (pending + current, or tree rows) */
        POSS_MAX_TOPK = 16,
-       POSS_MAX_DEPTH = 16 };
+       POSS_MAX_DEPTH = 16,
+       POSS_MAX_BATCH = 16 };    /* sequences of one batched draft round */
 
 typedef struct poss_ctx poss_ctx;
 typedef void* poss_stream;       /* a cudaStream_t */
@@ -74,6 +75,7 @@ typedef struct {
                                     prefix_len + n_new + (depth-1)*topk of them             */
   int n_target_layers;           /* 0 = drafter only */
   int target_kv_slots;           /* slots per target layer cache */
+  int max_batch;                 /* sequences per poss_draft_round_batched call (0 or 1: single rounds only) */
 } poss_config;
 
 /* One decoder layer.  fc_w [H][2H]: columns [0,H) multiply the token embedding, [H,2H) the
@@ -126,6 +128,25 @@ POSS_API int poss_draft_round(poss_ctx* ctx, void* draft_kv, int prefix_len,
                      int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                      int32_t* out_depth, uint64_t* out_anc_mask, int32_t* out_n_nodes,
                      poss_stream stream);
+
+/* One draft phase for `batch` independent sequences at once (the paper measures decoding speed as throughput
+ * against vanilla decoding, Section 4.1 "Metrics"; at one sequence every matrix product of a draft step streams its
+ * weights for at most 64 rows, so drafting for B sequences in one pass pays each step's weights once for B trees).
+ * Every sequence is drafted exactly as by poss_draft_round -- the result of sequence b equals, bit for bit, that of a
+ * single-sequence call on its inputs -- and the sequences share depth, topk and total_tokens.
+ * h_draft_kv: HOST array of `batch` device pointers, one cache set [S][2][n_kv_heads][draft_kv_slots][head_dim]
+ * per sequence; h_prefix_len, h_n_new: HOST int[batch].  new_tokens int32[sum n_new] and new_features
+ * [sum n_new][H]: the sequences' verified pairs one after the other (each sequence's last pair is its root).
+ * Outputs as in poss_draft_round with a leading batch dimension: tokens, parents, depth int32[batch][total+1],
+ * scores float[batch][total+1], anc_mask uint64[batch][total+1][ceil((total+1)/64)], n_nodes int32[batch].
+ * The stacked rows of every step (all sequences' pending and current rows) must fit POSS_MAX_ROWS and batch must
+ * not exceed the context's max_batch, else POSS_E_CAPACITY.  Errors: INVALID, CAPACITY. */
+POSS_API int poss_draft_round_batched(poss_ctx* ctx, int batch, void* const* h_draft_kv, const int* h_prefix_len,
+                             const int32_t* new_tokens, const void* new_features, const int* h_n_new,
+                             int depth, int topk, int total_tokens,
+                             int32_t* out_tokens, int32_t* out_parents, float* out_scores,
+                             int32_t* out_depth, uint64_t* out_anc_mask, int32_t* out_n_nodes,
+                             poss_stream stream);
 
 /* Tree-masked attention: every draft token attends to the committed context and to its own path in the draft
  * tree only, which is what lets the target check all draft tokens in one parallel pass (Section 2.1, the

@@ -23,6 +23,10 @@ extern "C" {
  * by the rerank, ascending. */
 POSS_API int poss_draft_trace(poss_ctx* ctx, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores,
                      int32_t* frontier, float* step_features, int32_t* selected, poss_stream stream);
+/* The same for sequence `seq` of the last batched draft round (poss_draft_trace is sequence 0). */
+POSS_API int poss_draft_trace_seq(poss_ctx* ctx, int seq, int32_t* cand_tokens, int32_t* cand_parents,
+                         float* cand_scores, int32_t* frontier, float* step_features, int32_t* selected,
+                         poss_stream stream);
 
 /* Device-time bracketing of the draft steps' stages, for roofline reporting.  mode 0: off (also switches the timeline
  * recording below off); mode 1: the LM-head

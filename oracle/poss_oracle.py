@@ -422,6 +422,14 @@ def draft_round(cfg, w, draft_kv, prefix_len, new_tokens, new_features, depth, t
     return res
 
 
+def draft_round_batched(cfg, w, draft_kvs, prefix_lens, new_tokens, new_features, depth, topk, total, num: Num):
+    """Drafting for several independent sequences in one call: by definition every sequence is drafted on its own
+    (its own caches, prefix length and verified pairs); nothing couples them.  Speed is measured as throughput
+    against vanilla decoding (Section 4.1), which is what batching the sequences serves."""
+    return [draft_round(cfg, w, draft_kvs[b], prefix_lens[b], new_tokens[b], new_features[b], depth, topk, total, num)
+            for b in range(len(draft_kvs))]
+
+
 def rerank(cand_tok, cand_parent, cand_score, cand_level, root_tok, total, selected=None) -> DraftResult:
     """Keep the `total` best candidates by cumulative log-prob (ties -> lower flat index), list them
     in creation order behind the root, remap parents, and build the packed ancestor masks."""

@@ -39,7 +39,7 @@ class poss_config(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("hidden", "n_q_heads", "n_kv_heads", "head_dim", "ffn", "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
                [(n, C.c_int) for n in ("dtype", "n_specialists", "positions_per_specialist", "max_depth", "max_topk",
-                                       "max_total", "draft_kv_slots", "n_target_layers", "target_kv_slots")]
+                                       "max_total", "draft_kv_slots", "n_target_layers", "target_kv_slots", "max_batch")]
 
 
 LAYER_FIELDS = ("fc_w", "fc_b", "norm_in", "wq", "wk", "wv", "wo", "norm_post", "w_gate", "w_up", "w_down")
@@ -64,7 +64,11 @@ EXPORTS = {
     "poss_draft_round": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                    C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p]),
+    "poss_draft_round_batched": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_int), C.c_void_p,
+                                           C.c_void_p, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "poss_draft_trace": (C.c_int, [C.c_void_p] * 8),
+    "poss_draft_trace_seq": (C.c_int, [C.c_void_p, C.c_int] + [C.c_void_p] * 7),
     "poss_tree_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                       C.c_float, C.c_void_p, C.c_void_p]),
     "poss_verify_accept": (C.c_int, [C.c_void_p] * 6 + [C.c_int] + [C.c_void_p] * 6),
@@ -138,12 +142,12 @@ def to_device(a: np.ndarray | None, device="cuda"):
 
 
 def make_config(cfg, draft_kv_slots: int, target_kv_slots: int = 0, max_depth=None, max_topk=None,
-                max_total=None) -> poss_config:
+                max_total=None, max_batch: int = 1) -> poss_config:
     """cfg: any object with the model fields of the synthetic PossConfig."""
     return poss_config(cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                        float(cfg.rope_theta), float(cfg.rms_eps), POSS_BF16 if cfg.dtype == "bf16" else POSS_FP32,
                        cfg.S, cfg.n, max_depth or cfg.depth, max_topk or cfg.topk, max_total or cfg.total,
-                       int(draft_kv_slots), cfg.n_target_layers, int(max(target_kv_slots, 1)))
+                       int(draft_kv_slots), cfg.n_target_layers, int(max(target_kv_slots, 1)), int(max_batch))
 
 
 class Poss:
@@ -237,7 +241,31 @@ class Poss:
                                          _ptr(out["n_nodes"]), _stream()), "poss_draft_round")
         return out
 
-    def poss_draft_trace(self, depth, topk, n_nodes):
+    def poss_draft_round_batched(self, draft_kvs, prefix_lens, new_tokens, new_features, n_news, depth, topk, total,
+                                 out=None):
+        """draft_kvs: list of per-sequence cache tensors; prefix_lens, n_news: lists of ints; new_tokens /
+        new_features: the sequences' verified pairs one after the other.  Returns dict of device tensors with a
+        leading batch dimension."""
+        B = len(draft_kvs)
+        if out is None:
+            words = (total + 1 + 63) // 64
+            dev = "cuda"
+            out = {"tokens": torch.empty((B, total + 1), dtype=torch.int32, device=dev),
+                   "parents": torch.empty((B, total + 1), dtype=torch.int32, device=dev),
+                   "scores": torch.empty((B, total + 1), dtype=torch.float32, device=dev),
+                   "depth": torch.empty((B, total + 1), dtype=torch.int32, device=dev),
+                   "anc_mask": torch.empty((B, total + 1, words), dtype=torch.int64, device=dev),
+                   "n_nodes": torch.empty(B, dtype=torch.int32, device=dev)}
+        kvp = (C.c_void_p * B)(*[_ptr(k) for k in draft_kvs])
+        pl = (C.c_int * B)(*[int(p) for p in prefix_lens])
+        nn = (C.c_int * B)(*[int(n) for n in n_news])
+        _check(self.lib.poss_draft_round_batched(self.ctx, B, kvp, pl, _ptr(new_tokens), _ptr(new_features), nn, depth,
+                                                 topk, total, _ptr(out["tokens"]), _ptr(out["parents"]),
+                                                 _ptr(out["scores"]), _ptr(out["depth"]), _ptr(out["anc_mask"]),
+                                                 _ptr(out["n_nodes"]), _stream()), "poss_draft_round_batched")
+        return out
+
+    def poss_draft_trace(self, depth, topk, n_nodes, seq=None):
         H = self.config.hidden
         nc = topk + (depth - 1) * topk * topk
         dev = "cuda"
@@ -247,9 +275,14 @@ class Poss:
              "frontier": torch.empty((max(depth - 1, 1), topk), dtype=torch.int32, device=dev),
              "step_features": torch.zeros((depth, topk, H), dtype=torch.float32, device=dev),
              "selected": torch.empty(max(n_nodes - 1, 1), dtype=torch.int32, device=dev)}
-        _check(self.lib.poss_draft_trace(self.ctx, _ptr(t["cand_tokens"]), _ptr(t["cand_parents"]),
-                                         _ptr(t["cand_scores"]), _ptr(t["frontier"]), _ptr(t["step_features"]),
-                                         _ptr(t["selected"]), _stream()), "poss_draft_trace")
+        if seq is None:
+            _check(self.lib.poss_draft_trace(self.ctx, _ptr(t["cand_tokens"]), _ptr(t["cand_parents"]),
+                                             _ptr(t["cand_scores"]), _ptr(t["frontier"]), _ptr(t["step_features"]),
+                                             _ptr(t["selected"]), _stream()), "poss_draft_trace")
+        else:
+            _check(self.lib.poss_draft_trace_seq(self.ctx, int(seq), _ptr(t["cand_tokens"]), _ptr(t["cand_parents"]),
+                                                 _ptr(t["cand_scores"]), _ptr(t["frontier"]), _ptr(t["step_features"]),
+                                                 _ptr(t["selected"]), _stream()), "poss_draft_trace_seq")
         return t
 
     def poss_tree_attention(self, q, kv, prefix_len, anc_mask, scale, out=None):

@@ -86,24 +86,25 @@ template void launch_gemm_simt<bf16>(Launcher&, const bf16*, int, int, const Gem
 
 // ------------------------------------------------------------------ layer-input pairs [E[tok] ; feature]
 template <typename T>
-__global__ void __launch_bounds__(256) k_gather_x(StepRows s, const int32_t* new_tokens,
-                                                  const T* new_features,
-                                                  const int32_t* node_tok,
-                                                  const int32_t* node_prow, int Kmax,
-                                                  const T* fb, const T* embed, int H,
+__global__ void __launch_bounds__(256) k_gather_x(BatchRows s, const int32_t* new_tokens,
+                                                  const T* new_features, TreeState ts, int Kmax,
+                                                  const T* fb, int level_rows, const T* embed, int H,
                                                   T* X) {
   pdl_enter(POSS_K_GATHER_X);
   int m = blockIdx.x;
-  RowInfo r = row_info(s, m);
+  RowRef r = batch_row(s, m);
   int tok;
   const T* feat;
   if (r.level == 0) {
-    tok = new_tokens[r.j];
-    feat = new_features + (size_t)r.j * H;
+    const int at = s.tok_off[r.seq] + r.j;
+    tok = new_tokens[at];
+    feat = new_features + (size_t)at * H;
   } else {
-    tok = node_tok[r.level * Kmax + r.j];
-    int prow = node_prow[r.level * Kmax + r.j];
-    feat = fb + ((size_t)(r.level - 1) * Kmax + prow) * H;   // the parent's output feature
+    const TreeState t = tree_of(ts, r.seq);
+    tok = t.node_tok[r.level * Kmax + r.j];
+    int prow = t.node_prow[r.level * Kmax + r.j];
+    const int pmc = r.level == 1 ? 1 : s.K;                  // expanded rows per sequence at the parent's level
+    feat = fb + ((size_t)(r.level - 1) * level_rows + r.seq * pmc + prow) * H;   // the parent's output feature
   }
   const T* e = embed + (size_t)tok * H;
   T* x = X + (size_t)m * 2 * H;
@@ -127,16 +128,16 @@ __global__ void __launch_bounds__(256) k_gather_x(StepRows s, const int32_t* new
   }
 }
 template <typename T>
-void launch_gather_x(Launcher& L, StepRows s, const int32_t* new_tokens, const T* new_features,
-                     const TreeState& ts, int Kmax, const T* fb, const T* embed, int H, T* X) {
+void launch_gather_x(Launcher& L, const BatchRows& s, const int32_t* new_tokens, const T* new_features,
+                     const TreeState& ts, int Kmax, const T* fb, int level_rows, const T* embed, int H, T* X) {
   if (s.M <= 0) return;
-  launch_pdl(L, k_gather_x<T>, dim3(s.M), dim3(256), 0, s, new_tokens, new_features, ts.node_tok, ts.node_prow, Kmax,
-             fb, embed, H, X);
+  launch_pdl(L, k_gather_x<T>, dim3(s.M), dim3(256), 0, s, new_tokens, new_features, ts, Kmax, fb, level_rows, embed, H,
+             X);
 }
-template void launch_gather_x<float>(Launcher&, StepRows, const int32_t*, const float*, const TreeState&, int,
-                                     const float*, const float*, int, float*);
-template void launch_gather_x<bf16>(Launcher&, StepRows, const int32_t*, const bf16*, const TreeState&, int,
-                                    const bf16*, const bf16*, int, bf16*);
+template void launch_gather_x<float>(Launcher&, const BatchRows&, const int32_t*, const float*, const TreeState&, int,
+                                     const float*, int, const float*, int, float*);
+template void launch_gather_x<bf16>(Launcher&, const BatchRows&, const int32_t*, const bf16*, const TreeState&, int,
+                                    const bf16*, int, const bf16*, int, bf16*);
 
 template <typename T>
 __global__ void k_embed_rows(const int32_t* tokens, const T* embed, int H,
@@ -522,7 +523,7 @@ template void launch_splitk_swiglu<bf16>(Launcher&, const SplitKView&, int, int,
 // of every tile need only the launch parameters and are done before the predecessor is awaited.
 #define ROPE_ITEMS 256
 template <typename T>
-__global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, SplitKView qkv, T* kcache, T* vcache,
+__global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, SplitKView qkv, CachePtrs caches,
                                                                   T* qout) {
   __shared__ TileContrib tab[512];
   __shared__ __align__(16) float cs[64], sn[64];
@@ -561,18 +562,21 @@ __global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, Spl
     splitk_locate(qkv, col, &tile_lo, &t_lo);
     if (kind != 2) splitk_locate(qkv, col + half, &tile_hi, &t_hi);
   }
-  const bool vec = aligned16(kcache) && aligned16(vcache) && (a.q_rows == 0 || aligned16(qout));
-  __syncthreads();
-  pdl_sync(POSS_K_ROPE_APPEND);
-  int slot, pos;
+  int slot, pos, seq = 0;
   if (a.mode == 0) {
-    RowInfo r = row_info(a.s, m);
+    RowRef r = batch_row(a.s, m);
+    seq = r.seq;
     slot = row_slot(a.s, r);
     pos = row_pos(a.s, r);
   } else {
     slot = a.base + m;
-    pos = a.base + a.depth[m];
   }
+  T* kcache = reinterpret_cast<T*>(caches.k[seq]);
+  T* vcache = reinterpret_cast<T*>(caches.v[seq]);
+  const bool vec = aligned16(kcache) && aligned16(vcache) && (a.q_rows == 0 || aligned16(qout));
+  __syncthreads();
+  pdl_sync(POSS_K_ROPE_APPEND);
+  if (a.mode != 0) pos = a.base + a.depth[m];
   float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
   if (!item_thread) {
     const int jj = threadIdx.x - ROPE_ITEMS;
@@ -632,15 +636,15 @@ __global__ void __launch_bounds__(ROPE_ITEMS + 64) k_rope_append(RopeArgs a, Spl
   POSS_TRACE_POINT(2);
 }
 template <typename T>
-void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout) {
+void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, const CachePtrs& caches, T* qout) {
   if (a.rows <= 0) return;
   const int per_head = a.d / 8;
   const int n_items = (a.q_rows > 0 ? a.Hq * per_head : 0) + a.Hkv * per_head + a.Hkv * a.d / 4;
   launch_pdl(L, k_rope_append<T>, dim3(a.rows, (n_items + ROPE_ITEMS - 1) / ROPE_ITEMS), dim3(ROPE_ITEMS + 64), 0, a, qkv,
-             kcache, vcache, qout);
+             caches, qout);
 }
-template void launch_rope_append<float>(Launcher&, const RopeArgs&, const SplitKView&, float*, float*, float*);
-template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKView&, bf16*, bf16*, bf16*);
+template void launch_rope_append<float>(Launcher&, const RopeArgs&, const SplitKView&, const CachePtrs&, float*);
+template void launch_rope_append<bf16>(Launcher&, const RopeArgs&, const SplitKView&, const CachePtrs&, bf16*);
 
 // chain mask / depth for causal prefill chunks: row r sees rows 0..r of its chunk
 __global__ void k_chain_mask(uint64_t* mask, int32_t* depth, int rows) {

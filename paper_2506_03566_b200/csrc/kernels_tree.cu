@@ -315,19 +315,29 @@ __global__ void __launch_bounds__(128) k_topk_merge(int K, int n_lists, const fl
   __syncthreads();
   if (!s_is_last) return;
   __threadfence();
-  expand_block(ts, x, out_ids, out_logp, vals);      // vals is free now: K*K <= its size is checked by the host
+  for (int b = 0; b < x.batch; ++b) {                // vals is free now: Mc*K <= its size is checked by the host
+    expand_block(tree_of(ts, b), x, out_ids + (size_t)b * x.Mc * K, out_logp + (size_t)b * x.Mc * K, vals);
+    __syncthreads();
+  }
   if (threadIdx.x == 0) *done = 0;
 }
 
-// ------------------------------------------------------------------ the same for a draft step, in one block
-// A draft step has at most POSS_MAX_TOPK rows and is followed by the tree expansion, which needs every
-// row's result: one block of 1024 threads stages all partial lists in shared memory with 16-byte loads
-// (one round trip), warp r merges row r, and after one barrier the block expands the tree.  No second
-// kernel, no counter.
+// ------------------------------------------------------------------ the same for a draft step, in one block per sequence
+// A sequence's draft step has at most POSS_MAX_TOPK rows and is followed by the tree expansion, which needs
+// every row's result: one block of 1024 threads stages all partial lists of its sequence's rows in shared memory
+// with 16-byte loads (one round trip), warp r merges row r, and after one barrier the block expands the
+// sequence's tree.  No second kernel, no counter.  Block b: rows [b * rows, (b + 1) * rows), tree state b.
 __global__ void __launch_bounds__(1024) k_topk_merge_expand(int rows, int K, int n_lists, const float* pmax,
                                                             const float* psum, const float* pval,
                                                             const int32_t* pidx, int32_t* out_ids, float* out_logp,
-                                                            TreeState ts, ExpandArgs x) {
+                                                            TreeState ts_all, ExpandArgs x) {
+  {
+    const size_t row0 = (size_t)blockIdx.x * rows;
+    pmax += row0 * n_lists; psum += row0 * n_lists;
+    pval += row0 * n_lists * K; pidx += row0 * n_lists * K;
+    out_ids += row0 * K; out_logp += row0 * K;
+  }
+  const TreeState ts = tree_of(ts_all, blockIdx.x);
   extern __shared__ __align__(16) unsigned char me_smem[];
   const int per_row = n_lists * K;
   const int total = rows * per_row;
@@ -339,7 +349,9 @@ __global__ void __launch_bounds__(1024) k_topk_merge_expand(int rows, int K, int
   int* heads = reinterpret_cast<int*>(ssum + rows * n_lists);    // [rows][n_lists]
   pdl_enter(POSS_K_TOPK_MERGE_EXPAND);
   {
-    const int n4 = total / 4;
+    // 16-byte loads when this sequence's lists start on a 16-byte boundary, else element by element
+    const bool al = ((reinterpret_cast<uintptr_t>(pval) | reinterpret_cast<uintptr_t>(pidx)) & 15) == 0;
+    const int n4 = al ? total / 4 : 0;
     const float4* pv4 = reinterpret_cast<const float4*>(pval);
     const int4* pi4 = reinterpret_cast<const int4*>(pidx);
     for (int base = 0; base < n4; base += 1024 * 4) {
@@ -468,35 +480,40 @@ void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* p
   TreeState t;
   memset(&t, 0, sizeof(t));
   if (x && ts && x->enabled) { xa = *x; t = *ts; }
-  if (xa.enabled && rows <= POSS_MAX_TOPK) {
-    size_t total4 = ((size_t)rows * n_lists * K + 3) & ~(size_t)3;
-    size_t smem1 = total4 * 8 + (size_t)rows * n_lists * 12;
+  const int batch = xa.enabled && xa.batch > 0 ? xa.batch : 1;
+  xa.batch = batch;
+  if (xa.enabled && rows == batch * xa.Mc && xa.Mc <= POSS_MAX_TOPK) {
+    const int rows_seq = xa.Mc;
+    size_t total4 = ((size_t)rows_seq * n_lists * K + 3) & ~(size_t)3;
+    size_t smem1 = total4 * 8 + (size_t)rows_seq * n_lists * 12;
     if (smem1 < (size_t)xa.Mc * K * 4) smem1 = (size_t)xa.Mc * K * 4;
     if (smem1 <= 200 * 1024) {
-      static bool attr1_done = false;
-      if (!attr1_done) {
+      static PerDeviceFlags attr1_done;
+      bool* a1 = attr1_done.current();
+      if (!a1 || !*a1) {
         if (cudaFuncSetAttribute(k_topk_merge_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) !=
             cudaSuccess) {
           L.err = POSS_E_CUDA;
           return;
         }
-        attr1_done = true;
+        if (a1) *a1 = true;
       }
-      launch_pdl(L, k_topk_merge_expand, dim3(1), dim3(1024), smem1, rows, K, n_lists, pmax, psum, pval, pidx, out_ids,
-                 out_logp, t, xa);
+      launch_pdl(L, k_topk_merge_expand, dim3(batch), dim3(1024), smem1, rows_seq, K, n_lists, pmax, psum, pval, pidx,
+                 out_ids, out_logp, t, xa);
       return;
     }
   }
   size_t elems = (size_t)n_lists * K;
   if (xa.enabled && elems < (size_t)xa.Mc * K) elems = (size_t)xa.Mc * K;      // room for the expansion's scores
   size_t smem = elems * 8 + (size_t)n_lists * 4;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceFlags attr_done;
+  bool* a0 = attr_done.current();
+  if (!a0 || !*a0) {
     if (cudaFuncSetAttribute(k_topk_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
-    attr_done = true;
+    if (a0) *a0 = true;
   }
   if (smem > 100 * 1024) { L.err = POSS_E_CAPACITY; return; }
   launch_pdl(L, k_topk_merge, dim3(rows), dim3(128), smem, K, n_lists, pmax, psum, pval, pidx, out_ids, out_logp, t, xa,
@@ -507,13 +524,22 @@ void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* p
 // One block.  rank(c) = number of candidates that order before c; kept iff rank < total.  Kept
 // candidates are listed in flat (creation) order behind the root, so a parent always precedes its
 // children; level of flat index c is 1 for c < K, else 2 + (c - K) / K^2.
-__global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K, int total,
-                                                 const int32_t* root_tok,
+__global__ void __launch_bounds__(1024) k_rerank(TreeState ts_all, int n_cand, int K, int total, RerankBatch rb,
+                                                 const int32_t* new_tokens,
                                                  int32_t* out_tokens, int32_t* out_parents,
                                                  float* out_scores, int32_t* out_depth,
                                                  uint64_t* out_mask, int32_t* out_n_nodes) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ int wtot[32];
+  // block b = sequence b: its tree state, its root token, its slice of the outputs
+  const TreeState ts = tree_of(ts_all, blockIdx.x);
+  const int32_t* root_tok = new_tokens + rb.root_index[blockIdx.x];
+  {
+    const size_t o = (size_t)blockIdx.x * (total + 1);
+    out_tokens += o; out_parents += o; out_scores += o; out_depth += o;
+    out_mask += o * ((total + 1 + 63) / 64);
+    out_n_nodes += blockIdx.x;
+  }
   pdl_enter(POSS_K_RERANK);
   float* sc = reinterpret_cast<float*>(smem_raw);               // [n_cand]
   int* newidx = reinterpret_cast<int*>(sc + n_cand);            // [n_cand] node index or 0 if dropped
@@ -587,11 +613,11 @@ __global__ void __launch_bounds__(1024) k_rerank(TreeState ts, int n_cand, int K
   }
 }
 
-void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, int root_tok_index,
+void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, const RerankBatch& rb,
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
   size_t smem = (size_t)n_cand * 12;
-  launch_pdl(L, k_rerank, dim3(1), dim3(1024), smem, ts, n_cand, K, total, new_tokens + root_tok_index, out_tokens,
+  launch_pdl(L, k_rerank, dim3(rb.batch), dim3(1024), smem, ts, n_cand, K, total, rb, new_tokens, out_tokens,
              out_parents, out_scores, out_depth, out_mask, out_n_nodes);
 }
 

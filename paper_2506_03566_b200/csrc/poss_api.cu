@@ -71,8 +71,10 @@ struct poss_ctx {
   size_t esize;          // bytes of the context dtype
   int n_chunks;          // vocabulary chunks of the top-k kernels
   int n_cand_max;
+  int max_batch;         // sequences a batched draft round may hold
+  int level_rows;        // rows per level of fout / fb: max_batch * POSS_MAX_TOPK
   int64_t launches;
-  int last_depth, last_topk, last_nodes;
+  int last_depth, last_topk, last_nodes, last_batch;
   TcGemmPlanCache* tc;
   bool attn_tc;          // tree attention on the tcgen05 kernel where it covers the call
   bool swiglu_in_kernel; // gate/up product finished by the GEMM's own SwiGLU epilogue instead of the consumer kernel
@@ -109,6 +111,7 @@ bool config_ok(const poss_config* c, int* why) {
   if ((c->max_depth - 1) * c->max_topk > 128) return false;   // tree-slot mask is two 64-bit words
   if ((c->max_depth - 1) * c->max_topk + 1 > R) return false;
   if (c->vocab < c->max_topk) return false;
+  if (c->max_batch < 0 || c->max_batch > POSS_MAX_BATCH) return false;
   *why = POSS_OK;
   return true;
 }
@@ -118,6 +121,7 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   size_t H = c.hidden, F = c.ffn, V = c.vocab;
   size_t qd = (size_t)c.n_q_heads * c.head_dim, kd = (size_t)c.n_kv_heads * c.head_dim;
   int L = c.max_depth;
+  const size_t NB = c.max_batch > 1 ? c.max_batch : 1;
   *n_chunks = (int)((V + POSS_TOPK_CHUNK - 1) / POSS_TOPK_CHUNK);
   *n_cand_max = n_cand_of(c.max_depth, c.max_topk);
   b.X = bp.take<void>(R * 2 * H, es);
@@ -134,8 +138,8 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.u = bp.take<void>(R * H, es);
   b.gu = bp.take<float>(R * 2 * F, 4);
   b.act = bp.take<void>(R * F, es);
-  b.fout = bp.take<float>((size_t)L * KMAX * H, 4);
-  b.fb = bp.take<void>((size_t)L * KMAX * H, es);
+  b.fout = bp.take<float>((size_t)L * NB * KMAX * H, 4);
+  b.fb = bp.take<void>((size_t)L * NB * KMAX * H, es);
   b.hx = bp.take<float>(R * H, 4);
   b.tfeat = bp.take<float>(R * H, 4);
   b.logits = bp.take<float>(R * V, 4);
@@ -155,15 +159,18 @@ void layout(const poss_config& c, Bump& bp, Buffers& b, int* n_chunks, int* n_ca
   b.rope_inv = bp.take<double>(64, 8);
   b.tc_scratch = bp.take<void>(tc_gemm_scratch_bytes(), 1);
   b.timeline = bp.take<unsigned long long>(poss_trace::HEADER_WORDS + poss_trace::ROW_WORDS * poss_trace::MAX_ROWS, 8);
-  b.ts.cand_tok = bp.take<int32_t>(*n_cand_max, 4);
-  b.ts.cand_parent = bp.take<int32_t>(*n_cand_max, 4);
-  b.ts.cand_score = bp.take<float>(*n_cand_max, 4);
-  b.ts.node_tok = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
-  b.ts.node_prow = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
-  b.ts.node_cand = bp.take<int32_t>((size_t)(L + 1) * KMAX, 4);
-  b.ts.node_score = bp.take<float>((size_t)(L + 1) * KMAX, 4);
-  b.ts.node_mask = bp.take<uint64_t>((size_t)(L + 1) * KMAX * 2, 8);
-  b.ts.selected = bp.take<int32_t>(256, 4);
+  // tree state: one block per sequence of a batched round
+  b.ts.cand_cap = (*n_cand_max + 3) / 4 * 4;
+  b.ts.node_cap = (L + 1) * KMAX;
+  b.ts.cand_tok = bp.take<int32_t>(NB * b.ts.cand_cap, 4);
+  b.ts.cand_parent = bp.take<int32_t>(NB * b.ts.cand_cap, 4);
+  b.ts.cand_score = bp.take<float>(NB * b.ts.cand_cap, 4);
+  b.ts.node_tok = bp.take<int32_t>(NB * b.ts.node_cap, 4);
+  b.ts.node_prow = bp.take<int32_t>(NB * b.ts.node_cap, 4);
+  b.ts.node_cand = bp.take<int32_t>(NB * b.ts.node_cap, 4);
+  b.ts.node_score = bp.take<float>(NB * b.ts.node_cap, 4);
+  b.ts.node_mask = bp.take<uint64_t>(NB * b.ts.node_cap * 2, 8);
+  b.ts.selected = bp.take<int32_t>(NB * 256, 4);
 }
 
 inline cudaStream_t S(poss_stream s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -226,13 +233,13 @@ struct Impl {
                       c->b.merge_done);
   }
 
-  // fc + norm + K/V(+Q) projection + rotary + cache append for one batch of a specialist
-  void project_rows(const poss_layer_w& lw, const StepRows& s, const int32_t* new_tokens, const T* new_features,
-                    T* kcache, T* vcache, bool with_q) {
+  // fc + norm + K/V(+Q) projection + rotary + cache append for one stacked batch of a specialist
+  void project_rows(const poss_layer_w& lw, const BatchRows& s, const int32_t* new_tokens, const T* new_features,
+                    const CachePtrs& caches, bool with_q) {
     const poss_config& g = c->cfg;
     Buffers& b = c->b;
     int H = g.hidden, qd = g.n_q_heads * g.head_dim, kd = g.n_kv_heads * g.head_dim;
-    launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), W(c->embed), H, A(b.X));
+    launch_gather_x<T>(L, s, new_tokens, new_features, b.ts, KMAX, A(b.fb), c->level_rows, W(c->embed), H, A(b.X));
     GemmSegs fc; fc.n = 1; fc.w[0] = lw.fc_w; fc.rows[0] = H;
     int pr = prof_begin(POSS_PROF_FC);
     SplitKView v_fc = gemm_view(A(b.X), 2 * H, s.M, fc, 2 * H, b.ptmp, H, POSS_K_GEMM_FC);
@@ -245,9 +252,33 @@ struct Impl {
     prof_end(pr);
     RopeArgs ra;
     ra.inv_freq = b.rope_inv;
-    ra.mode = 0; ra.s = s; ra.base = 0; ra.depth = nullptr; ra.rows = s.M; ra.q_rows = with_q ? s.Mc : 0;
+    ra.mode = 0; ra.s = s; ra.base = 0; ra.depth = nullptr; ra.rows = s.M; ra.q_rows = with_q ? s.B * s.Mc : 0;
     ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.draft_kv_slots; ra.theta = g.rope_theta;
-    launch_rope_append<T>(L, ra, v_qkv, kcache, vcache, A(b.q));
+    launch_rope_append<T>(L, ra, v_qkv, caches, A(b.q));
+  }
+
+  // Rows of a cache fill or of draft step `level` for `batch` sequences (first: the step's specialist has not yet
+  // cached this round's verified pairs and earlier levels).  level < 0: verified pairs only, no current rows.
+  static BatchRows step_rows(int batch, const int* prefix_len, const int* n_new, int K, int level, bool first) {
+    BatchRows s;
+    memset(&s, 0, sizeof(s));
+    s.B = batch; s.K = K; s.cur_level = level < 0 ? 0 : level;
+    s.Mc = level < 0 ? 0 : (level == 0 ? 1 : K);
+    s.n_lvl = first && level >= 1 ? (level - 1) * K : 0;
+    int off = 0, tok = 0;
+    for (int b = 0; b < batch; ++b) {
+      s.prefix_len[b] = prefix_len[b]; s.n_new[b] = n_new[b];
+      // at level 0 the last verified pair is the current row, not a pending one
+      s.n_ver[b] = level < 0 ? n_new[b] : (first ? (level == 0 ? n_new[b] - 1 : n_new[b]) : 0);
+      s.pend_off[b] = off;
+      s.tok_off[b] = tok;
+      off += s.n_ver[b] + s.n_lvl;
+      tok += n_new[b];
+    }
+    for (int b = batch; b <= MAXB; ++b) s.pend_off[b] = off;
+    s.n_pend = off;
+    s.M = off + batch * s.Mc;
+    return s;
   }
 
   // attention output -> O-proj + residual -> MLP + residual; x0 = layer input rows.  The result
@@ -274,30 +305,45 @@ struct Impl {
     else launch_splitk_reduce<T>(L, v_d, rows, H, nullptr, b.h1, H, out, H, out_act);
   }
 
+  CachePtrs caches_of(void* const* kvs, int batch, int spec) const {
+    const poss_config& g = c->cfg;
+    const size_t per_spec = (size_t)2 * g.n_kv_heads * g.draft_kv_slots * g.head_dim;
+    CachePtrs cp;
+    memset(&cp, 0, sizeof(cp));
+    for (int b = 0; b < batch; ++b) {
+      T* kc = A(kvs[b]) + (size_t)spec * per_spec;
+      cp.k[b] = kc;
+      cp.v[b] = kc + per_spec / 2;
+    }
+    return cp;
+  }
+
   int draft_prefill(void* draft_kv, int start, const int32_t* tokens, const void* features, int n) {
     const poss_config& g = c->cfg;
-    size_t per_spec = (size_t)2 * g.n_kv_heads * g.draft_kv_slots * g.head_dim;
-    size_t half = per_spec / 2;
+    void* kvs[1] = {draft_kv};
     for (int s = 0; s < g.n_specialists; ++s) {
-      T* kc = A(draft_kv) + s * per_spec;
+      const CachePtrs cp = caches_of(kvs, 1, s);
       for (int off = 0; off < n; off += R) {
         int m = n - off < R ? n - off : R;
-        StepRows sr; sr.n_ver = m; sr.n_lvl = 0; sr.cur_level = 0; sr.K = 1; sr.n_new = m;
-        sr.prefix_len = start + off; sr.M = m; sr.Mc = 0;
-        project_rows(c->spec[s], sr, tokens + off, W(features) + (size_t)off * g.hidden, kc, kc + half, false);
+        int pl = start + off;
+        BatchRows sr = step_rows(1, &pl, &m, 1, -1, true);
+        project_rows(c->spec[s], sr, tokens + off, W(features) + (size_t)off * g.hidden, cp, false);
       }
     }
     return L.err;
   }
 
-  int draft_round(void* draft_kv, int prefix_len, const int32_t* new_tokens, const void* new_features, int n_new,
-                  int depth, int K, int total, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
-                  int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
+  // One draft phase for `batch` sequences (batch = 1: poss_draft_round).  Every matrix product runs once over the
+  // stacked rows of all sequences; attention runs per sequence on its own cache; the tree state, the expansion and
+  // the rerank are per sequence (one block each).
+  int draft_round(int batch, void* const* kvs, const int* prefix_len, const int32_t* new_tokens,
+                  const void* new_features, const int* n_new, int depth, int K, int total, int32_t* out_tokens,
+                  int32_t* out_parents, float* out_scores, int32_t* out_depth, uint64_t* out_mask,
+                  int32_t* out_n_nodes) {
     const poss_config& g = c->cfg;
     Buffers& b = c->b;
     int H = g.hidden, n = g.positions_per_specialist, Sn = g.n_specialists;
-    size_t per_spec = (size_t)2 * g.n_kv_heads * g.draft_kv_slots * g.head_dim;
-    size_t half = per_spec / 2;
+    const int qd = g.n_q_heads * g.head_dim;
     bool used[64] = {false};
     int cand_base = 0;
     in_draft = true;
@@ -305,45 +351,44 @@ struct Impl {
       int s = i / n < Sn - 1 ? i / n : Sn - 1;          // specialist ceil((i+1)/n), clamped, 0-based
       bool first = !used[s < 64 ? s : 63];
       used[s < 64 ? s : 63] = true;
-      StepRows sr;
-      sr.K = K; sr.n_new = n_new; sr.prefix_len = prefix_len; sr.cur_level = i;
-      sr.n_ver = first ? n_new : 0;
-      sr.n_lvl = first && i >= 1 ? (i - 1) * K : 0;
-      sr.Mc = i == 0 ? 1 : K;
-      sr.M = sr.n_ver + sr.n_lvl + (i == 0 ? 0 : K);
-      if (i == 0 && !first) { sr.n_ver = 1; sr.M = 1; }   // unreachable: step 0 is always a first use
-      T* kc = A(draft_kv) + s * per_spec;
-      T* vc = kc + half;
+      const BatchRows sr = step_rows(batch, prefix_len, n_new, K, i, first);
+      const CachePtrs cp = caches_of(kvs, batch, s);
       const poss_layer_w& lw = c->spec[s];
-      project_rows(lw, sr, new_tokens, W(new_features), kc, vc, true);
-      AttnArgs aa;
-      aa.rows = sr.Mc; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.draft_kv_slots;
-      aa.n_all = prefix_len + n_new; aa.n_tree = i * K;
-      aa.mask = b.ts.node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
-      aa.scale = 1.0f / sqrtf((float)g.head_dim);
+      project_rows(lw, sr, new_tokens, W(new_features), cp, true);
       int pr = prof_begin(POSS_PROF_ATTENTION);
-      attention(aa, A(b.q), kc, vc, A(b.o));
+      for (int bq = 0; bq < batch; ++bq) {
+        AttnArgs aa;
+        aa.rows = sr.Mc; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.draft_kv_slots;
+        aa.n_all = prefix_len[bq] + n_new[bq]; aa.n_tree = i * K;
+        aa.mask = tree_of(b.ts, bq).node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
+        aa.scale = 1.0f / sqrtf((float)g.head_dim);
+        attention(aa, A(b.q) + (size_t)bq * sr.Mc * qd, reinterpret_cast<T*>(cp.k[bq]), reinterpret_cast<T*>(cp.v[bq]),
+                  A(b.o) + (size_t)bq * sr.Mc * qd);
+      }
       prof_end(pr);
-      float* fo = b.fout + (size_t)i * KMAX * H;
-      T* fbi = A(b.fb) + (size_t)i * KMAX * H;
-      layer_tail(lw, b.h0 + (size_t)(sr.M - sr.Mc) * H, sr.Mc, fo, fbi);
+      const int Mc_all = batch * sr.Mc;
+      float* fo = b.fout + (size_t)i * c->level_rows * H;
+      T* fbi = A(b.fb) + (size_t)i * c->level_rows * H;
+      layer_tail(lw, b.h0 + (size_t)sr.n_pend * H, Mc_all, fo, fbi);
       ExpandArgs xa;
       xa.enabled = 1; xa.Kmax = KMAX; xa.step = i; xa.Mc = sr.Mc; xa.K = K; xa.cand_base = cand_base;
-      xa.last = i == depth - 1;
-      lm_head_topk(fbi, sr.Mc, K, b.top_ids, b.top_logp, nullptr, &xa);
+      xa.last = i == depth - 1; xa.batch = batch;
+      lm_head_topk(fbi, Mc_all, K, b.top_ids, b.top_logp, nullptr, &xa);
       cand_base += sr.Mc * K;
     }
     // specialists the round did not reach still cache the verified pairs
     for (int s = 0; s < Sn && s < 64; ++s) {
       if (used[s]) continue;
-      StepRows sr; sr.n_ver = n_new; sr.n_lvl = 0; sr.cur_level = 0; sr.K = K; sr.n_new = n_new;
-      sr.prefix_len = prefix_len; sr.M = n_new; sr.Mc = 0;
-      T* kc = A(draft_kv) + s * per_spec;
-      project_rows(c->spec[s], sr, new_tokens, W(new_features), kc, kc + half, false);
+      const BatchRows sr = step_rows(batch, prefix_len, n_new, K, -1, true);
+      project_rows(c->spec[s], sr, new_tokens, W(new_features), caches_of(kvs, batch, s), false);
     }
-    launch_rerank(L, b.ts, cand_base, K, total, n_new - 1, new_tokens, out_tokens, out_parents, out_scores, out_depth,
+    RerankBatch rb;
+    memset(&rb, 0, sizeof(rb));
+    rb.batch = batch;
+    for (int bq = 0, tok = 0; bq < batch; ++bq) { tok += n_new[bq]; rb.root_index[bq] = tok - 1; }
+    launch_rerank(L, b.ts, cand_base, K, total, rb, new_tokens, out_tokens, out_parents, out_scores, out_depth,
                   out_mask, out_n_nodes);
-    c->last_depth = depth; c->last_topk = K;
+    c->last_depth = depth; c->last_topk = K; c->last_batch = batch;
     c->last_nodes = 1 + (total < cand_base ? total : cand_base);
     return L.err;
   }
@@ -381,7 +426,10 @@ struct Impl {
       ra.mode = 1; ra.base = prefix_len; ra.depth = depth; ra.rows = rows; ra.q_rows = rows;
       ra.Hq = g.n_q_heads; ra.Hkv = g.n_kv_heads; ra.d = g.head_dim; ra.cap = g.target_kv_slots;
       ra.theta = g.rope_theta; memset(&ra.s, 0, sizeof(ra.s));
-      launch_rope_append<T>(L, ra, v_qkv, kc, vc, A(b.q));
+      CachePtrs cp;
+      memset(&cp, 0, sizeof(cp));
+      cp.k[0] = kc; cp.v[0] = vc;
+      launch_rope_append<T>(L, ra, v_qkv, cp, A(b.q));
       AttnArgs aa;
       aa.rows = rows; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.target_kv_slots;
       aa.n_all = prefix_len; aa.n_tree = rows; aa.mask = mask; aa.mask_words = mask_words;
@@ -563,7 +611,9 @@ int poss_init(poss_ctx** out, const poss_config* cfg, const poss_weights* w, voi
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->target_final_norm;
   c->esize = cfg->dtype == POSS_BF16 ? 2 : 4;
   c->prof_mode = 0; c->prof_n = 0; c->prof_ev = nullptr;
-  c->launches = 0; c->last_depth = 0; c->last_topk = 0; c->last_nodes = 0;
+  c->launches = 0; c->last_depth = 0; c->last_topk = 0; c->last_nodes = 0; c->last_batch = 0;
+  c->max_batch = cfg->max_batch > 1 ? cfg->max_batch : 1;
+  c->level_rows = c->max_batch * KMAX;
   Bump bp;
   bp.base = reinterpret_cast<char*>(workspace);
   layout(*cfg, bp, c->b, &c->n_chunks, &c->n_cand_max);
@@ -620,6 +670,36 @@ int poss_draft_prefill(poss_ctx* c, void* draft_kv, int start, const int32_t* to
   return DISPATCH(c, stream, draft_prefill(draft_kv, start, tokens, features, n));
 }
 
+namespace {
+// host-side checks shared by the single and the batched entry; POSS_OK when the round fits
+int check_round(const poss_ctx* c, int batch, const int* prefix_len, const int* n_new, int depth, int topk, int total) {
+  const poss_config& g = c->cfg;
+  if (batch < 1 || depth < 1 || topk < 1 || total < 1) return POSS_E_INVALID;
+  if (batch > c->max_batch || batch > POSS_MAX_BATCH) return POSS_E_CAPACITY;
+  if (depth > g.max_depth || topk > g.max_topk || total > g.max_total) return POSS_E_CAPACITY;
+  int sum_new = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (prefix_len[b] < 0 || n_new[b] < 1) return POSS_E_INVALID;
+    if (prefix_len[b] + n_new[b] + (depth - 1) * topk > g.draft_kv_slots) return POSS_E_CAPACITY;
+    sum_new += n_new[b];
+  }
+  // the stacked rows of every step must fit one matrix product: at a specialist's first step of the round the
+  // verified pairs and all earlier levels ride along as pending rows
+  bool used[64] = {false};
+  const int n = g.positions_per_specialist, Sn = g.n_specialists;
+  for (int i = 0; i < depth; ++i) {
+    const int s = i / n < Sn - 1 ? i / n : Sn - 1;
+    const bool first = !used[s < 64 ? s : 63];
+    used[s < 64 ? s : 63] = true;
+    const int cur = batch * (i == 0 ? 1 : topk);
+    const int pend = first ? (i == 0 ? sum_new - batch : sum_new + batch * (i - 1) * topk) : 0;
+    if (pend + cur > R) return POSS_E_CAPACITY;
+  }
+  if (sum_new > R) return POSS_E_CAPACITY;       // specialists the round does not reach cache the verified pairs
+  return POSS_OK;
+}
+}  // namespace
+
 int poss_draft_round(poss_ctx* c, void* draft_kv, int prefix_len, const int32_t* new_tokens, const void* new_features,
                      int n_new, int depth, int topk, int total, int32_t* out_tokens, int32_t* out_parents,
                      float* out_scores, int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes,
@@ -627,37 +707,60 @@ int poss_draft_round(poss_ctx* c, void* draft_kv, int prefix_len, const int32_t*
   if (!c || !draft_kv || !new_tokens || !new_features || !out_tokens || !out_parents || !out_scores || !out_depth ||
       !out_mask || !out_n_nodes)
     return POSS_E_INVALID;
-  if (prefix_len < 0 || n_new < 1 || depth < 1 || topk < 1 || total < 1) return POSS_E_INVALID;
-  const poss_config& g = c->cfg;
-  if (depth > g.max_depth || topk > g.max_topk || total > g.max_total) return POSS_E_CAPACITY;
-  if (n_new + (depth - 1) * topk > R) return POSS_E_CAPACITY;
-  if (prefix_len + n_new + (depth - 1) * topk > g.draft_kv_slots) return POSS_E_CAPACITY;
-  return DISPATCH(c, stream, draft_round(draft_kv, prefix_len, new_tokens, new_features, n_new, depth, topk, total,
+  int rc = check_round(c, 1, &prefix_len, &n_new, depth, topk, total);
+  if (rc != POSS_OK) return rc;
+  void* kvs[1] = {draft_kv};
+  return DISPATCH(c, stream, draft_round(1, kvs, &prefix_len, new_tokens, new_features, &n_new, depth, topk, total,
                                          out_tokens, out_parents, out_scores, out_depth, out_mask, out_n_nodes));
 }
 
-int poss_draft_trace(poss_ctx* c, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores, int32_t* frontier,
-                     float* step_features, int32_t* selected, poss_stream stream) {
-  if (!c || c->last_depth < 1) return POSS_E_INVALID;
+int poss_draft_round_batched(poss_ctx* c, int batch, void* const* h_draft_kv, const int* h_prefix_len,
+                             const int32_t* new_tokens, const void* new_features, const int* h_n_new, int depth,
+                             int topk, int total, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
+                             int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes, poss_stream stream) {
+  if (!c || !h_draft_kv || !h_prefix_len || !h_n_new || !new_tokens || !new_features || !out_tokens || !out_parents ||
+      !out_scores || !out_depth || !out_mask || !out_n_nodes)
+    return POSS_E_INVALID;
+  if (batch < 1) return POSS_E_INVALID;
+  if (batch > POSS_MAX_BATCH) return POSS_E_CAPACITY;
+  for (int b = 0; b < batch; ++b)
+    if (!h_draft_kv[b]) return POSS_E_INVALID;
+  int rc = check_round(c, batch, h_prefix_len, h_n_new, depth, topk, total);
+  if (rc != POSS_OK) return rc;
+  return DISPATCH(c, stream, draft_round(batch, h_draft_kv, h_prefix_len, new_tokens, new_features, h_n_new, depth, topk,
+                                         total, out_tokens, out_parents, out_scores, out_depth, out_mask, out_n_nodes));
+}
+
+int poss_draft_trace_seq(poss_ctx* c, int seq, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores,
+                         int32_t* frontier, float* step_features, int32_t* selected, poss_stream stream) {
+  if (!c || c->last_depth < 1 || seq < 0 || seq >= c->last_batch) return POSS_E_INVALID;
   cudaStream_t st = S(stream);
   int K = c->last_topk, Ld = c->last_depth, H = c->cfg.hidden;
   size_t nc = n_cand_of(Ld, K);
+  const TreeState ts = tree_of(c->b.ts, seq);
   bool ok = true;
   auto cp = [&](void* dst, const void* src, size_t bytes) {
     if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   };
-  cp(cand_tokens, c->b.ts.cand_tok, nc * 4);
-  cp(cand_parents, c->b.ts.cand_parent, nc * 4);
-  cp(cand_scores, c->b.ts.cand_score, nc * 4);
-  cp(selected, c->b.ts.selected, (size_t)(c->last_nodes - 1) * 4);
+  cp(cand_tokens, ts.cand_tok, nc * 4);
+  cp(cand_parents, ts.cand_parent, nc * 4);
+  cp(cand_scores, ts.cand_score, nc * 4);
+  cp(selected, ts.selected, (size_t)(c->last_nodes - 1) * 4);
   for (int l = 1; l < Ld; ++l) {
-    if (frontier) cp(frontier + (size_t)(l - 1) * K, c->b.ts.node_cand + (size_t)l * KMAX, (size_t)K * 4);
+    if (frontier) cp(frontier + (size_t)(l - 1) * K, ts.node_cand + (size_t)l * KMAX, (size_t)K * 4);
   }
   for (int l = 0; l < Ld; ++l) {
+    // level l holds (l == 0 ? 1 : K) expanded rows per sequence, sequence after sequence
+    const size_t mc = l == 0 ? 1 : K;
     if (step_features)
-      cp(step_features + (size_t)l * K * H, c->b.fout + (size_t)l * KMAX * H, (size_t)(l == 0 ? 1 : K) * H * 4);
+      cp(step_features + (size_t)l * K * H, c->b.fout + ((size_t)l * c->level_rows + (size_t)seq * mc) * H, mc * H * 4);
   }
   return ok ? POSS_OK : POSS_E_CUDA;
+}
+
+int poss_draft_trace(poss_ctx* c, int32_t* cand_tokens, int32_t* cand_parents, float* cand_scores, int32_t* frontier,
+                     float* step_features, int32_t* selected, poss_stream stream) {
+  return poss_draft_trace_seq(c, 0, cand_tokens, cand_parents, cand_scores, frontier, step_features, selected, stream);
 }
 
 int poss_tree_attention(poss_ctx* c, const void* q, const void* kv, int kv_slots, int prefix_len, int rows,

@@ -18,32 +18,60 @@ template <> __device__ __forceinline__ float from_f<float>(float v) { return v; 
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 
 // ------------------------------------------------------------------ row bookkeeping of one draft step
-// Rows of a step's projection batch, in order: n_ver verified pairs, then n_lvl pending rows of the
-// earlier tree levels 1.. (width K each), then the current level's K rows (cur_level >= 1).  At
-// cur_level == 0 the current row is the last verified pair.
-struct StepRows {
-  int n_ver, n_lvl, cur_level, K, n_new, prefix_len, M, Mc;
+// A draft step over B sequences stacks the rows of all of them into one batch for the matrix products:
+//   [ pending rows of sequence 0 | ... | pending rows of sequence B-1 | current rows of sequence 0 | ... ]
+// Pending rows of a sequence (keys/values only): n_ver verified pairs, then n_lvl rows of the earlier tree
+// levels 1.. (width K each).  Current rows (the whole layer): Mc per sequence -- the root pair (the sequence's
+// last verified pair) at level 0, the level's K frontier nodes afterwards.  Mc = 0: a cache fill without
+// current rows.
+constexpr int MAXB = POSS_MAX_BATCH;
+struct BatchRows {
+  int B, K, cur_level, Mc, n_lvl;
+  int n_pend;             // pending rows of all sequences
+  int M;                  // n_pend + B * Mc
+  int prefix_len[MAXB], n_new[MAXB];
+  int n_ver[MAXB];        // verified pairs among the sequence's pending rows
+  int pend_off[MAXB + 1]; // first pending row of each sequence
+  int tok_off[MAXB];      // the sequence's verified pairs start here in new_tokens / new_features
 };
 
-struct RowInfo {
+struct RowRef {
+  int seq;
   int level;  // 0 = verified pair
-  int j;      // index among verified pairs, or node index inside its level
+  int j;      // index among the sequence's verified pairs, or node index inside its level
 };
 
-__host__ __device__ __forceinline__ RowInfo row_info(const StepRows& s, int m) {
-  RowInfo r;
-  if (m < s.n_ver) { r.level = 0; r.j = m; return r; }
-  int mm = m - s.n_ver;
-  if (mm < s.n_lvl) { r.level = 1 + mm / s.K; r.j = mm % s.K; return r; }
-  r.level = s.cur_level; r.j = mm - s.n_lvl; return r;
+__host__ __device__ __forceinline__ RowRef batch_row(const BatchRows& s, int m) {
+  RowRef r;
+  if (m >= s.n_pend) {
+    const int cm = m - s.n_pend;
+    r.seq = cm / s.Mc;
+    r.level = s.cur_level;
+    r.j = s.cur_level == 0 ? s.n_new[r.seq] - 1 : cm - r.seq * s.Mc;
+    return r;
+  }
+  int b = 0;
+  while (b + 1 < s.B && m >= s.pend_off[b + 1]) ++b;
+  int mm = m - s.pend_off[b];
+  r.seq = b;
+  if (mm < s.n_ver[b]) { r.level = 0; r.j = mm; return r; }
+  mm -= s.n_ver[b];
+  r.level = 1 + mm / s.K;
+  r.j = mm % s.K;
+  return r;
 }
-// KV slot / rotary position of a row (verified pair j: prefix_len + j; node (level,j): behind them).
-__host__ __device__ __forceinline__ int row_slot(const StepRows& s, RowInfo r) {
-  return r.level == 0 ? s.prefix_len + r.j : s.prefix_len + s.n_new + (r.level - 1) * s.K + r.j;
+// KV slot / rotary position of a row (verified pair j: prefix_len + j; node (level, j): behind them).
+__host__ __device__ __forceinline__ int row_slot(const BatchRows& s, RowRef r) {
+  return r.level == 0 ? s.prefix_len[r.seq] + r.j : s.prefix_len[r.seq] + s.n_new[r.seq] + (r.level - 1) * s.K + r.j;
 }
-__host__ __device__ __forceinline__ int row_pos(const StepRows& s, RowInfo r) {
-  return r.level == 0 ? s.prefix_len + r.j : s.prefix_len + s.n_new - 1 + r.level;
+__host__ __device__ __forceinline__ int row_pos(const BatchRows& s, RowRef r) {
+  return r.level == 0 ? s.prefix_len[r.seq] + r.j : s.prefix_len[r.seq] + s.n_new[r.seq] - 1 + r.level;
 }
+// per-sequence key / value caches of the specialist (or target layer) a launch writes to
+struct CachePtrs {
+  void* k[MAXB];
+  void* v[MAXB];
+};
 
 // ------------------------------------------------------------------ GEMM segments (one launch, up to 3 weights)
 struct GemmSegs {
@@ -63,7 +91,18 @@ struct TreeState {
   float* node_score;      // [Lmax][Kmax]
   uint64_t* node_mask;    // [Lmax][Kmax][2] bits over tree slots (level-1)*K + j
   int32_t* selected;      // [Tmax]
+  // every array holds one such block per sequence of a batched round, cand_cap / node_cap / 256 elements apart
+  int cand_cap, node_cap;
 };
+// the tree state of sequence b
+__host__ __device__ __forceinline__ TreeState tree_of(const TreeState& t, int b) {
+  TreeState r = t;
+  r.cand_tok += (size_t)b * t.cand_cap; r.cand_parent += (size_t)b * t.cand_cap; r.cand_score += (size_t)b * t.cand_cap;
+  r.node_tok += (size_t)b * t.node_cap; r.node_prow += (size_t)b * t.node_cap; r.node_cand += (size_t)b * t.node_cap;
+  r.node_score += (size_t)b * t.node_cap; r.node_mask += (size_t)b * t.node_cap * 2;
+  r.selected += (size_t)b * 256;
+  return r;
+}
 
 // ------------------------------------------------------------------ kernel launchers (defined in the .cu files)
 struct Launcher {
@@ -294,9 +333,11 @@ template <typename T>
 void launch_gemm_simt(Launcher& L, const T* X, int ldx, int M, const GemmSegs& segs, int K, const T* bias,
                       const float* residual, int ldr, float* out, int ldo);
 
+// fb: the features of the expanded rows, [level][level_rows][H]; the rows of sequence b at level l start at
+// b * (l == 0 ? 1 : K)
 template <typename T>
-void launch_gather_x(Launcher& L, StepRows s, const int32_t* new_tokens, const T* new_features,
-                     const TreeState& ts, int Kmax, const T* fb, const T* embed, int H, T* X);
+void launch_gather_x(Launcher& L, const BatchRows& s, const int32_t* new_tokens, const T* new_features,
+                     const TreeState& ts, int Kmax, const T* fb, int level_rows, const T* embed, int H, T* X);
 template <typename T>
 void launch_embed_rows(Launcher& L, const int32_t* tokens, int rows, const T* embed, int H, float* out);
 template <typename T>
@@ -308,16 +349,17 @@ void launch_silu_mul(Launcher& L, const float* gu, int rows, int F, T* out);
 
 struct RopeArgs {
   const double* inv_freq;  // [d/2] theta^(-2j/d), filled at init
-  int mode;        // 0 = draft step rows (StepRows mapping), 1 = target rows (slot = base + r, pos = base + depth[r])
-  StepRows s;
+  int mode;        // 0 = draft step rows (BatchRows mapping), 1 = target rows (slot = base + r, pos = base + depth[r])
+  BatchRows s;
   int base;
   const int32_t* depth;
   int rows, q_rows;  // q is produced for the last q_rows rows
   int Hq, Hkv, d, cap;
   float theta;
 };
+// caches: per sequence in mode 0, entry 0 in mode 1
 template <typename T>
-void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, T* kcache, T* vcache, T* qout);
+void launch_rope_append(Launcher& L, const RopeArgs& a, const SplitKView& qkv, const CachePtrs& caches, T* qout);
 // h[m][n] (fp32) = product + bias[n] + residual[m][n];  xn[m][n] = T(gain[n] * h / rms(h row))  (gain NULL: xn = T(h))
 template <typename T>
 void launch_reduce_norm(Launcher& L, const SplitKView& prod, int rows, int H, const T* bias, const float* residual,
@@ -365,15 +407,21 @@ int launch_argmax_partial(Launcher& L, const T* logits, int rows, int V, float* 
                           int32_t* pidx);
 void launch_topk_partial(Launcher& L, const float* logits, int rows, int V, int K, float* pmax, float* psum,
                          float* pval, int32_t* pidx, int n_chunks);
-// Tree expansion run by the merge kernel's last block (enabled = 0: merge only)
+// Tree expansion run by the merge kernel (enabled = 0: merge only).  batch sequences of Mc rows each: rows
+// [b * Mc, (b + 1) * Mc) belong to sequence b and expand its tree.
 struct ExpandArgs {
-  int enabled, Kmax, step, Mc, K, cand_base, last;
+  int enabled, Kmax, step, Mc, K, cand_base, last, batch;
 };
 void launch_topk_merge(Launcher& L, int rows, int K, int n_lists, const float* pmax, const float* psum,
                        const float* pval, const int32_t* pidx, int32_t* out_ids, float* out_logp,
                        const TreeState* ts = nullptr, const ExpandArgs* x = nullptr, int* done = nullptr);
 
-void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, int root_tok_index,
+// one block per sequence; root_index[b]: position of sequence b's root token in new_tokens; outputs [batch][total+1]
+struct RerankBatch {
+  int batch;
+  int root_index[MAXB];
+};
+void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int total, const RerankBatch& rb,
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes);
 template <typename T>

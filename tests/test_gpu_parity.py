@@ -389,6 +389,75 @@ def test_draft_round_matches_oracle(name, over, n_new, seed, require_exact):
     assert np.array_equal(trace["step_features"], trace2["step_features"])
 
 
+@pytest.mark.parametrize("name,over,B,seed", [
+    ("t_fp32", {}, 3, 61),                                   # check mode, 3 specialists x 2 positions
+    ("t_bf16", {}, 7, 62),                                   # the row limit: 7 sequences' pending + current rows
+    ("t_bf16", {"S": 1, "n": 6, "norm_in": False}, 16, 63),  # the batch limit, one specialist, no input norm
+    ("m_bf16", {}, 2, 64),                                   # six specialists, width 10: two sequences fit
+    ("m_bf16", {"S": 1, "n": 6}, 12, 65),                    # one specialist, width 10: twelve sequences (120 rows)
+    ("t_bf16", {"head_dim": 128, "n_q_heads": 4, "n_kv_heads": 2, "S": 2, "n": 3}, 5, 66),   # tcgen05 attention
+])
+def test_batched_draft_round_equals_single_rounds_bitwise_and_the_oracle(name, over, B, seed):
+    """poss_draft_round_batched: sequences with different prefix lengths, different numbers of verified pairs, their
+    own caches and inputs.  Every sequence's tree, scores, per-step features and cache entries equal, bit for bit,
+    what poss_draft_round gives for that sequence alone (the products see more rows, and a row's value does not
+    depend on the rows around it), and each sequence matches the oracle's definition -- independent rounds -- under
+    the rules of the single-sequence test."""
+    cfg = ps.CONFIGS[name].replace(n_target_layers=0, **over)
+    w = ps.make_weights(cfg, seed)
+    n_news = [1 + (b % 3) for b in range(B)]
+    prefixes = [cfg.prefix - 5 * b for b in range(B)]
+    cap = cfg.prefix + 3 + cfg.tree_slots
+    from paper_2506_03566_b200 import Poss, make_config
+    P = Poss(make_config(cfg, cap, 0, max_batch=B), w)
+    kvs_np = [ps.make_draft_kv(cfg, seed + 100 * b, cap, prefixes[b]) for b in range(B)]
+    ins = [ps.make_round_inputs(cfg, seed + 100 * b, n_news[b]) for b in range(B)]
+    tok_all = torch.from_numpy(np.concatenate([t for t, _ in ins])).cuda()
+    feat_all = dev(np.concatenate([f for _, f in ins], axis=0))
+    kvs = [dev(k) for k in kvs_np]
+    out = P.poss_draft_round_batched(kvs, prefixes, tok_all, feat_all, n_news, cfg.depth, cfg.topk, cfg.total)
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 0
+    host = {k: pu.np_of(v) for k, v in out.items()}
+    traces = [{k: pu.np_of(v) for k, v in P.poss_draft_trace(cfg.depth, cfg.topk, int(host["n_nodes"][b]), seq=b).items()}
+              for b in range(B)]
+    num = pu.oracle_num(cfg)
+    for b in range(B):
+        g1, tr1, dkv1 = pu.run_gpu_round(P, cfg, kvs_np[b], prefixes[b], ins[b][0], ins[b][1], cfg.depth, cfg.topk, cfg.total)
+        gb = {k: (host[k][b] if k != "n_nodes" else host[k][b:b + 1]) for k in host}
+        gb["anc_mask"] = gb["anc_mask"].view(np.uint64)
+        for k in ("tokens", "parents", "scores", "depth", "anc_mask", "n_nodes"):
+            assert np.array_equal(gb[k], g1[k]), (b, k)
+        for k in tr1:
+            assert np.array_equal(traces[b][k], tr1[k]), (b, k)
+        assert torch.equal(kvs[b], dkv1), f"sequence {b}: cache entries differ from the single round's"
+        if b in (0, B - 1):                                  # the oracle comparison proper, on the batch's two ends
+            rep = pu.compare_round(cfg, w, kvs_np[b], prefixes[b], ins[b][0], ins[b][1], cfg.depth, cfg.topk, cfg.total,
+                                   gb, traces[b], num, cfg.dtype == "fp32")
+            pu.compare_kv(cfg, kvs[b], rep["kv_oracle"], prefixes[b], prefixes[b] + n_news[b],
+                          pu.TOL[cfg.dtype])
+
+
+def test_batched_round_capacity_errors():
+    from paper_2506_03566_b200 import Poss, PossError, make_config
+    cfg = ps.CONFIGS["t_bf16"].replace(n_target_layers=0)
+    cap = cfg.prefix + 3 + cfg.tree_slots
+    P = Poss(make_config(cfg, cap, 0, max_batch=8), ps.make_weights(cfg, 1))
+    kv = [P.new_draft_kv() for _ in range(9)]
+    tok = torch.zeros(9, dtype=torch.int32, device="cuda")
+    feat = torch.zeros((9, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(PossError) as e:                      # more sequences than the context was sized for
+        P.poss_draft_round_batched(kv, [10] * 9, tok, feat, [1] * 9, cfg.depth, cfg.topk, cfg.total)
+    assert e.value.code == 3
+    with pytest.raises(PossError) as e:                      # 8 x (1 + 3 x 4 + 4) + ... rows exceed one product
+        P.poss_draft_round_batched(kv[:8], [10] * 8, tok[:8], feat[:8], [1] * 8, cfg.depth, cfg.topk, cfg.total)
+    assert e.value.code == 3
+    with pytest.raises(PossError) as e:
+        P.poss_draft_round_batched(kv[:2], [10, -1], tok[:2], feat[:2], [1, 1], cfg.depth, cfg.topk, cfg.total)
+    assert e.value.code == 1
+    assert P.poss_last_status() == 0
+
+
 def test_alternative_kernel_paths_give_the_same_round_bitwise():
     """Two kernels exist for two stages and the library picks one per call; the choice must not show in the
     result.  The gate/up product finished by the GEMM's own SwiGLU epilogue (POSS_OPT_SWIGLU_IN_KERNEL) against the
