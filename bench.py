@@ -137,6 +137,80 @@ def chain_spans(records):
     return out
 
 
+def run_batched(args, cfg):
+    """--batch B: the draft round for B independent sequences in one call (poss_draft_round_batched), timed like
+    the single round; one JSON line with the batched round's time and the sequences drafted per second."""
+    import torch
+    import poss_synth as ps
+    from paper_2506_03566_b200 import Poss, make_config, to_device
+    from paper_2506_03566_b200 import build as pbuild
+    pbuild.build()
+    torch.cuda.set_device(0)
+    B = args.batch
+    seed = replica_seed(0)
+    w = ps.make_weights(cfg, seed, alias_specialists=args.alias_specialists)
+    cap = cfg.prefix + 8 + cfg.tree_slots
+    P = Poss(make_config(cfg, cap, 0, max_batch=B), w)
+    del w
+    kvs = [to_device(ps.make_draft_kv(cfg, seed + 100 * b, cap)) for b in range(B)]
+    ins = [ps.make_round_inputs(cfg, seed + 100 * b, 1) for b in range(B)]
+    tok = torch.from_numpy(np.concatenate([t for t, _ in ins])).cuda()
+    feat = to_device(np.concatenate([f for _, f in ins], axis=0))
+    pl, nn = [cfg.prefix] * B, [1] * B
+    out = P.poss_draft_round_batched(kvs, pl, tok, feat, nn, cfg.depth, cfg.topk, cfg.total)
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        P.poss_draft_round_batched(kvs, pl, tok, feat, nn, cfg.depth, cfg.topk, cfg.total, out=out)
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 0
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(0).uuid)
+    except Exception:
+        gpu_id = "0"
+    clocks = ClockSampler(gpu_id)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = P.poss_launch_count()
+    t_a = time.perf_counter()
+    e0.record()
+    for _ in range(args.steps):
+        P.poss_draft_round_batched(kvs, pl, tok, feat, nn, cfg.depth, cfg.topk, cfg.total, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks.window(t_a, time.perf_counter())
+    clocks.close()
+    ms = e0.elapsed_time(e1) / args.steps
+    P.poss_profile(3)
+    for _ in range(min(args.steps, 5)):
+        P.poss_draft_round_batched(kvs, pl, tok, feat, nn, cfg.depth, cfg.topk, cfg.total, out=out)
+    chain = chain_spans(P.poss_timeline_read())["draft"]
+    P.poss_profile(0)
+    try:
+        hbm_peak, which = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]), "measured"
+    except Exception:
+        hbm_peak, which = 6650.0, "fallback"
+    round_bytes, _ = algorithmic_bytes(cfg)
+    # tensor work of the round: 2 x rows x weights per step (rows = B x K current rows; pending rows left out)
+    H, F, V = cfg.hidden, cfg.ffn, cfg.vocab
+    qd, kd = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+    w_elems = 2 * H * H + H * (qd + 2 * kd) + qd * H + 3 * H * F + V * H
+    flops = sum(2.0 * B * (1 if i == 0 else cfg.topk) * w_elems for i in range(cfg.depth))
+    line = {"metric": METRIC, "value": ms * 1e3, "unit": "us", "n_gpus": 1, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "batch": B,
+                       "step": f"one batched draft round: {B} independent sequences drafted in one call",
+                       "l2": "inputs larger than L2 (1.56 GB of weights per specialist step)"},
+            "batch": B, "us_per_sequence": ms * 1e3 / B, "sequences_per_s": B * 1e3 / ms,
+            "weight_stream_gbs": round_bytes / (ms * 1e-3) / 1e9,
+            "weight_stream_frac_of_hbm_peak": round_bytes / (ms * 1e-3) / 1e9 / hbm_peak, "peak_source": which,
+            "tensor_tflops": flops / (ms * 1e-3) / 1e12,
+            "gpu_launches": int((P.poss_launch_count() - launches0) // args.steps),
+            "chain_us_per_launch": {n: round(c[1] / c[0], 2) for n, c in sorted(chain.items())},
+            "clocks": clocks.summary()}
+    print(json.dumps(line))
+
+
 def run_reference(args, cfg):
     """The oracle, as it stands, on the host cores: one full draft round per step."""
     import poss_synth as ps
@@ -181,6 +255,8 @@ def main():
     ap.add_argument("--total", type=int, help="override the workload's kept draft tokens T")
     ap.add_argument("--specialists", type=int, help="override the number of position specialists S")
     ap.add_argument("--positions", type=int, help="override the positions per specialist n (PosS-n)")
+    ap.add_argument("--batch", type=int, default=1,
+                    help="B > 1: time poss_draft_round_batched for B independent sequences (draft round only, 1 GPU)")
     ap.add_argument("--no-target", action="store_true", help="verification side = stand-alone stages, no target layers")
     ap.add_argument("--alias-specialists", action="store_true",
                     help="profiler captures only: all specialists share one weight set, so the process holds "
@@ -200,6 +276,9 @@ def main():
         cfg = cfg.replace(**over)
     if args.impl == "reference":
         run_reference(args, cfg)
+        return
+    if args.batch > 1:
+        run_batched(args, cfg)
         return
 
     import torch
