@@ -7,17 +7,16 @@
 // (KV head, 128 query rows) are dealt round-robin to the CTAs that walk them (unit u goes to walker
 // u mod n_walk); a walker pipelines its groups:
 //   * one thread (warp 16) issues every copy and every product.  TMA brings the query tile once and, per group,
-//     128 keys (one stage: a group's keys are free again as soon as its scores exist) and 128 values (two
-//     stages), 128-byte swizzle, rows past the last key or the last tree row arriving as zeros.  S_g = Q' K_g^T
+//     128 keys and 128 values (two stages each, loaded two to three groups ahead), 128-byte swizzle, rows past the last key or the last tree row arriving as zeros.  S_g = Q' K_g^T
 //     (tcgen05.mma, M = 128 query rows, N = 128 keys, fp32 in TMEM) runs two groups ahead into one of two score
 //     buffers; O_g = P_g V_g (two MMAs per 16 keys: hi and lo; V is the MN-major B operand, read as it sits in
 //     the cache: [key][d]) goes into one of two output accumulators, one per group of the unit;
 //   * sixteen warps do the softmax of one group at a time, one thread per (query row, quarter of the group's
 //     keys): scores out of TMEM once (32 registers), ancestor mask, row maximum (the quarters meet through shared
-//     memory), p = 2^(s - m), row sum; p is written to shared memory as a two-term bf16 split (p = hi + lo), laid
+//     memory), p = 2^(s - m), the quarter's share of the row sum; p is written to shared memory as a two-term bf16 split (p = hi + lo), laid
 //     out as the A operand of the second product;
-//   * when a unit's groups are done the same warps merge the two accumulators and park (m, l) and the 128 x 128
-//     fp32 O of the unit in global memory (short-lived, read back out of L2).
+//   * when a unit's groups are done the same warps merge the two accumulators and park the 128 x 128 fp32 O of the
+//     unit, its maximum and the four quarters' row sums in global memory (short-lived, read back out of L2).
 // The walkers of one (KV head, query tile) form one or more thread-block clusters of up to 8 CTAs.  After a
 // cluster barrier the CTA of cluster rank j merges its share of the query rows over ALL units in key order and
 // writes the bf16 result.  With several clusters, the rank-j CTAs count their arrivals per (KV head, query tile,
@@ -53,31 +52,41 @@ constexpr int UNIT_KEYS = 2 * KG;     // keys per parked partial
 constexpr int N_SOFTMAX = 512;        // sixteen softmax warps: TMEM lane quarter x quarter of the group's keys
 constexpr int N_THREADS = N_SOFTMAX + 32;   // + the warp whose first lane issues copies and products
 constexpr int MAX_CLUSTER = 8;        // portable cluster size
-constexpr int MAX_UNITS = 40;         // 10240 keys
+constexpr int MAX_UNITS = 40;         // 10240 keys (the merge's first pass covers up to 48 units)
 constexpr int MAX_ARRIVAL_SETS = 512; // (KV head, query tile) pairs that can run with several clusters
-constexpr int O_LD = D + 4;           // floats per parked partial: 128 outputs, m, l, padding to 16 bytes
+constexpr int O_LD = D + 8;           // floats per parked partial: 128 outputs, four quarter row sums, m, padding
 constexpr int TILE = 128 * 128;       // bytes of a [128 rows][64 bf16] tile
 constexpr float NEG_BIG = -1.0e30f;
-// shared memory: query tile (two 64-column halves), one key stage, two value stages, P as hi and lo (two 64-key
+// shared memory: query tile (two 64-column halves), two key stages, two value stages, P as hi and lo (two 64-key
 // blocks each)
-constexpr uint32_t Q_OFF = 0, K_OFF = 2 * TILE, V_OFF = 4 * TILE, P_HI = 8 * TILE, P_LO = 10 * TILE;
-constexpr uint32_t SMEM_TILES = 12 * TILE;                // 192 KB
+constexpr uint32_t Q_OFF = 0, K_OFF = 2 * TILE, V_OFF = 6 * TILE, P_HI = 10 * TILE, P_LO = 12 * TILE;
+constexpr uint32_t SMEM_TILES = 14 * TILE;                // 224 KB
+constexpr uint32_t SMEM_LIMIT = 227 * 1024;               // static + dynamic shared memory a CTA may hold
 constexpr uint32_t TMEM_COLS = 512;                       // S0 | S1 | O0 | O1, 128 columns each
 
+// One launch serves `batch` sequences (a batched draft step; 1 otherwise): the same rows per sequence, each
+// sequence with its own cache, key count and masks.  blockIdx.z = sequence * q_tiles + query tile.
 struct AttnTcArgs {
-  int rows, Hq, G, n_q;               // n_q = rows * G query rows per KV head
-  int n_all, n_tree, total;
-  int n_units;                        // 256-key units of the call
-  int n_walk;                         // CTAs that share the units of one (KV head, query tile)
+  int rows, Hq, G, n_q;               // per sequence; n_q = rows * G query rows per KV head
+  int batch, q_tiles;
+  int n_walk;                         // CTAs that share the units of one (sequence, KV head, query tile)
   int cluster, n_clusters;            // n_walk = cluster * n_clusters
-  const uint64_t* mask;
   int mask_words;
   float scale_log2;                   // softmax scale times log2(e)
   int inject_lost_load;               // test hook: the value tiles are never requested
-  float* part;                        // [rows][Hq][n_units][O_LD]: a unit's partial, 128 outputs then (m, l)
-  int* arrivals;                      // [Hkv * query tiles][MAX_CLUSTER], zero between launches
-  bf16* out;
+  int n_all[MAXB], total[MAXB];       // keys every row sees / all keys, per sequence
+  int n_units[MAXB];                  // 256-key units, per sequence
+  const uint64_t* mask[MAXB];
+  unsigned long long part_off[MAXB];  // the sequence's partials start here in `part` (floats)
+  float* part;                        // per sequence [rows][Hq][n_units][O_LD]: 128 outputs, 4 row-sum shares, m
+  uint32_t smem_bytes;                // dynamic shared memory of the launch (the tiles must fit behind the alignment)
+  int* arrivals;                      // [batch * query tiles * Hkv][MAX_CLUSTER], zero between launches
+  bf16* out;                          // [batch * rows][Hq][D]
   int32_t* status;
+};
+struct AttnMaps {
+  CUtensorMap q;                      // the stacked queries of all sequences
+  CUtensorMap k[MAXB], v[MAXB];       // each sequence's keys / values
 };
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
@@ -151,30 +160,34 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
 // 544 threads.  Softmax warp w (0..15) owns TMEM lane quarter q = w & 3 (32 query rows) and quarter cq = w >> 2 of
 // a group's eight 16-key chunks; when a unit is parked the same thread owns output columns [32 cq, 32 cq + 32).
 // Lane 0 of warp 16 issues the copies and both products.
-__global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant__ CUtensorMap map_q,
-                                                          const __grid_constant__ CUtensorMap map_k,
-                                                          const __grid_constant__ CUtensorMap map_v, const AttnTcArgs a) {
+__global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant__ AttnMaps maps, const AttnTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[9];
+  __shared__ __align__(8) uint64_t bars[10];
   __shared__ uint32_t tmem_slot;
   __shared__ int s_abort, s_last;
-  __shared__ float x_max[4][QT], x_sum[4][QT];                 // [key quarter][query row]
+  __shared__ float x_max[4][QT];                               // [key quarter][query row]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int walker = blockIdx.x, kvh = blockIdx.y, qtile = blockIdx.z;
+  const int walker = blockIdx.x, kvh = blockIdx.y;
+  const int seq = blockIdx.z / a.q_tiles, qtile = blockIdx.z - seq * a.q_tiles;
+  const int n_all = a.n_all[seq], total = a.total[seq], n_units = a.n_units[seq];
+  const CUtensorMap* const map_q = &maps.q;
+  const CUtensorMap* const map_k = &maps.k[seq];
+  const CUtensorMap* const map_v = &maps.v[seq];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t bar_q = smem_u32(&bars[0]), bar_k = smem_u32(&bars[1]), bar_p = smem_u32(&bars[6]),
-                 bar_pv = smem_u32(&bars[7]), bar_of = smem_u32(&bars[8]);
-  auto bar_v = [&](int st) { return smem_u32(&bars[2 + st]); };
-  auto bar_s = [&](int b) { return smem_u32(&bars[4 + b]); };
+  const uint32_t bar_q = smem_u32(&bars[0]), bar_p = smem_u32(&bars[7]), bar_pv = smem_u32(&bars[8]),
+                 bar_of = smem_u32(&bars[9]);
+  auto bar_k = [&](int st) { return smem_u32(&bars[1 + st]); };
+  auto bar_v = [&](int st) { return smem_u32(&bars[3 + st]); };
+  auto bar_s = [&](int b) { return smem_u32(&bars[5 + b]); };
 
   // this walker's groups, in the order it meets them: its units walker, walker + n_walk, ...; a unit's second
   // group exists when it holds at least one key
-  const int n_my_units = walker < a.n_units ? (a.n_units - 1 - walker) / a.n_walk + 1 : 0;
+  const int n_my_units = walker < n_units ? (n_units - 1 - walker) / a.n_walk + 1 : 0;
   auto group_of = [&](int gi) { return 2 * (walker + (gi >> 1) * a.n_walk) + (gi & 1); };
   auto keys_of = [&](int grp) {
-    int n = a.total - grp * KG;
+    int n = total - grp * KG;
     return n < 0 ? 0 : (n > KG ? KG : n);
   };
   int n_g = 2 * n_my_units;
@@ -182,10 +195,12 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
 
   if (warp == 0) {
     if (lane == 0) {
-      s_abort = 0;
+      // (the tiles need SMEM_TILES bytes behind the 1024-byte alignment: checked on the host, and here)
+      s_abort = base + SMEM_TILES > smem_u32(smem_raw) + a.smem_bytes ? 1 : 0;
       s_last = 0;
       mbar_init(bar_q, 1);
-      mbar_init(bar_k, 1);
+      mbar_init(bar_k(0), 1);
+      mbar_init(bar_k(1), 1);
       mbar_init(bar_v(0), 1);
       mbar_init(bar_v(1), 1);
       mbar_init(bar_s(0), 1);
@@ -195,9 +210,9 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
       mbar_init(bar_of, N_SOFTMAX);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      prefetch_tensormap(&map_q);
-      prefetch_tensormap(&map_k);
-      prefetch_tensormap(&map_v);
+      prefetch_tensormap(map_q);
+      prefetch_tensormap(map_k);
+      prefetch_tensormap(map_v);
     }
     __syncwarp();
     tmem_alloc(smem_u32(&tmem_slot), TMEM_COLS);
@@ -216,20 +231,20 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   if (warp == 16) {
     if (lane == 0 && n_g > 0) {
       // ---------------- copies and products
-      int k_loads = 0, v_loads0 = 0, v_loads1 = 0;
+      int k_loads0 = 0, k_loads1 = 0, v_loads0 = 0, v_loads1 = 0;
       auto load_k = [&](int gi) {
-        const int key0 = group_of(gi) * KG;
-        mbar_expect_tx(bar_k, 2u * TILE);
-        tma_load_3d(base + K_OFF, &map_k, bar_k, 0, key0, kvh);
-        tma_load_3d(base + K_OFF + TILE, &map_k, bar_k, 64, key0, kvh);
-        ++k_loads;
+        const int key0 = group_of(gi) * KG, st = gi & 1;
+        mbar_expect_tx(bar_k(st), 2u * TILE);
+        tma_load_3d(base + K_OFF + st * 2u * TILE, map_k, bar_k(st), 0, key0, kvh);
+        tma_load_3d(base + K_OFF + st * 2u * TILE + TILE, map_k, bar_k(st), 64, key0, kvh);
+        if (st) ++k_loads1; else ++k_loads0;
       };
       auto load_v = [&](int gi) {
         const int key0 = group_of(gi) * KG, st = gi & 1;
         mbar_expect_tx(bar_v(st), 2u * TILE);
         if (!a.inject_lost_load) {
-          tma_load_3d(base + V_OFF + st * 2u * TILE, &map_v, bar_v(st), 0, key0, kvh);
-          tma_load_3d(base + V_OFF + st * 2u * TILE + TILE, &map_v, bar_v(st), 64, key0, kvh);
+          tma_load_3d(base + V_OFF + st * 2u * TILE, map_v, bar_v(st), 0, key0, kvh);
+          tma_load_3d(base + V_OFF + st * 2u * TILE + TILE, map_v, bar_v(st), 64, key0, kvh);
         }
         if (st) ++v_loads1; else ++v_loads0;
       };
@@ -239,7 +254,8 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         const uint32_t t_s = tmem_base + (uint32_t)((gi & 1) * KG);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const uint64_t ad = smem_desc_sw128(base + Q_OFF + h * TILE), bd = smem_desc_sw128(base + K_OFF + h * TILE);
+          const uint64_t ad = smem_desc_sw128(base + Q_OFF + h * TILE),
+                         bd = smem_desc_sw128(base + K_OFF + (uint32_t)(gi & 1) * 2u * TILE + h * TILE);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)          // 16 bf16 = 32 bytes = 2 descriptor address units
             umma_bf16(t_s, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc_s, (h | kk) ? 1u : 0u);
@@ -262,31 +278,31 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
       };
 
       mbar_expect_tx(bar_q, 2u * TILE);
-      tma_load_4d(base + Q_OFF, &map_q, bar_q, 0, 0, kvh, qtile * (QT / a.G));
-      tma_load_4d(base + Q_OFF + TILE, &map_q, bar_q, 64, 0, kvh, qtile * (QT / a.G));
+      // (query rows past this sequence's last row are the next sequence's or zeros: they are computed and dropped)
+      tma_load_4d(base + Q_OFF, map_q, bar_q, 0, 0, kvh, seq * a.rows + qtile * (QT / a.G));
+      tma_load_4d(base + Q_OFF + TILE, map_q, bar_q, 64, 0, kvh, seq * a.rows + qtile * (QT / a.G));
       load_k(0);
       load_v(0);
-      if (n_g > 1) load_v(1);
-      bool ok = mbar_wait(bar_q, 0, abort_flag) && mbar_wait(bar_k, 0, abort_flag);
+      if (n_g > 1) { load_k(1); load_v(1); }
+      bool ok = *abort_flag == 0 && mbar_wait(bar_q, 0, abort_flag) && mbar_wait(bar_k(0), 0, abort_flag);
       if (ok) {
         tc_fence_after();
         issue_s(0);
       }
       if (ok && n_g > 1) {
-        ok = mbar_wait(bar_s(0), 0, abort_flag);              // the first group's scores exist: its keys may go
-        if (ok) {
-          load_k(1);
-          ok = mbar_wait(bar_k, 1, abort_flag);
-        }
+        ok = mbar_wait(bar_k(1), 0, abort_flag);
         if (ok) {
           tc_fence_after();
           issue_s(1);
-          if (n_g > 2) {
-            ok = mbar_wait(bar_s(1), 0, abort_flag);
-            if (ok) load_k(2);
-          }
+        }
+        if (ok && n_g > 2) {
+          ok = mbar_wait(bar_s(0), 0, abort_flag);            // the first group's scores exist: its keys may go
+          if (ok) load_k(2);
         }
       }
+      // Group gi: its second product as soon as its P is written; then the scores two groups ahead (into the
+      // buffer this group's softmax has just left), the keys three groups ahead (into the stage the scores of
+      // group gi + 1 have long left) and the values two groups ahead (into this group's stage).
       for (int gi = 0; gi < n_g && ok; ++gi) {
         ok = mbar_wait(bar_p, (uint32_t)(gi & 1), abort_flag) &&                      // P of this group is written
              mbar_wait(bar_v(gi & 1), (uint32_t)((gi >> 1) & 1), abort_flag);         // its values have landed
@@ -296,16 +312,17 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         tc_fence_after();
         issue_pv(gi);
         if (gi + 2 < n_g) {
-          // scores two groups ahead, into the buffer this group's softmax has just left
-          ok = mbar_wait(bar_k, (uint32_t)((gi + 2) & 1), abort_flag);
+          ok = mbar_wait(bar_k(gi & 1), (uint32_t)(((gi + 2) >> 1) & 1), abort_flag);
           if (!ok) break;
           tc_fence_after();
           issue_s(gi + 2);
-          if (gi + 3 < n_g) {
-            ok = mbar_wait(bar_s(gi & 1), (uint32_t)(((gi + 2) >> 1) & 1), abort_flag);
-            if (!ok) break;
-            load_k(gi + 3);
-          }
+        }
+        if (gi + 3 < n_g) {
+          ok = mbar_wait(bar_s((gi + 1) & 1), (uint32_t)(((gi + 1) >> 1) & 1), abort_flag);
+          if (!ok) break;
+          load_k(gi + 3);
+        }
+        if (gi + 2 < n_g) {
           ok = mbar_wait(bar_pv, (uint32_t)(gi & 1), abort_flag);                     // this group's values may go
           if (!ok) break;
           load_v(gi + 2);
@@ -320,7 +337,8 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
           while (!mbar_try_wait(bar, par) && global_ns() - t0 < WAIT_LIMIT_NS / 2) __nanosleep(64);
         };
         drain(bar_q, 1);
-        drain(bar_k, k_loads);
+        drain(bar_k(0), k_loads0);
+        drain(bar_k(1), k_loads1);
         drain(bar_v(0), v_loads0);
         drain(bar_v(1), v_loads1);
       }
@@ -334,11 +352,14 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
     const int r = valid ? qi / a.G : 0;
     uint64_t mk0 = 0, mk1 = 0;
     if (valid) {
-      mk0 = a.mask[(size_t)r * a.mask_words];
-      if (a.mask_words > 1) mk1 = a.mask[(size_t)r * a.mask_words + 1];
+      const uint64_t* mask = a.mask[seq];
+      mk0 = mask[(size_t)r * a.mask_words];
+      if (a.mask_words > 1) mk1 = mask[(size_t)r * a.mask_words + 1];
     }
+    float* const part = a.part + a.part_off[seq];
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-    float m_g0 = NEG_BIG, m_g1 = NEG_BIG, l_g0 = 0.f, l_g1 = 0.f;   // scaled maximum / row sum of the unit's two groups
+    float m_g0 = NEG_BIG, m_g1 = NEG_BIG;   // scaled row maximum of the unit's two groups
+    float l_g0 = 0.f, l_g1 = 0.f;           // this thread's share (its quarter of the keys) of their row sums
 
     for (int gi = 0; gi < n_g; ++gi) {
       const int grp = group_of(gi);
@@ -358,15 +379,15 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
           tmem_ld16_async(t_lane + (uint32_t)((gi & 1) * KG + c * 16), sr[j]);
           tmem_wait16(sr[j]);
           const int key0 = key_g + c * 16;
-          if (key0 + 16 > a.n_all) {                           // the chunk reaches the tree slots or the end
+          if (key0 + 16 > n_all) {                             // the chunk reaches the tree slots or the end
             // bit i = key0 + i is visible: 16 bits cut out of (all ones below n_all | the row's ancestor mask)
-            const int t0 = key0 - a.n_all;                     // tree slot of the chunk's first key; > -16
+            const int t0 = key0 - n_all;                       // tree slot of the chunk's first key; > -16
             uint32_t vis;
             if (t0 >= 64) vis = t0 >= 128 ? 0u : (uint32_t)(mk1 >> (t0 - 64));
             else if (t0 > 48) vis = (uint32_t)(mk0 >> t0) | (uint32_t)(mk1 << (64 - t0));
             else if (t0 >= 0) vis = (uint32_t)(mk0 >> t0);
             else vis = ((uint32_t)mk0 << (-t0)) | ((1u << (-t0)) - 1u);
-            const int n_valid = a.total - key0;                // keys of the chunk that exist
+            const int n_valid = total - key0;                  // keys of the chunk that exist
             if (n_valid < 16) vis &= (1u << (n_valid < 0 ? 0 : n_valid)) - 1u;
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -410,16 +431,14 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
           *reinterpret_cast<uint4*>(base_ptr + P_LO + line + (((pc + 1) ^ sw) << 4)) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         }
       }
-      x_sum[cq][row] = ls;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P becomes visible to the tensor core
       tc_fence_before();
       mbar_arrive(bar_p);
-      softmax_sync(2);
+      softmax_sync(2);                                         // every quarter has read this group's maxima
       POSS_TRACE_POINT(2);
       {
         const float mg = mraw == -INFINITY ? NEG_BIG : ms;
-        const float lg = (x_sum[0][row] + x_sum[1][row]) + (x_sum[2][row] + x_sum[3][row]);
-        if (gi & 1) { m_g1 = mg; l_g1 = lg; } else { m_g0 = mg; l_g0 = lg; }
+        if (gi & 1) { m_g1 = mg; l_g1 = ls; } else { m_g0 = mg; l_g0 = ls; }
       }
 
       if ((gi & 1) == 1 || gi == n_g - 1) {
@@ -436,8 +455,11 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         const float c0 = ex2(m0 - mu), c1 = two ? ex2(m1 - mu) : 0.f;
         const int unit = walker + (gi >> 1) * a.n_walk;
         const uint32_t t_o = t_lane + 2u * KG + (uint32_t)(cq * 32);
-        float* dst = a.part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * a.n_units + unit) * O_LD;
-        if (valid && cq == 0) *reinterpret_cast<float2*>(dst + D) = make_float2(mu, l0 * c0 + l1 * c1);
+        float* dst = part + (((size_t)r * a.Hq + kvh * a.G + (qi - r * a.G)) * n_units + unit) * O_LD;
+        if (valid) {
+          dst[D + cq] = l0 * c0 + l1 * c1;                     // this quarter's share of the unit's row sum
+          if (cq == 0) dst[D + 4] = mu;
+        }
 #pragma unroll 1
         for (int cc = 0; cc < 2; ++cc) {
           uint32_t v0[16], v1[16];
@@ -478,7 +500,7 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
   bool do_merge = true;
   if (a.n_clusters > 1) {
     if (threadIdx.x == 0) {
-      int* cnt = a.arrivals + ((size_t)(kvh * gridDim.z + qtile) * MAX_CLUSTER + rank);
+      int* cnt = a.arrivals + ((size_t)(blockIdx.z * gridDim.y + kvh) * MAX_CLUSTER + rank);
       __threadfence();
       const int prev = atomicAdd(cnt, 1);
       const int last = prev == a.n_clusters - 1;
@@ -490,7 +512,9 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
     do_merge = s_last != 0;
   }
   if (do_merge) {
-    const int nu = a.n_units;
+    const int nu = n_units;
+    const float* const part = a.part + a.part_off[seq];
+    bf16* const out = a.out + (size_t)seq * a.rows * a.Hq * D;
     const int row_lo = rank * QT / a.cluster, row_hi = (rank + 1) * QT / a.cluster;
 #pragma unroll 1
     for (int item = threadIdx.x; item < (row_hi - row_lo) * 16; item += N_THREADS) {
@@ -498,38 +522,41 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
       const int qj = qtile * QT + rr;
       if (qj >= a.n_q) continue;
       const int rj = qj / a.G, gj = qj - rj * a.G;
-      const float* src = a.part + (((size_t)rj * a.Hq + kvh * a.G + gj) * nu) * O_LD;
-      // the maximum over all units first (every load in flight before the first use, in batches)
+      const float* src = part + (((size_t)rj * a.Hq + kvh * a.G + gj) * nu) * O_LD;
+      // the maximum over all units first: the row's sixteen threads (half a warp) share the loads
       float mm = NEG_BIG;
-#pragma unroll 1
-      for (int u0 = 0; u0 < nu; u0 += 8) {
-        float mv[8];
+      {
+        const int l16 = item & 15;
+        float mv[3];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          mv[j] = u0 + j < nu ? __ldcg(src + (size_t)(u0 + j) * O_LD + D) : NEG_BIG;
+        for (int j = 0; j < 3; ++j) mv[j] = l16 + 16 * j < nu ? __ldcg(src + (size_t)(l16 + 16 * j) * O_LD + D + 4) : NEG_BIG;
+        mm = fmaxf(fmaxf(mv[0], mv[1]), mv[2]);
+        // (the sixteen threads of a row are one half of a warp and take every branch together)
+        const unsigned half_mask = (threadIdx.x & 16) ? 0xffff0000u : 0x0000ffffu;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) mm = fmaxf(mm, mv[j]);
+        for (int o = 8; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(half_mask, mm, o));
       }
       float ll = 0.f, acc[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 #pragma unroll 1
-      for (int u0 = 0; u0 < nu; u0 += 6) {
-        float2 ml[6];
-        float4 x0[6], x1[6];
+      for (int u0 = 0; u0 < nu; u0 += 5) {
+        float ml[5];
+        float4 lp[5], x0[5], x1[5];
 #pragma unroll
-        for (int j = 0; j < 6; ++j) {
+        for (int j = 0; j < 5; ++j) {
           if (u0 + j < nu) {
-            ml[j] = __ldcg(reinterpret_cast<const float2*>(src + (size_t)(u0 + j) * O_LD + D));
+            ml[j] = __ldcg(src + (size_t)(u0 + j) * O_LD + D + 4);
+            lp[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + D));
             x0[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg));
             x1[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg + 4));
           }
         }
 #pragma unroll
-        for (int j = 0; j < 6; ++j) {
+        for (int j = 0; j < 5; ++j) {
           if (u0 + j < nu) {
-            const float c = ex2(ml[j].x - mm);
-            ll += ml[j].y * c;
+            const float c = ex2(ml[j] - mm);
+            ll += ((lp[j].x + lp[j].y) + (lp[j].z + lp[j].w)) * c;
             acc[0] += x0[j].x * c; acc[1] += x0[j].y * c; acc[2] += x0[j].z * c; acc[3] += x0[j].w * c;
             acc[4] += x1[j].x * c; acc[5] += x1[j].y * c; acc[6] += x1[j].z * c; acc[7] += x1[j].w * c;
           }
@@ -542,7 +569,7 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
         __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * j] * inv, acc[2 * j + 1] * inv);
         w[j] = *reinterpret_cast<uint32_t*>(&b);
       }
-      *reinterpret_cast<uint4*>(a.out + ((size_t)rj * a.Hq + kvh * a.G + gj) * D + cg) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(out + ((size_t)rj * a.Hq + kvh * a.G + gj) * D + cg) = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 
@@ -584,28 +611,41 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
-                              const bf16* vc, float* part, size_t part_floats, int* arrivals, bf16* out,
-                              int32_t* status) {
-  if (!tree_attention_tc_supported(a, q, kc, vc, out) || !status || !part || (reinterpret_cast<uintptr_t>(part) & 15))
-    return false;
+bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const AttnBatch& ab, const bf16* q,
+                              float* part, size_t part_floats, int* arrivals, bf16* out, int32_t* status) {
+  if (ab.batch < 1 || ab.batch > MAXB || !status || !part || (reinterpret_cast<uintptr_t>(part) & 15)) return false;
   EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(tc_encode_fn(cache));
   if (!encode) return false;
-  const int G = a.Hq / a.Hkv, total = a.n_all + a.n_tree;
+  const int G = a.Hkv > 0 ? a.Hq / a.Hkv : 1;
+  AttnMaps maps;                       // the launch's tensor maps (copied into the kernel's parameters)
   AttnTcArgs k;
   memset(&k, 0, sizeof(k));
   k.rows = a.rows; k.Hq = a.Hq; k.G = G; k.n_q = a.rows * G;
-  k.n_all = a.n_all; k.n_tree = a.n_tree; k.total = total;
-  int unit_keys = 0;
-  if (!tree_attention_tc_plan(total, &unit_keys, &k.n_units)) return false;
-  if ((size_t)a.rows * a.Hq * k.n_units * O_LD > part_floats) return false;
-  // Walkers per (KV head, query tile): as many as the units, as long as the whole grid still fits the SMs at one
-  // CTA each; more than eight of them form several clusters.  (Scheduling only: the result does not depend on it.)
-  const int q_tiles = (k.n_q + QT - 1) / QT;
-  const int sets = a.Hkv * q_tiles;
+  k.batch = ab.batch;
+  int max_units = 0;
+  size_t part_need = 0;
+  for (int b = 0; b < ab.batch; ++b) {
+    AttnArgs ai = a;
+    ai.n_all = ab.n_all[b];
+    if (!tree_attention_tc_supported(ai, q, ab.kc[b], ab.vc[b], out) || !ab.mask[b]) return false;
+    k.n_all[b] = ab.n_all[b];
+    k.total[b] = ab.n_all[b] + a.n_tree;
+    int unit_keys = 0;
+    if (!tree_attention_tc_plan(k.total[b], &unit_keys, &k.n_units[b])) return false;
+    if (k.n_units[b] > max_units) max_units = k.n_units[b];
+    k.mask[b] = ab.mask[b];
+    k.part_off[b] = part_need;
+    part_need += (size_t)a.rows * a.Hq * k.n_units[b] * O_LD;
+  }
+  if (part_need > part_floats) return false;
+  // Walkers per (sequence, KV head, query tile): as many as the units, as long as the whole grid still fits the SMs
+  // at one CTA each; more than eight of them form several clusters.  (Scheduling only: the result does not depend
+  // on it.)
+  k.q_tiles = (k.n_q + QT - 1) / QT;
+  const int sets = a.Hkv * k.q_tiles * ab.batch;
   int walk = tc_sm_count(cache) / sets;
   if (walk < 1) walk = 1;
-  if (walk > k.n_units) walk = k.n_units;
+  if (walk > max_units) walk = max_units;
   if (walk > MAX_CLUSTER && (!arrivals || sets > MAX_ARRIVAL_SETS)) walk = MAX_CLUSTER;
   if (walk > MAX_CLUSTER) {
     k.n_clusters = walk / MAX_CLUSTER;
@@ -615,46 +655,57 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
     k.cluster = walk;
   }
   k.n_walk = k.cluster * k.n_clusters;
-  k.mask = a.mask; k.mask_words = a.mask_words;
+  k.mask_words = a.mask_words;
   k.scale_log2 = a.scale * 1.4426950408889634f;
   k.part = part; k.arrivals = arrivals; k.out = out; k.status = status;
   k.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
   // More than half an SM's shared memory, so that two of these CTAs never share an SM: each holds all of the SM's
   // TMEM until its whole cluster has merged.
-  const size_t smem = (size_t)SMEM_TILES + 1024u;
+  // Shared memory: the tiles behind a 1024-byte alignment of the dynamic part, which starts behind the kernel's
+  // static part; together they must fit what a CTA may hold.
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, k_attn_tc) != cudaSuccess) return false;
+  const size_t static_bytes = (fa.sharedSizeBytes + 15) / 16 * 16;
+  const size_t pad = (1024 - static_bytes % 1024) % 1024;
+  if (static_bytes + pad + SMEM_TILES > SMEM_LIMIT) return false;
+  const size_t smem = SMEM_LIMIT - static_bytes;
+  k.smem_bytes = (uint32_t)smem;
 
   // The maps carry the call's extents (rows, key count): rows past them are filled with zeros by the copy.
-  CUtensorMap mq, mk, mv;
   {
-    cuuint64_t gdim[4] = {(cuuint64_t)D, (cuuint64_t)G, (cuuint64_t)a.Hkv, (cuuint64_t)a.rows};
+    cuuint64_t gdim[4] = {(cuuint64_t)D, (cuuint64_t)G, (cuuint64_t)a.Hkv, (cuuint64_t)(a.rows * ab.batch)};
     cuuint64_t gstr[3] = {(cuuint64_t)D * 2, (cuuint64_t)G * D * 2, (cuuint64_t)a.Hq * D * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)G, 1, (cuuint32_t)(QT / G)};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    if (encode(&mq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<bf16*>(q), gdim, gstr, box, estr,
+    if (encode(&maps.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<bf16*>(q), gdim, gstr, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }
-  for (int i = 0; i < 2; ++i) {
-    cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)total, (cuuint64_t)a.Hkv};
-    cuuint64_t gstr[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.cap * D * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)KG, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    if (encode(i ? &mv : &mk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(i ? vc : kc), gdim, gstr, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return false;
+  for (int b = 0; b < ab.batch; ++b) {
+    for (int i = 0; i < 2; ++i) {
+      cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)k.total[b], (cuuint64_t)a.Hkv};
+      cuuint64_t gstr[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.cap * D * 2};
+      cuuint32_t box[3] = {64, (cuuint32_t)KG, 1};
+      cuuint32_t estr[3] = {1, 1, 1};
+      if (encode(i ? &maps.v[b] : &maps.k[b], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                 const_cast<bf16*>(i ? ab.vc[b] : ab.kc[b]), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    }
   }
   // the shared-memory opt-in is a per-device property of the kernel
   static PerDeviceFlags attr_done;
   bool* attr = attr_done.current();
   if (!attr || !*attr) {
-    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT) != cudaSuccess)
+      return false;
     if (attr) *attr = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(k.n_walk, a.Hkv, q_tiles);
+  cfg.gridDim = dim3(k.n_walk, a.Hkv, k.q_tiles * ab.batch);
   cfg.blockDim = dim3(N_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = L.stream;
@@ -672,7 +723,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   static PerDeviceFlags refused[MAX_CLUSTER + 1];
   bool* ref = refused[k.cluster].current();
   if (ref && *ref) return false;
-  if (cudaLaunchKernelEx(&cfg, k_attn_tc, mq, mk, mv, k) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, k_attn_tc, maps, k) != cudaSuccess) {
     cudaGetLastError();
     if (ref) *ref = true;
     return false;

@@ -26,9 +26,17 @@ int tc_sm_count(const TcGemmPlanCache*);
 bool tree_attention_tc_plan(int total_keys, int* keys_per_unit, int* n_units);
 size_t tree_attention_tc_arrival_ints();
 bool tree_attention_tc_supported(const AttnArgs& a, const void* q, const void* kc, const void* vc, const void* out);
-bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const bf16* q, const bf16* kc,
-                              const bf16* vc, float* part, size_t part_floats, int* arrivals, bf16* out,
-                              int32_t* status);
+// One launch for `batch` sequences: q / out hold the sequences' rows one after the other (a.rows each), every
+// sequence has its own cache, key count a.n_tree + n_all[b] and masks; a.n_all and a.mask are not read.
+struct AttnBatch {
+  int batch;
+  const bf16* kc[MAXB];
+  const bf16* vc[MAXB];
+  int n_all[MAXB];
+  const uint64_t* mask[MAXB];
+};
+bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const AttnBatch& ab, const bf16* q,
+                              float* part, size_t part_floats, int* arrivals, bf16* out, int32_t* status);
 
 // true when the tensor-core kernel covers this product (bf16, K and leading dimension multiples of 8, ...)
 bool tc_gemm_supported(const GemmSegs& segs, int K, int ldx, int M);

@@ -211,6 +211,7 @@ struct Impl {
   // tree-masked attention: the tcgen05 kernel where it covers the call (bf16, head dimension 128, at most
   // 2048 keys), else the split-KV kernels with their partial buffer
   void attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc, T* out);
+  void attention_batch(const AttnArgs& aa, const AttnBatch& ab, const T* q, T* out);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
   bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists, bool argmax_only = false);
 
@@ -343,7 +344,6 @@ struct Impl {
     const poss_config& g = c->cfg;
     Buffers& b = c->b;
     int H = g.hidden, n = g.positions_per_specialist, Sn = g.n_specialists;
-    const int qd = g.n_q_heads * g.head_dim;
     bool used[64] = {false};
     int cand_base = 0;
     in_draft = true;
@@ -356,14 +356,23 @@ struct Impl {
       const poss_layer_w& lw = c->spec[s];
       project_rows(lw, sr, new_tokens, W(new_features), cp, true);
       int pr = prof_begin(POSS_PROF_ATTENTION);
-      for (int bq = 0; bq < batch; ++bq) {
+      {
         AttnArgs aa;
+        memset(&aa, 0, sizeof(aa));
         aa.rows = sr.Mc; aa.Hq = g.n_q_heads; aa.Hkv = g.n_kv_heads; aa.d = g.head_dim; aa.cap = g.draft_kv_slots;
-        aa.n_all = prefix_len[bq] + n_new[bq]; aa.n_tree = i * K;
-        aa.mask = tree_of(b.ts, bq).node_mask + (size_t)i * KMAX * 2; aa.mask_words = 2;
+        aa.n_tree = i * K; aa.mask_words = 2;
         aa.scale = 1.0f / sqrtf((float)g.head_dim);
-        attention(aa, A(b.q) + (size_t)bq * sr.Mc * qd, reinterpret_cast<T*>(cp.k[bq]), reinterpret_cast<T*>(cp.v[bq]),
-                  A(b.o) + (size_t)bq * sr.Mc * qd);
+        AttnBatch ab;
+        memset(&ab, 0, sizeof(ab));
+        ab.batch = batch;
+        for (int bq = 0; bq < batch; ++bq) {
+          ab.kc[bq] = reinterpret_cast<const bf16*>(cp.k[bq]);
+          ab.vc[bq] = reinterpret_cast<const bf16*>(cp.v[bq]);
+          ab.n_all[bq] = prefix_len[bq] + n_new[bq];
+          ab.mask[bq] = tree_of(b.ts, bq).node_mask + (size_t)i * KMAX * 2;
+        }
+        aa.n_all = ab.n_all[0]; aa.mask = ab.mask[0];
+        attention_batch(aa, ab, A(b.q), A(b.o));
       }
       prof_end(pr);
       const int Mc_all = batch * sr.Mc;
@@ -526,10 +535,37 @@ void Impl<T>::attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc
 }
 template <>
 void Impl<bf16>::attention(const AttnArgs& aa, const bf16* q, const bf16* kc, const bf16* vc, bf16* out) {
-  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, q, kc, vc, c->b.attn_part, c->b.attn_part_floats,
+  AttnBatch ab;
+  memset(&ab, 0, sizeof(ab));
+  ab.batch = 1; ab.kc[0] = kc; ab.vc[0] = vc; ab.n_all[0] = aa.n_all; ab.mask[0] = aa.mask;
+  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, ab, q, c->b.attn_part, c->b.attn_part_floats,
                                              c->b.attn_arrivals, out, c->b.status))
     return;
   run_tree_attention<bf16>(L, aa, ATTN_MAX_SPLITS, q, kc, vc, c->b.attn_part, out);
+}
+
+// the attention of a batched draft step: one launch where the tcgen05 kernel takes it, else sequence by sequence
+template <typename T>
+void Impl<T>::attention_batch(const AttnArgs& aa, const AttnBatch& ab, const T* q, T* out) {
+  const size_t per_seq = (size_t)aa.rows * aa.Hq * aa.d;
+  for (int b = 0; b < ab.batch; ++b) {
+    AttnArgs ai = aa;
+    ai.n_all = ab.n_all[b]; ai.mask = ab.mask[b];
+    attention(ai, q + b * per_seq, reinterpret_cast<const T*>(ab.kc[b]), reinterpret_cast<const T*>(ab.vc[b]),
+              out + b * per_seq);
+  }
+}
+template <>
+void Impl<bf16>::attention_batch(const AttnArgs& aa, const AttnBatch& ab, const bf16* q, bf16* out) {
+  if (c->attn_tc && launch_tree_attention_tc(L, c->tc, aa, ab, q, c->b.attn_part, c->b.attn_part_floats,
+                                             c->b.attn_arrivals, out, c->b.status))
+    return;
+  const size_t per_seq = (size_t)aa.rows * aa.Hq * aa.d;
+  for (int b = 0; b < ab.batch; ++b) {
+    AttnArgs ai = aa;
+    ai.n_all = ab.n_all[b]; ai.mask = ab.mask[b];
+    run_tree_attention<bf16>(L, ai, ATTN_MAX_SPLITS, q + b * per_seq, ab.kc[b], ab.vc[b], c->b.attn_part, out + b * per_seq);
+  }
 }
 
 template <typename T>
