@@ -699,7 +699,7 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   static PerDeviceFlags attr_done;
   bool* attr = attr_done.current();
   if (!attr || !*attr) {
-    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT) != cudaSuccess)
+    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return false;
     if (attr) *attr = true;
   }

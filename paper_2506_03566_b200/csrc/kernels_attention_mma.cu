@@ -378,6 +378,7 @@ void plan_attention_splits_mma(int rows, int Hq, int Hkv, int total_keys, int ma
   int chunks = (total_keys + CHUNK - 1) / CHUNK;
   int ns = chunks;
   if (ns > max_splits) ns = max_splits;
+  if (ns > 32) ns = 32;                             // the combine kernel keeps one split per lane
   if (ns < 1) ns = 1;
   int cps = (chunks + ns - 1) / ns;
   int kps = cps * CHUNK;

@@ -128,6 +128,33 @@ def test_tensor_core_tree_attention_at_its_block_boundaries(rows, P_len, Hq, Hkv
         pu.check_attention(got, want, "bf16", f"{rows}x{P_len} Hq{Hq} Hkv{Hkv}")
 
 
+@pytest.mark.parametrize("rows,P_len,Hq,Hkv", [(10, 100, 8, 2), (61, 1024, 32, 8), (61, 1988, 8, 2), (10, 8262, 32, 8),
+                                               (10, 2100, 40, 40)])
+def test_the_tcgen05_attention_kernel_is_the_one_that_runs(rows, P_len, Hq, Hkv):
+    """A launch the device refuses is handed to the split-KV kernels without an error; this checks, from the
+    library's own launch records, that the tcgen05 kernel takes the shapes it is there for (one launch, no combine
+    kernel), and that switching it off sends the same call to the mma.sync kernels."""
+    from paper_2506_03566_b200.binding import POSS_OPT_ATTENTION_TCGEN05
+    d = 128
+    cfg = ps.CONFIGS["t_bf16"].replace(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, hidden=Hq * d, vocab=64, ffn=64)
+    P = make_poss(cfg, ps.make_weights(cfg, 1), 64)
+    q, kv = ps.make_attention_case(11, rows, Hq, Hkv, d, P_len, P_len + rows, cfg.dtype)
+    mask = torch.from_numpy(po.pack_mask(po.ancestor_matrix(po.chain_parents(rows))).view(np.int64)).cuda()
+    qd, kvd = dev(q), dev(kv)
+    P.poss_profile(3)
+    a = P.poss_tree_attention(qd, kvd, P_len, mask, 1.0 / math.sqrt(d))
+    names = [n for n, _ in P.poss_timeline_read()]
+    assert names == ["attn_tc"], names
+    P.poss_debug_option(POSS_OPT_ATTENTION_TCGEN05, 0)
+    b = P.poss_tree_attention(qd, kvd, P_len, mask, 1.0 / math.sqrt(d))
+    names = [n for n, _ in P.poss_timeline_read()]
+    assert names[0] == "attn_mma" and "attn_tc" not in names, names
+    P.poss_profile(0)
+    assert P.poss_last_status() == 0
+    # the two kernels group their sums differently: a bf16 unit apart at most
+    assert (a.float() - b.float()).abs().max().item() <= 2e-2
+
+
 def test_tensor_core_tree_attention_on_random_shapes():
     """24 seeded random shapes at head dimension 128 (1..64 rows, prefix 0..1500 and, every fourth trial, up to 9000;
     1..8 KV heads, GQA 1..8, cache capacity with and without slack, random trees and chains) against the oracle."""
