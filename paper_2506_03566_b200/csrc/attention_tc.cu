@@ -156,6 +156,118 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
   lo = __byte_perm(__float_as_uint(xr), __float_as_uint(yr), 0x7632);
 }
 
+// ------------------------------------------------------------------ merge of a row's parked units
+// One group of LANES threads (half a warp or a warp) per query row, 128 / LANES consecutive output columns per
+// thread.  Lane j of the group loads the maxima and row-sum shares of units j, j + LANES, ... (together with the
+// first batch of outputs: one round trip for everything when the units fit one batch); the row maximum is a
+// shuffle reduction, each unit's weight c_u = 2^(m_u - max) reaches the other lanes by shuffle, and row sum and
+// outputs are added in unit order.
+struct MergeJob {
+  int nu, row_lo, row_hi, q0, n_q, G, Hq, head0;
+  const float* part;
+  bf16* out;
+};
+template <int LANES>
+__device__ __forceinline__ void merge_rows(const MergeJob& job) {
+  constexpr int COLS = D / LANES;                  // 8 or 4 output columns per thread
+  constexpr int NV = COLS / 4;                     // 16-byte loads per unit
+  constexpr int BATCH = LANES == 16 ? 6 : 12;      // units in flight per thread
+  constexpr int PER_LANE = LANES == 16 ? 3 : 2;    // units whose (m, l) one lane holds: 48 or 64 >= MAX_UNITS
+  const int lane_g = threadIdx.x & (LANES - 1);
+  const unsigned mask = LANES == 32 ? 0xffffffffu : ((threadIdx.x & 16) ? 0xffff0000u : 0x0000ffffu);
+  const int groups = N_THREADS / LANES;
+  const int nu = job.nu;
+#pragma unroll 1
+  for (int rr = job.row_lo + (int)threadIdx.x / LANES; rr < job.row_hi; rr += groups) {
+    const int qj = job.q0 + rr;
+    if (qj >= job.n_q) break;                      // rows only grow: the group is done
+    const int rj = qj / job.G, gj = qj - rj * job.G;
+    const float* src = job.part + (((size_t)rj * job.Hq + job.head0 + gj) * nu) * O_LD;
+    const int cg = lane_g * COLS;
+    // every load of the first batch before the first use
+    float m_l[PER_LANE], l_l[PER_LANE];
+    float4 lp[PER_LANE];
+#pragma unroll
+    for (int j = 0; j < PER_LANE; ++j) {
+      const int u = lane_g + LANES * j;
+      m_l[j] = u < nu ? __ldcg(src + (size_t)u * O_LD + D + 4) : NEG_BIG;
+      lp[j] = u < nu ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)u * O_LD + D)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 x[BATCH][NV];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      if (j < nu) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) x[j][v] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)j * O_LD + cg + 4 * v));
+      }
+    }
+    float mm = NEG_BIG;
+#pragma unroll
+    for (int j = 0; j < PER_LANE; ++j) {
+      mm = fmaxf(mm, m_l[j]);
+      l_l[j] = (lp[j].x + lp[j].y) + (lp[j].z + lp[j].w);
+    }
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(mask, mm, o));
+    float c_l[PER_LANE];
+#pragma unroll
+    for (int j = 0; j < PER_LANE; ++j) {
+      c_l[j] = ex2(m_l[j] - mm);
+      l_l[j] *= c_l[j];
+    }
+    float ll = 0.f, acc[COLS];
+#pragma unroll
+    for (int j = 0; j < COLS; ++j) acc[j] = 0.f;
+    // unit u's weight and weighted row sum sit in lane u % LANES, slot u / LANES
+    auto unit_c = [&](int u, float& c, float& l) {
+      float cs = c_l[0], ls = l_l[0];
+#pragma unroll
+      for (int j = 1; j < PER_LANE; ++j)
+        if (u >= LANES * j) { cs = c_l[j]; ls = l_l[j]; }
+      c = __shfl_sync(mask, cs, u & (LANES - 1), LANES);
+      l = __shfl_sync(mask, ls, u & (LANES - 1), LANES);
+    };
+#pragma unroll 1
+    for (int u0 = 0; u0 < nu; u0 += BATCH) {
+      if (u0 > 0) {
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+          if (u0 + j < nu) {
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+              x[j][v] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg + 4 * v));
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) {
+        if (u0 + j < nu) {
+          float c, l;
+          unit_c(u0 + j, c, l);
+          ll += l;
+#pragma unroll
+          for (int v = 0; v < NV; ++v) {
+            acc[4 * v + 0] = fmaf(x[j][v].x, c, acc[4 * v + 0]);
+            acc[4 * v + 1] = fmaf(x[j][v].y, c, acc[4 * v + 1]);
+            acc[4 * v + 2] = fmaf(x[j][v].z, c, acc[4 * v + 2]);
+            acc[4 * v + 3] = fmaf(x[j][v].w, c, acc[4 * v + 3]);
+          }
+        }
+      }
+    }
+    const float inv = 1.f / ll;
+    uint32_t w[COLS / 2];
+#pragma unroll
+    for (int j = 0; j < COLS / 2; ++j) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * j] * inv, acc[2 * j + 1] * inv);
+      w[j] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    bf16* dst = job.out + ((size_t)rj * job.Hq + job.head0 + gj) * D + cg;
+    if (COLS == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[COLS / 2 - 2], w[COLS / 2 - 1]);
+    else *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+  }
+}
+
 // ------------------------------------------------------------------ the kernel
 // 544 threads.  Softmax warp w (0..15) owns TMEM lane quarter q = w & 3 (32 query rows) and quarter cq = w >> 2 of
 // a group's eight 16-key chunks; when a unit is parked the same thread owns output columns [32 cq, 32 cq + 32).
@@ -512,65 +624,18 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
     do_merge = s_last != 0;
   }
   if (do_merge) {
-    const int nu = n_units;
-    const float* const part = a.part + a.part_off[seq];
-    bf16* const out = a.out + (size_t)seq * a.rows * a.Hq * D;
-    const int row_lo = rank * QT / a.cluster, row_hi = (rank + 1) * QT / a.cluster;
-#pragma unroll 1
-    for (int item = threadIdx.x; item < (row_hi - row_lo) * 16; item += N_THREADS) {
-      const int rr = row_lo + (item >> 4), cg = (item & 15) * 8;
-      const int qj = qtile * QT + rr;
-      if (qj >= a.n_q) continue;
-      const int rj = qj / a.G, gj = qj - rj * a.G;
-      const float* src = part + (((size_t)rj * a.Hq + kvh * a.G + gj) * nu) * O_LD;
-      // the maximum over all units first: the row's sixteen threads (half a warp) share the loads
-      float mm = NEG_BIG;
-      {
-        const int l16 = item & 15;
-        float mv[3];
-#pragma unroll
-        for (int j = 0; j < 3; ++j) mv[j] = l16 + 16 * j < nu ? __ldcg(src + (size_t)(l16 + 16 * j) * O_LD + D + 4) : NEG_BIG;
-        mm = fmaxf(fmaxf(mv[0], mv[1]), mv[2]);
-        // (the sixteen threads of a row are one half of a warp and take every branch together)
-        const unsigned half_mask = (threadIdx.x & 16) ? 0xffff0000u : 0x0000ffffu;
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(half_mask, mm, o));
-      }
-      float ll = 0.f, acc[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll 1
-      for (int u0 = 0; u0 < nu; u0 += 5) {
-        float ml[5];
-        float4 lp[5], x0[5], x1[5];
-#pragma unroll
-        for (int j = 0; j < 5; ++j) {
-          if (u0 + j < nu) {
-            ml[j] = __ldcg(src + (size_t)(u0 + j) * O_LD + D + 4);
-            lp[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + D));
-            x0[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg));
-            x1[j] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg + 4));
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 5; ++j) {
-          if (u0 + j < nu) {
-            const float c = ex2(ml[j] - mm);
-            ll += ((lp[j].x + lp[j].y) + (lp[j].z + lp[j].w)) * c;
-            acc[0] += x0[j].x * c; acc[1] += x0[j].y * c; acc[2] += x0[j].z * c; acc[3] += x0[j].w * c;
-            acc[4] += x1[j].x * c; acc[5] += x1[j].y * c; acc[6] += x1[j].z * c; acc[7] += x1[j].w * c;
-          }
-        }
-      }
-      const float inv = 1.f / ll;
-      uint32_t w[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * j] * inv, acc[2 * j + 1] * inv);
-        w[j] = *reinterpret_cast<uint32_t*>(&b);
-      }
-      *reinterpret_cast<uint4*>(out + ((size_t)rj * a.Hq + kvh * a.G + gj) * D + cg) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    MergeJob job;
+    job.nu = n_units;
+    job.part = a.part + a.part_off[seq];
+    job.out = a.out + (size_t)seq * a.rows * a.Hq * D;
+    job.row_lo = rank * QT / a.cluster;
+    job.row_hi = (rank + 1) * QT / a.cluster;
+    job.q0 = qtile * QT; job.n_q = a.n_q; job.G = a.G; job.Hq = a.Hq; job.head0 = kvh * a.G;
+    // few units: half a warp per row, eight columns per thread, every load of the row in one round trip;
+    // many units: a warp per row, four columns per thread, twelve units in flight per thread.  Both add a
+    // column's terms in unit order with the same operations, so the result does not depend on the choice.
+    if (job.nu <= 6) merge_rows<16>(job);
+    else merge_rows<32>(job);
   }
 
   POSS_TRACE_POINT(5);
@@ -663,9 +728,13 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   // TMEM until its whole cluster has merged.
   // Shared memory: the tiles behind a 1024-byte alignment of the dynamic part, which starts behind the kernel's
   // static part; together they must fit what a CTA may hold.
-  cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, k_attn_tc) != cudaSuccess) return false;
-  const size_t static_bytes = (fa.sharedSizeBytes + 15) / 16 * 16;
+  static size_t static_smem = 0;       // a property of the compiled kernel: asked for once
+  if (!static_smem) {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, k_attn_tc) != cudaSuccess) return false;
+    static_smem = fa.sharedSizeBytes ? fa.sharedSizeBytes : 1;
+  }
+  const size_t static_bytes = (static_smem + 15) / 16 * 16;
   const size_t pad = (1024 - static_bytes % 1024) % 1024;
   if (static_bytes + pad + SMEM_TILES > SMEM_LIMIT) return false;
   const size_t smem = SMEM_LIMIT - static_bytes;
