@@ -24,7 +24,9 @@
 // 64 gate rows and 64 up rows of the same ffn columns and the epilogue writes bf16(silu(g) * u);
 // (2) LM head: running max / sum-exp / top-k per activation row over the CTA's vocabulary tiles, one
 // partial list per CTA, the logits never reach memory (template variant: argmax only, every lane keeps
-// its rows' best in registers); (3) nothing: every tile segment is parked as an fp32 partial and the
+// its rows' best in registers; with more than 16 activation rows -- batched rounds -- the LM-head product runs
+// un-swapped, activation row = TMEM lane, so that one thread owns one row and keeps its running maximum,
+// sum and top-k list without any warp-wide exchange); (3) nothing: every tile segment is parked as an fp32 partial and the
 // kernel that consumes the product adds a tile's segments in range order while it loads (no counter, no
 // last-arriver tail: that reduction is spread over all of the consumer's blocks).
 //
@@ -67,6 +69,7 @@ struct TcArgs {
   int M, Npad, n_stages, mode;
   int n_segs, seg_tiles[3], seg_rows[3], seg_col[3];
   int n_tiles, kb_total, gran, slots, pair_tiles;
+  int rows_on_lanes;      // LM-head mode with many rows: activation rows are the MMA's M dimension (TMEM lane = row)
   int inject_lost_load;   // test hook: the producer leaves out the activation tile of its first stage
   int trace_tag;          // kernel id for the timeline recording (POSS_K_GEMM_*)
   const bf16* bias;
@@ -94,7 +97,10 @@ struct Segment {
 };
 
 // ------------------------------------------------------------------ the kernel
-template <bool ARGMAX>
+// VARIANT 0: every epilogue but the two below; 1: LM-head argmax only (lane-local state in registers); 2: LM-head
+// lists with the activation rows on the TMEM lanes (more than 16 rows).  Separate instantiations, so that the
+// registers of one epilogue never cost another.
+template <int VARIANT>
 __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
                                                        const __grid_constant__ CUtensorMap map_w0,
                                                        const __grid_constant__ CUtensorMap map_w1,
@@ -109,7 +115,10 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
-  const uint32_t x_tile_bytes = (uint32_t)a.Npad * 128u;
+  constexpr bool ARGMAX = VARIANT == 1;
+  constexpr bool rows_on_lanes = VARIANT == 2;
+  const uint32_t x_tile_bytes = rows_on_lanes ? (uint32_t)W_TILE_BYTES : (uint32_t)a.Npad * 128u;
+  const int acc_cols = rows_on_lanes ? TILE_N : a.Npad;     // TMEM columns of one accumulator
   const uint32_t stage_bytes = W_TILE_BYTES + x_tile_bytes;
   const int S = a.n_stages;
   auto w_tile = [&](int s) { return tiles_base + (uint32_t)s * stage_bytes; };
@@ -126,7 +135,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   const long long u1 = splitk_range_begin(blockIdx.x + 1, groups, G, a.gran);
   const int n_kb = (int)(u1 - u0);
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < 2 * a.Npad) tmem_cols <<= 1;
+  while ((int)tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -223,7 +232,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   } else if (warp == 1) {
     if (lane == 0 && n_kb > 0) {
       // ---------------- MMA issuer
-      const uint32_t idesc = instr_desc_bf16(TILE_N, a.Npad);
+      const uint32_t idesc = rows_on_lanes ? instr_desc_bf16(128, TILE_N) : instr_desc_bf16(TILE_N, a.Npad);
       bool ok = true;
       int it = 0, seg_i = 0, s = 0;
       uint32_t phase = 0;
@@ -234,12 +243,14 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         int buf = seg_i & 1, use = seg_i >> 1;
         if (use > 0) ok = mbar_wait(acc_empty(buf), (uint32_t)((use - 1) & 1), abort_flag);
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * a.Npad);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * acc_cols);
         for (int i = 0; i < len && ok; ++i, ++it) {
           ok = mbar_wait(full_bar(s), phase, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          uint64_t ad = smem_desc_sw128(w_tile(s)), bd = smem_desc_sw128(x_tile(s));
+          // swapped: weights are the M operand; rows on lanes: the (zero-padded, 128-row) activation tile is
+          uint64_t ad = smem_desc_sw128(rows_on_lanes ? x_tile(s) : w_tile(s)),
+                   bd = smem_desc_sw128(rows_on_lanes ? w_tile(s) : x_tile(s));
 #pragma unroll
           for (int kk = 0; kk < TILE_K / 16; ++kk)      // 16 bf16 = 32 bytes = 2 descriptor address units
             umma_bf16(tmem_d, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, (i > 0 || kk > 0) ? 1u : 0u);
@@ -261,10 +272,20 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     float* st_sum = extra + (size_t)(4 + q) * a.M;
     float* lst_val = extra + (size_t)8 * a.M + (size_t)q * a.M * K;
     int* lst_idx = reinterpret_cast<int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K) + (size_t)q * a.M * K;
-    if (!ARGMAX && a.mode == 2) {
+    if (!ARGMAX && a.mode == 2 && !rows_on_lanes) {
       for (int m = lane; m < a.M; m += 32) { st_max[m] = -INFINITY; st_sum[m] = 0.f; }
       for (int i = lane; i < a.M * K; i += 32) { lst_val[i] = -INFINITY; lst_idx[i] = 0x7fffffff; }
       __syncwarp();
+    }
+    // rows on lanes: this thread owns activation row t; running maximum and sum in registers, an unordered list
+    // of the K best (value, id) in shared memory, and in registers the list's worst entry: a candidate enters
+    // only if it beats that one (a later equal value carries a higher id and loses)
+    float* my_val = extra + (size_t)t * K;
+    int* my_idx = reinterpret_cast<int*>(extra + (size_t)TILE_N * K) + (size_t)t * K;
+    float r_max = -INFINITY, r_sum = 0.f, worst_v = -INFINITY;
+    int worst_pos = 0, worst_i = 0x7fffffff;
+    if (rows_on_lanes) {
+      for (int i = 0; i < K; ++i) { my_val[i] = -INFINITY; my_idx[i] = 0x7fffffff; }
     }
     // argmax mode: every lane keeps, in registers, the best (value, id) of its own rows for each of up to
     // 64 activation rows; the lanes are merged once, after the CTA's last tile
@@ -293,7 +314,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
       ok = s_epi_ok != 0;
       if (!ok) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.Npad);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * acc_cols);
 
       // where this thread's row lands
       int lt, seg = 0, col, n_local;
@@ -438,6 +459,52 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
             }
           }
         }
+      } else if (rows_on_lanes) {
+        // (LM-head launches always hand out whole tiles)  Columns = the tile's vocabulary rows.
+        const int n0 = lt * TILE_N;
+        const int n_cols = min(TILE_N, a.seg_rows[0] - n0);
+        for (int c0 = 0; c0 < TILE_N; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + (uint32_t)c0, v);
+          if (c0 + 16 >= TILE_N) {                              // last read of this accumulator: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(buf));
+          }
+          if (t < a.M && c0 < n_cols) {
+            const int nv = min(16, n_cols - c0);
+            float cm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (j >= nv) v[j] = -INFINITY;
+              cm = fmaxf(cm, v[j]);
+            }
+            if (cm > r_max) {                                    // (never -inf here: a real logit is finite)
+              r_sum *= expf(r_max - cm);                         // exp(-inf) = 0 at the first chunk
+              r_max = cm;
+            }
+            float add = 0.f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) add += expf(v[j] - r_max);   // exp(-inf) = 0 for the columns past the end
+            r_sum += add;
+            if (cm > worst_v) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                if (v[j] > worst_v) {                            // (columns past the end are -inf and never enter)
+                  my_val[worst_pos] = v[j];
+                  my_idx[worst_pos] = n0 + c0 + j;
+                  // the list's new worst entry: lowest value, among equals the highest id
+                  worst_v = my_val[0]; worst_i = my_idx[0]; worst_pos = 0;
+                  for (int i = 1; i < K; ++i) {
+                    const float lv = my_val[i];
+                    const int li = my_idx[i];
+                    if (lv < worst_v || (lv == worst_v && li > worst_i)) { worst_v = lv; worst_i = li; worst_pos = i; }
+                  }
+                }
+              }
+            }
+          }
+        }
       } else if (whole && a.mode != 3) {
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
           float v[16];
@@ -545,7 +612,26 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         a.pmax[o] = bv; a.psum[o] = 1.f; a.pval[o] = bv; a.pidx[o] = bi;
       }
     }
-    if (!ARGMAX && a.mode == 2) {
+    if (!ARGMAX && a.mode == 2 && rows_on_lanes) {
+      // ---- this thread's list, best first (value down, id up), is the CTA's list of its row
+      if (t < a.M) {
+        const size_t o = (size_t)t * gridDim.x + blockIdx.x;
+        for (int k = 0; k < K; ++k) {
+          int best = 0;
+          float bv = my_val[0];
+          int bi = my_idx[0];
+          for (int i = 1; i < K; ++i)
+            if (better(my_val[i], my_idx[i], bv, bi)) { bv = my_val[i]; bi = my_idx[i]; best = i; }
+          a.pval[o * K + k] = bv;
+          a.pidx[o * K + k] = bi;
+          my_val[best] = -INFINITY;                              // taken: orders behind every remaining entry
+          my_idx[best] = 0x7fffffff;
+        }
+        a.pmax[o] = r_max;
+        a.psum[o] = r_sum;
+      }
+    }
+    if (!ARGMAX && a.mode == 2 && !rows_on_lanes) {
       // ---- merge the four warps' running states into this CTA's list (columns dealt round-robin)
       epi_sync();
       const float* all_max = extra;
@@ -771,11 +857,15 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
     v->slots = a.slots; v->swiglu = ep.mode == TC_EPI_SWIGLU ? 1 : 0;
     for (int i = 0; i < segs.n; ++i) { v->seg_tiles[i] = a.seg_tiles[i]; v->seg_rows[i] = a.seg_rows[i]; }
   }
-  uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
+  // LM head with lists and more than 16 rows (batched rounds): activation rows on the TMEM lanes, a 128-row
+  // activation tile per stage (rows past M arrive as zeros) and one list per thread
+  a.rows_on_lanes = ep.mode == TC_EPI_TOPK && !argmax && a.Npad > 16 ? 1 : 0;
+  uint32_t stage_bytes = W_TILE_BYTES + (a.rows_on_lanes ? (uint32_t)W_TILE_BYTES : (uint32_t)a.Npad * 128u);
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
-  if (ep.mode == TC_EPI_TOPK && !argmax) extra = ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
+  if (ep.mode == TC_EPI_TOPK && !argmax)
+    extra = a.rows_on_lanes ? (size_t)TILE_N * ep.topk * 8 : ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
   // Ring size (measured on the c2 round): 170 KB = nine 18 KB stages for up to 16 rows (150 KB: +12 us per draft
   // round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass; 176 and 220 KB: +18 us
   // per pass)
@@ -795,15 +885,16 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   a.pmax = ep.pmax; a.psum = ep.psum; a.pval = ep.pval; a.pidx = ep.pidx;
 
   CUtensorMap mx, mw[3];
-  if (!get_map(cache, X, M, K, ldx, a.Npad, false, &mx)) { L.err = POSS_E_CUDA; return; }
+  if (!get_map(cache, X, M, K, ldx, a.rows_on_lanes ? TILE_N : a.Npad, false, &mx)) { L.err = POSS_E_CUDA; return; }
   for (int i = 0; i < 3; ++i) {
     int j = i < segs.n ? i : 0;
     if (!get_map(cache, segs.w[j], segs.rows[j], K, K, tile_rows, true, &mw[i])) { L.err = POSS_E_CUDA; return; }
   }
   size_t smem = (size_t)stages * stage_bytes + extra + 1024;
   if (!cache->attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
@@ -821,8 +912,9 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  cudaError_t le = argmax ? cudaLaunchKernelEx(&cfg, k_gemm_tc<true>, mx, mw[0], mw[1], mw[2], a)
-                          : cudaLaunchKernelEx(&cfg, k_gemm_tc<false>, mx, mw[0], mw[1], mw[2], a);
+  cudaError_t le = argmax ? cudaLaunchKernelEx(&cfg, k_gemm_tc<1>, mx, mw[0], mw[1], mw[2], a)
+                   : a.rows_on_lanes ? cudaLaunchKernelEx(&cfg, k_gemm_tc<2>, mx, mw[0], mw[1], mw[2], a)
+                                     : cudaLaunchKernelEx(&cfg, k_gemm_tc<0>, mx, mw[0], mw[1], mw[2], a);
   if (le != cudaSuccess) L.err = POSS_E_CUDA;
   LAUNCH_CHECK(L);
 }

@@ -226,6 +226,18 @@ def test_lm_head_topk_matches_oracle(name, rows, K):
     # the kernel's own logits decide its own top-k exactly (ties -> lowest id)
     own = po.topk_rows(logits.astype(np.float64), K)
     assert np.array_equal(own, ids)
+    # the production form: lists built in the product's epilogue, the logits never stored (up to 16 rows: vocabulary
+    # rows on the accumulator's lanes and warp-wide lists; more rows: one thread per activation row)
+    ids2, logp2, _ = P.poss_lm_head_topk(dev(f), K)
+    ids2, logp2 = ids2.cpu().numpy(), logp2.cpu().numpy()
+    assert P.poss_last_status() == 0
+    for r in range(rows):
+        if not np.array_equal(ids2[r], want[r]):
+            srt = np.sort(z[r])[::-1]
+            assert po._decision_margin(srt, K) < pu.MARGIN, "fused top-k differs although the margin is large"
+            assert np.all(z[r][ids2[r]] >= srt[K - 1] - pu.MARGIN)
+        assert len(set(ids2[r].tolist())) == K
+        assert np.abs(logp2[r] - lp[r][ids2[r]]).max() <= tol
 
 
 def test_lm_head_topk_exact_ties_go_to_the_lowest_id():
