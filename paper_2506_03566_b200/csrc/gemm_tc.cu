@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
   constexpr bool ARGMAX = VARIANT == 1;
   constexpr bool rows_on_lanes = VARIANT == 2;
-  const uint32_t x_tile_bytes = rows_on_lanes ? (uint32_t)W_TILE_BYTES : (uint32_t)a.Npad * 128u;
+  const uint32_t x_tile_bytes = (uint32_t)a.Npad * 128u;
   const int acc_cols = rows_on_lanes ? TILE_N : a.Npad;     // TMEM columns of one accumulator
   const uint32_t stage_bytes = W_TILE_BYTES + x_tile_bytes;
   const int S = a.n_stages;
@@ -127,7 +127,8 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   auto empty_bar = [&](int s) { return smem_u32(&bars[MAX_STAGES + s]); };
   auto acc_full = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + b]); };
   auto acc_empty = [&](int b) { return smem_u32(&bars[2 * MAX_STAGES + 2 + b]); };
-  float* extra = reinterpret_cast<float*>(tiles_ptr + (size_t)S * stage_bytes);   // mode-specific scratch
+  // mode-specific scratch (behind the ring and, rows on lanes, the 16 KB the last stage's operand read runs into)
+  float* extra = reinterpret_cast<float*>(tiles_ptr + (size_t)S * stage_bytes + (VARIANT == 2 ? W_TILE_BYTES : 0));
 
   const int G = gridDim.x;
   const long long groups = (long long)a.n_tiles * a.kb_total / a.gran;
@@ -248,7 +249,9 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
           ok = mbar_wait(full_bar(s), phase, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          // swapped: weights are the M operand; rows on lanes: the (zero-padded, 128-row) activation tile is
+          // swapped: the weight tile is the M operand.  Rows on lanes: the activation tile is, read as 128 rows:
+          // the rows past its Npad loaded ones are whatever shared memory follows (the next stage, or the slack
+          // behind the ring) and fill accumulator lanes that no thread reads.
           uint64_t ad = smem_desc_sw128(rows_on_lanes ? x_tile(s) : w_tile(s)),
                    bd = smem_desc_sw128(rows_on_lanes ? w_tile(s) : x_tile(s));
 #pragma unroll
@@ -267,16 +270,6 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int t = q * 32 + lane;                  // row inside the tile
     const int K = a.topk;
-    // LM-head running state of this warp: max, sum-exp and a best-first list per activation row
-    float* st_max = extra + (size_t)q * a.M;
-    float* st_sum = extra + (size_t)(4 + q) * a.M;
-    float* lst_val = extra + (size_t)8 * a.M + (size_t)q * a.M * K;
-    int* lst_idx = reinterpret_cast<int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K) + (size_t)q * a.M * K;
-    if (!ARGMAX && a.mode == 2 && !rows_on_lanes) {
-      for (int m = lane; m < a.M; m += 32) { st_max[m] = -INFINITY; st_sum[m] = 0.f; }
-      for (int i = lane; i < a.M * K; i += 32) { lst_val[i] = -INFINITY; lst_idx[i] = 0x7fffffff; }
-      __syncwarp();
-    }
     // rows on lanes: this thread owns activation row t; running maximum and sum in registers, an unordered list
     // of the K best (value, id) in shared memory, and in registers the list's worst entry: a candidate enters
     // only if it beats that one (a later equal value carries a higher id and loses)
@@ -363,79 +356,6 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
             }
           }
           epi_sync();
-        } else {
-          const int n_glob = n_local;             // vocabulary id of this lane's row
-          for (int j = 0; j < 16; ++j) {
-            int m = c0 + j;
-            if (m >= a.M) break;
-            float val = n_ok ? v[j] : -INFINITY;
-            // running log-sum-exp
-            float tmax = val;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-            float omax = st_max[m];
-            float nmax = fmaxf(omax, tmax);
-            float p = n_ok ? expf(val - nmax) : 0.f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
-            // running top-k: lanes 0..K-1 hold the list, best first
-            float lv = lane < K ? lst_val[m * K + lane] : -INFINITY;
-            int li = lane < K ? lst_idx[m * K + lane] : 0x7fffffff;
-            float thr = __shfl_sync(0xffffffffu, lv, K - 1);
-            unsigned cand = __ballot_sync(0xffffffffu, val > thr);
-            bool changed = false;
-            if (__popc(cand) > 8) {
-              // Many rows of this slice beat the list's last entry (a CTA's first tiles): place them all at
-              // once.  A candidate's final place is its rank inside the slice plus the list entries that stay
-              // ahead of it; a list entry's place is its index plus the candidates that pass it.  The order
-              // (value down, id up) is total, so the places 0..K-1 are each written exactly once.
-              int rank = 0;
-#pragma unroll 8
-              for (int l = 0; l < 32; ++l) {
-                float ov = __shfl_sync(0xffffffffu, val, l);
-                rank += better(ov, n_glob - lane + l, val, n_glob) ? 1 : 0;
-              }
-              const bool mine = val > thr && rank < K;
-              int ahead_me = 0, ahead_list = 0;
-              for (int j = 0; j < K; ++j) {
-                float ljv = __shfl_sync(0xffffffffu, lv, j);
-                int lji = __shfl_sync(0xffffffffu, li, j);
-                if (better(ljv, lji, val, n_glob)) ++ahead_me;
-                unsigned who = __ballot_sync(0xffffffffu, mine && rank == j);
-                if (who) {
-                  int src = __ffs(who) - 1;
-                  float cv = __shfl_sync(0xffffffffu, val, src);
-                  if (better(cv, n_glob - lane + src, lv, li)) ++ahead_list;
-                }
-              }
-              __syncwarp();
-              if (lane < K && lane + ahead_list < K) { lst_val[m * K + lane + ahead_list] = lv; lst_idx[m * K + lane + ahead_list] = li; }
-              if (mine && rank + ahead_me < K) { lst_val[m * K + rank + ahead_me] = val; lst_idx[m * K + rank + ahead_me] = n_glob; }
-              cand = 0;
-            }
-            while (cand) {
-              int src = __ffs(cand) - 1;
-              cand &= cand - 1;
-              float x = __shfl_sync(0xffffffffu, val, src);
-              int xi = n_glob - lane + src;
-              if (!(x > thr)) continue;
-              unsigned ahead = __ballot_sync(0xffffffffu, lane < K && better(lv, li, x, xi));
-              int pos = __popc(ahead);
-              float pv = __shfl_up_sync(0xffffffffu, lv, 1);
-              int pi = __shfl_up_sync(0xffffffffu, li, 1);
-              if (lane == pos) { lv = x; li = xi; }
-              else if (lane > pos) { lv = pv; li = pi; }
-              thr = __shfl_sync(0xffffffffu, lv, K - 1);
-              changed = true;
-            }
-            __syncwarp();
-            if (lane == 0 && tmax > -INFINITY) {
-              st_sum[m] = st_sum[m] * expf(omax - nmax) + p;
-              st_max[m] = nmax;
-            }
-            if (changed && lane < K) { lst_val[m * K + lane] = lv; lst_idx[m * K + lane] = li; }
-            __syncwarp();
-          }
         }
       };
 
@@ -612,7 +532,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         a.pmax[o] = bv; a.psum[o] = 1.f; a.pval[o] = bv; a.pidx[o] = bi;
       }
     }
-    if (!ARGMAX && a.mode == 2 && rows_on_lanes) {
+    if (rows_on_lanes) {
       // ---- this thread's list, best first (value down, id up), is the CTA's list of its row
       if (t < a.M) {
         const size_t o = (size_t)t * gridDim.x + blockIdx.x;
@@ -629,49 +549,6 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         }
         a.pmax[o] = r_max;
         a.psum[o] = r_sum;
-      }
-    }
-    if (!ARGMAX && a.mode == 2 && !rows_on_lanes) {
-      // ---- merge the four warps' running states into this CTA's list (columns dealt round-robin)
-      epi_sync();
-      const float* all_max = extra;
-      const float* all_sum = extra + (size_t)4 * a.M;
-      const float* all_val = extra + (size_t)8 * a.M;
-      const int* all_idx = reinterpret_cast<const int*>(extra + (size_t)8 * a.M + (size_t)4 * a.M * K);
-      for (int m = q; m < a.M; m += 4) {
-        float mx = -INFINITY;
-        for (int w = 0; w < 4; ++w) mx = fmaxf(mx, all_max[w * a.M + m]);
-        float sm = 0.f;
-        for (int w = 0; w < 4; ++w) {
-          float wm = all_max[w * a.M + m];
-          if (wm > -INFINITY) sm += all_sum[w * a.M + m] * expf(wm - mx);
-        }
-        // K rounds: take the best head among the four best-first lists
-        int head = 0;                              // lane w < 4 tracks list w's head
-        size_t o = ((size_t)m * gridDim.x + blockIdx.x);
-        for (int k = 0; k < K; ++k) {
-          float hv = -INFINITY;
-          int hi = 0x7fffffff;
-          if (lane < 4 && head < K) {
-            hv = all_val[((size_t)lane * a.M + m) * K + head];
-            hi = all_idx[((size_t)lane * a.M + m) * K + head];
-          }
-          float bv = hv;
-          int bi = hi, bw = lane;
-#pragma unroll
-          for (int off = 2; off > 0; off >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            int ow = __shfl_xor_sync(0xffffffffu, bw, off);
-            if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bw = ow; }
-          }
-          bv = __shfl_sync(0xffffffffu, bv, 0);
-          bi = __shfl_sync(0xffffffffu, bi, 0);
-          bw = __shfl_sync(0xffffffffu, bw, 0);
-          if (lane == bw && bi != 0x7fffffff) ++head;
-          if (lane == 0) { a.pval[o * K + k] = bv; a.pidx[o * K + k] = bi; }
-        }
-        if (lane == 0) { a.pmax[o] = mx; a.psum[o] = sm; }
       }
     }
   }
@@ -857,20 +734,23 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
     v->slots = a.slots; v->swiglu = ep.mode == TC_EPI_SWIGLU ? 1 : 0;
     for (int i = 0; i < segs.n; ++i) { v->seg_tiles[i] = a.seg_tiles[i]; v->seg_rows[i] = a.seg_rows[i]; }
   }
-  // LM head with lists and more than 16 rows (batched rounds): activation rows on the TMEM lanes, a 128-row
-  // activation tile per stage (rows past M arrive as zeros) and one list per thread
-  a.rows_on_lanes = ep.mode == TC_EPI_TOPK && !argmax && a.Npad > 16 ? 1 : 0;
-  uint32_t stage_bytes = W_TILE_BYTES + (a.rows_on_lanes ? (uint32_t)W_TILE_BYTES : (uint32_t)a.Npad * 128u);
+  // LM head with lists: activation rows on the TMEM lanes and one list per thread, whatever the row count (the
+  // same arithmetic for one sequence and for a batch of them)
+  a.rows_on_lanes = ep.mode == TC_EPI_TOPK && !argmax ? 1 : 0;
+  uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
   if (ep.mode == TC_EPI_TOPK && !argmax)
-    extra = a.rows_on_lanes ? (size_t)TILE_N * ep.topk * 8 : ((size_t)8 * M + (size_t)8 * M * ep.topk) * sizeof(float);
+    extra = (size_t)TILE_N * ep.topk * 8;
+  // rows on lanes: the activation operand is read as 128 rows from a tile that holds Npad of them; the last
+  // stage's read runs up to 16 KB past the ring, into this slack (never written, never used)
+  const size_t slack = a.rows_on_lanes ? (size_t)W_TILE_BYTES : 0;
   // Ring size (measured on the c2 round): 170 KB = nine 18 KB stages for up to 16 rows (150 KB: +12 us per draft
   // round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass; 176 and 220 KB: +18 us
   // per pass)
   const int smem_kb = a.Npad <= 16 ? 170 : 200;
-  int stages = (int)(((size_t)smem_kb * 1024u - extra - 1024u) / stage_bytes);
+  int stages = (int)(((size_t)smem_kb * 1024u - extra - slack - 1024u) / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
@@ -885,12 +765,12 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   a.pmax = ep.pmax; a.psum = ep.psum; a.pval = ep.pval; a.pidx = ep.pidx;
 
   CUtensorMap mx, mw[3];
-  if (!get_map(cache, X, M, K, ldx, a.rows_on_lanes ? TILE_N : a.Npad, false, &mx)) { L.err = POSS_E_CUDA; return; }
+  if (!get_map(cache, X, M, K, ldx, a.Npad, false, &mx)) { L.err = POSS_E_CUDA; return; }
   for (int i = 0; i < 3; ++i) {
     int j = i < segs.n ? i : 0;
     if (!get_map(cache, segs.w[j], segs.rows[j], K, K, tile_rows, true, &mw[i])) { L.err = POSS_E_CUDA; return; }
   }
-  size_t smem = (size_t)stages * stage_bytes + extra + 1024;
+  size_t smem = (size_t)stages * stage_bytes + slack + extra + 1024;
   if (!cache->attr_set) {
     if (cudaFuncSetAttribute(k_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
