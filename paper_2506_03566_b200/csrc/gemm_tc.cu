@@ -97,9 +97,12 @@ struct Segment {
 };
 
 // ------------------------------------------------------------------ the kernel
-// VARIANT 0: every epilogue but the two below; 1: LM-head argmax only (lane-local state in registers); 2: LM-head
-// lists with the activation rows on the TMEM lanes (more than 16 rows).  Separate instantiations, so that the
-// registers of one epilogue never cost another.
+// VARIANT 0: every epilogue but those below; 1: LM-head argmax only (lane-local state in registers); 2: LM-head
+// lists with the activation rows on the TMEM lanes (more than 16 rows); 3: LM-head lists for up to 16 rows, product
+// swapped like everywhere else and the accumulator tile turned through shared memory.  In 2 and 3 one thread owns
+// one activation row and scans its logits in the same order with the same operations, so a row's lists do not
+// depend on how many rows share the launch.  Separate instantiations, so that the registers of one epilogue never
+// cost another.
 template <int VARIANT>
 __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
                                                        const __grid_constant__ CUtensorMap map_w0,
@@ -117,6 +120,8 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
   uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
   constexpr bool ARGMAX = VARIANT == 1;
   constexpr bool rows_on_lanes = VARIANT == 2;
+  constexpr bool row_lists = VARIANT == 2 || VARIANT == 3;       // one thread per activation row keeps its lists
+  constexpr int XT_LD = TILE_N + 4;                              // row length of the turned tile (variant 3)
   const uint32_t x_tile_bytes = (uint32_t)a.Npad * 128u;
   const int acc_cols = rows_on_lanes ? TILE_N : a.Npad;     // TMEM columns of one accumulator
   const uint32_t stage_bytes = W_TILE_BYTES + x_tile_bytes;
@@ -270,16 +275,51 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int t = q * 32 + lane;                  // row inside the tile
     const int K = a.topk;
-    // rows on lanes: this thread owns activation row t; running maximum and sum in registers, an unordered list
+    // LM-head lists: this thread owns activation row t; running maximum and sum in registers, an unordered list
     // of the K best (value, id) in shared memory, and in registers the list's worst entry: a candidate enters
     // only if it beats that one (a later equal value carries a higher id and loses)
-    float* my_val = extra + (size_t)t * K;
-    int* my_idx = reinterpret_cast<int*>(extra + (size_t)TILE_N * K) + (size_t)t * K;
+    float* xt = extra;                                           // variant 3: the turned tile [16][XT_LD]
+    float* lists = extra + (VARIANT == 3 ? 16 * XT_LD : 0);
+    float* my_val = lists + (size_t)t * K;
+    int* my_idx = reinterpret_cast<int*>(lists + (size_t)TILE_N * K) + (size_t)t * K;
     float r_max = -INFINITY, r_sum = 0.f, worst_v = -INFINITY;
     int worst_pos = 0, worst_i = 0x7fffffff;
-    if (rows_on_lanes) {
+    if (row_lists) {
       for (int i = 0; i < K; ++i) { my_val[i] = -INFINITY; my_idx[i] = 0x7fffffff; }
     }
+    // sixteen consecutive logits of this thread's row (the first nv of them exist), vocabulary ids from id0 on
+    auto scan16 = [&](float* v, int nv, int id0) {
+      float cm = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (j >= nv) v[j] = -INFINITY;
+        cm = fmaxf(cm, v[j]);
+      }
+      if (cm > r_max) {                                          // (never -inf here: a real logit is finite)
+        r_sum *= expf(r_max - cm);                               // exp(-inf) = 0 at the first chunk
+        r_max = cm;
+      }
+      float add = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) add += expf(v[j] - r_max);   // exp(-inf) = 0 for the columns past the end
+      r_sum += add;
+      if (cm > worst_v) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          if (v[j] > worst_v) {                                  // (columns past the end are -inf and never enter)
+            my_val[worst_pos] = v[j];
+            my_idx[worst_pos] = id0 + j;
+            // the list's new worst entry: lowest value, among equals the highest id
+            worst_v = my_val[0]; worst_i = my_idx[0]; worst_pos = 0;
+            for (int i = 1; i < K; ++i) {
+              const float lv = my_val[i];
+              const int li = my_idx[i];
+              if (lv < worst_v || (lv == worst_v && li > worst_i)) { worst_v = lv; worst_i = li; worst_pos = i; }
+            }
+          }
+        }
+      }
+    };
     // argmax mode: every lane keeps, in registers, the best (value, id) of its own rows for each of up to
     // 64 activation rows; the lanes are merged once, after the CTA's last tile
     float abv[ARGMAX ? 4 : 1][16];
@@ -391,40 +431,36 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(buf));
           }
-          if (t < a.M && c0 < n_cols) {
-            const int nv = min(16, n_cols - c0);
-            float cm = -INFINITY;
+          if (t < a.M && c0 < n_cols) scan16(v, min(16, n_cols - c0), n0 + c0);
+        }
+      } else if (VARIANT == 3) {
+        // (whole tiles; at most 16 activation rows = one chunk of accumulator columns)  The warps turn the tile
+        // through shared memory -- lane = vocabulary row in, thread = activation row out -- and the row's thread
+        // scans its 128 logits exactly as above.
+        const int n0 = lt * TILE_N;
+        const int n_cols = min(TILE_N, a.seg_rows[0] - n0);
+        {
+          float v[16];
+          tmem_ld16(taddr, v);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty(buf));
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              if (j >= nv) v[j] = -INFINITY;
-              cm = fmaxf(cm, v[j]);
-            }
-            if (cm > r_max) {                                    // (never -inf here: a real logit is finite)
-              r_sum *= expf(r_max - cm);                         // exp(-inf) = 0 at the first chunk
-              r_max = cm;
-            }
-            float add = 0.f;
+          for (int j = 0; j < 16; ++j) xt[j * XT_LD + t] = v[j];
+        }
+        epi_sync();
+        if (t < a.M) {
+          for (int c0 = 0; c0 < n_cols; c0 += 16) {
+            float v[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) add += expf(v[j] - r_max);   // exp(-inf) = 0 for the columns past the end
-            r_sum += add;
-            if (cm > worst_v) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                if (v[j] > worst_v) {                            // (columns past the end are -inf and never enter)
-                  my_val[worst_pos] = v[j];
-                  my_idx[worst_pos] = n0 + c0 + j;
-                  // the list's new worst entry: lowest value, among equals the highest id
-                  worst_v = my_val[0]; worst_i = my_idx[0]; worst_pos = 0;
-                  for (int i = 1; i < K; ++i) {
-                    const float lv = my_val[i];
-                    const int li = my_idx[i];
-                    if (lv < worst_v || (lv == worst_v && li > worst_i)) { worst_v = lv; worst_i = li; worst_pos = i; }
-                  }
-                }
-              }
+            for (int j = 0; j < 16; j += 4) {
+              const float4 x4 = *reinterpret_cast<const float4*>(xt + t * XT_LD + c0 + j);
+              v[j] = x4.x; v[j + 1] = x4.y; v[j + 2] = x4.z; v[j + 3] = x4.w;
             }
+            scan16(v, min(16, n_cols - c0), n0 + c0);
           }
         }
+        epi_sync();                                              // the next tile overwrites the turned tile
       } else if (whole && a.mode != 3) {
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
           float v[16];
@@ -532,7 +568,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         a.pmax[o] = bv; a.psum[o] = 1.f; a.pval[o] = bv; a.pidx[o] = bi;
       }
     }
-    if (rows_on_lanes) {
+    if (row_lists) {
       // ---- this thread's list, best first (value down, id up), is the CTA's list of its row
       if (t < a.M) {
         const size_t o = (size_t)t * gridDim.x + blockIdx.x;
@@ -734,15 +770,17 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
     v->slots = a.slots; v->swiglu = ep.mode == TC_EPI_SWIGLU ? 1 : 0;
     for (int i = 0; i < segs.n; ++i) { v->seg_tiles[i] = a.seg_tiles[i]; v->seg_rows[i] = a.seg_rows[i]; }
   }
-  // LM head with lists: activation rows on the TMEM lanes and one list per thread, whatever the row count (the
-  // same arithmetic for one sequence and for a batch of them)
-  a.rows_on_lanes = ep.mode == TC_EPI_TOPK && !argmax ? 1 : 0;
+  // LM head with lists: one thread per activation row.  More than 16 rows: the rows sit on the TMEM lanes; up to
+  // 16: the product stays swapped (an eighth of the tensor work) and the tile is turned through shared memory.
+  // Both scan a row's logits in the same order with the same operations.
+  const bool lists = ep.mode == TC_EPI_TOPK && !argmax;
+  a.rows_on_lanes = lists && a.Npad > 16 ? 1 : 0;
   uint32_t stage_bytes = W_TILE_BYTES + (uint32_t)a.Npad * 128u;
   size_t extra = 0;
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
   if (ep.mode == TC_EPI_TOPK && !argmax)
-    extra = (size_t)TILE_N * ep.topk * 8;
+    extra = (size_t)TILE_N * ep.topk * 8 + (a.rows_on_lanes ? 0 : (size_t)16 * (TILE_N + 4) * sizeof(float));
   // rows on lanes: the activation operand is read as 128 rows from a tile that holds Npad of them; the last
   // stage's read runs up to 16 KB past the ring, into this slack (never written, never used)
   const size_t slack = a.rows_on_lanes ? (size_t)W_TILE_BYTES : 0;
@@ -750,7 +788,10 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   // round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass; 176 and 220 KB: +18 us
   // per pass)
   const int smem_kb = a.Npad <= 16 ? 170 : 200;
-  int stages = (int)(((size_t)smem_kb * 1024u - extra - slack - 1024u) / stage_bytes);
+  // (the slack and the per-thread lists of the LM-head epilogue come on top: the ring keeps its stages)
+  const size_t on_top = lists ? slack + extra : 0;
+  int stages = (int)(((size_t)smem_kb * 1024u + on_top - extra - slack - 1024u) / stage_bytes);
+  while (stages > 2 && (size_t)stages * stage_bytes + slack + extra + 1024 > 225u * 1024u) --stages;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) stages = 2;
   a.n_stages = stages;
@@ -774,7 +815,8 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (!cache->attr_set) {
     if (cudaFuncSetAttribute(k_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
+        cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(k_gemm_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess) {
       L.err = POSS_E_CUDA;
       return;
     }
@@ -794,6 +836,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   cfg.numAttrs = 1;
   cudaError_t le = argmax ? cudaLaunchKernelEx(&cfg, k_gemm_tc<1>, mx, mw[0], mw[1], mw[2], a)
                    : a.rows_on_lanes ? cudaLaunchKernelEx(&cfg, k_gemm_tc<2>, mx, mw[0], mw[1], mw[2], a)
+                   : lists ? cudaLaunchKernelEx(&cfg, k_gemm_tc<3>, mx, mw[0], mw[1], mw[2], a)
                                      : cudaLaunchKernelEx(&cfg, k_gemm_tc<0>, mx, mw[0], mw[1], mw[2], a);
   if (le != cudaSuccess) L.err = POSS_E_CUDA;
   LAUNCH_CHECK(L);
