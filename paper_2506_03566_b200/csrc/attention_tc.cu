@@ -162,6 +162,19 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint3
 // first batch of outputs: one round trip for everything when the units fit one batch); the row maximum is a
 // shuffle reduction, each unit's weight c_u = 2^(m_u - max) reaches the other lanes by shuffle, and row sum and
 // outputs are added in unit order.
+// A load past L1 that stays where it is written: the merge wants every load of a batch in flight before the first
+// use, and a plain load under a condition is free to sink to its use (one L2 round trip per unit instead of one per
+// batch).  The callers clamp the address instead of skipping the load.
+__device__ __forceinline__ float4 ld_cg_f4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float ld_cg_f1(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
 struct MergeJob {
   int nu, row_lo, row_hi, q0, n_q, G, Hq, head0;
   const float* part;
@@ -190,22 +203,24 @@ __device__ __forceinline__ void merge_rows(const MergeJob& job) {
 #pragma unroll
     for (int j = 0; j < PER_LANE; ++j) {
       const int u = lane_g + LANES * j;
-      m_l[j] = u < nu ? __ldcg(src + (size_t)u * O_LD + D + 4) : NEG_BIG;
-      lp[j] = u < nu ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)u * O_LD + D)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float* pu = src + (size_t)(u < nu ? u : nu - 1) * O_LD + D;
+      m_l[j] = ld_cg_f1(pu + 4);
+      lp[j] = ld_cg_f4(pu);
     }
     float4 x[BATCH][NV];
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
-      if (j < nu) {
+      const float* pj = src + (size_t)(j < nu ? j : nu - 1) * O_LD + cg;
 #pragma unroll
-        for (int v = 0; v < NV; ++v) x[j][v] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)j * O_LD + cg + 4 * v));
-      }
+      for (int v = 0; v < NV; ++v) x[j][v] = ld_cg_f4(pj + 4 * v);
     }
     float mm = NEG_BIG;
 #pragma unroll
     for (int j = 0; j < PER_LANE; ++j) {
+      const bool have = lane_g + LANES * j < nu;
+      if (!have) m_l[j] = NEG_BIG;
       mm = fmaxf(mm, m_l[j]);
-      l_l[j] = (lp[j].x + lp[j].y) + (lp[j].z + lp[j].w);
+      l_l[j] = have ? (lp[j].x + lp[j].y) + (lp[j].z + lp[j].w) : 0.f;
     }
 #pragma unroll
     for (int o = LANES / 2; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(mask, mm, o));
@@ -232,11 +247,9 @@ __device__ __forceinline__ void merge_rows(const MergeJob& job) {
       if (u0 > 0) {
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
-          if (u0 + j < nu) {
+          const float* pj = src + (size_t)(u0 + j < nu ? u0 + j : nu - 1) * O_LD + cg;
 #pragma unroll
-            for (int v = 0; v < NV; ++v)
-              x[j][v] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(u0 + j) * O_LD + cg + 4 * v));
-          }
+          for (int v = 0; v < NV; ++v) x[j][v] = ld_cg_f4(pj + 4 * v);
         }
       }
 #pragma unroll
@@ -628,8 +641,10 @@ __global__ void __launch_bounds__(N_THREADS, 1) k_attn_tc(const __grid_constant_
     job.nu = n_units;
     job.part = a.part + a.part_off[seq];
     job.out = a.out + (size_t)seq * a.rows * a.Hq * D;
-    job.row_lo = rank * QT / a.cluster;
-    job.row_hi = (rank + 1) * QT / a.cluster;
+    // the tile's rows that exist, in equal shares
+    const int n_here = a.n_q - qtile * QT < QT ? a.n_q - qtile * QT : QT;
+    job.row_lo = rank * n_here / a.cluster;
+    job.row_hi = (rank + 1) * n_here / a.cluster;
     job.q0 = qtile * QT; job.n_q = a.n_q; job.G = a.G; job.Hq = a.Hq; job.head0 = kvh * a.G;
     // few units: half a warp per row, eight columns per thread, every load of the row in one round trip;
     // many units: a warp per row, four columns per thread, twelve units in flight per thread.  Both add a
@@ -676,6 +691,37 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// How many clusters of `size` CTAs of the kernel the current device holds at once (0: cannot be had).  Asked once
+// per device and size.
+static int resident_clusters(int size, size_t smem) {
+  constexpr int MAX_DEVICES = 64;
+  static int known[MAX_DEVICES][MAX_CLUSTER + 1];              // 0 = not asked yet, -1 = the query failed
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 0;
+  int& slot = known[dev][size];
+  if (slot == 0) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(size, 1, 1);
+    cfg.blockDim = dim3(N_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = size;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, k_attn_tc, &cfg) != cudaSuccess || n < 1) {
+      cudaGetLastError();
+      n = -1;
+    }
+    slot = n;
+  }
+  return slot > 0 ? slot : 0;
+}
+
 bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArgs& a, const AttnBatch& ab, const bf16* q,
                               float* part, size_t part_floats, int* arrivals, bf16* out, int32_t* status) {
   if (ab.batch < 1 || ab.batch > MAXB || !status || !part || (reinterpret_cast<uintptr_t>(part) & 15)) return false;
@@ -703,31 +749,9 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
     part_need += (size_t)a.rows * a.Hq * k.n_units[b] * O_LD;
   }
   if (part_need > part_floats) return false;
-  // Walkers per (sequence, KV head, query tile): as many as the units, as long as the whole grid still fits the SMs
-  // at one CTA each; more than eight of them form several clusters.  (Scheduling only: the result does not depend
-  // on it.)
-  k.q_tiles = (k.n_q + QT - 1) / QT;
-  const int sets = a.Hkv * k.q_tiles * ab.batch;
-  int walk = tc_sm_count(cache) / sets;
-  if (walk < 1) walk = 1;
-  if (walk > max_units) walk = max_units;
-  if (walk > MAX_CLUSTER && (!arrivals || sets > MAX_ARRIVAL_SETS)) walk = MAX_CLUSTER;
-  if (walk > MAX_CLUSTER) {
-    k.n_clusters = walk / MAX_CLUSTER;
-    k.cluster = MAX_CLUSTER;
-  } else {
-    k.n_clusters = 1;
-    k.cluster = walk;
-  }
-  k.n_walk = k.cluster * k.n_clusters;
-  k.mask_words = a.mask_words;
-  k.scale_log2 = a.scale * 1.4426950408889634f;
-  k.part = part; k.arrivals = arrivals; k.out = out; k.status = status;
-  k.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
-  // More than half an SM's shared memory, so that two of these CTAs never share an SM: each holds all of the SM's
-  // TMEM until its whole cluster has merged.
   // Shared memory: the tiles behind a 1024-byte alignment of the dynamic part, which starts behind the kernel's
-  // static part; together they must fit what a CTA may hold.
+  // static part; together they must fit what a CTA may hold.  (More than half an SM's shared memory, so that two of
+  // these CTAs never share an SM: each holds all of the SM's TMEM until its whole cluster has merged.)
   static size_t static_smem = 0;       // a property of the compiled kernel: asked for once
   if (!static_smem) {
     cudaFuncAttributes fa;
@@ -739,7 +763,54 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
   if (static_bytes + pad + SMEM_TILES > SMEM_LIMIT) return false;
   const size_t smem = SMEM_LIMIT - static_bytes;
   k.smem_bytes = (uint32_t)smem;
-
+  // the shared-memory opt-in is a per-device property of the kernel
+  static PerDeviceFlags attr_done;
+  bool* attr = attr_done.current();
+  if (!attr || !*attr) {
+    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return false;
+    if (attr) *attr = true;
+  }
+  // Walkers per (sequence, KV head, query tile), as c clusters of s CTAs: the shape with the lowest estimated time.
+  // A cluster needs its s SMs inside one GPC, so fewer large clusters are resident at once than the SM count
+  // suggests (15 of eight on a 148-SM device), and a shape that needs a second wave takes twice as long; the merge
+  // is done by the s CTAs of the cluster that arrives last, so small clusters leave it to few SMs.  Estimates in
+  // tenths of a microsecond, from device timestamps: 6.2 us per unit walked, 4 us to start a wave, 1 us + 0.9 us
+  // per batch of units for every pass of the merge over a CTA's rows, its reads at 100 GB/s per SM.
+  // (Scheduling only: the result does not depend on it.)
+  k.q_tiles = (k.n_q + QT - 1) / QT;
+  const int sets = a.Hkv * k.q_tiles * ab.batch;
+  const bool several = arrivals && sets <= MAX_ARRIVAL_SETS;
+  const int tile_rows = k.n_q < QT ? k.n_q : QT;
+  long best_cost = -1;
+  k.cluster = 1;
+  k.n_clusters = 1;
+  for (int s = MAX_CLUSTER; s >= 1; --s) {
+    if (s > max_units) continue;
+    const int fit = resident_clusters(s, smem);
+    if (fit < 1) continue;
+    int c = fit / sets;
+    if (c < 1) c = 1;
+    if (c > max_units / s) c = max_units / s;
+    if (c > 1 && !several) c = 1;
+    const long waves = (sets * c + fit - 1) / fit;
+    const long walked = (max_units + s * c - 1) / (s * c);
+    const long rows_rank = (tile_rows + s - 1) / s;
+    const long passes = (rows_rank + (max_units <= 6 ? 33 : 16)) / (max_units <= 6 ? 34 : 17);
+    const long batches = max_units <= 6 ? 1 : (max_units + 11) / 12;
+    const long cost = waves * (40 + 62 * walked) + passes * (10 + 9 * batches) +
+                      rows_rank * max_units * (O_LD * 4) / 10000 + (c > 1 ? 10 : 0);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      k.cluster = s;
+      k.n_clusters = c;
+    }
+  }
+  k.n_walk = k.cluster * k.n_clusters;
+  k.mask_words = a.mask_words;
+  k.scale_log2 = a.scale * 1.4426950408889634f;
+  k.part = part; k.arrivals = arrivals; k.out = out; k.status = status;
+  k.inject_lost_load = tc_take_injection(cache) ? 1 : 0;
   // The maps carry the call's extents (rows, key count): rows past them are filled with zeros by the copy.
   {
     cuuint64_t gdim[4] = {(cuuint64_t)D, (cuuint64_t)G, (cuuint64_t)a.Hkv, (cuuint64_t)(a.rows * ab.batch)};
@@ -763,14 +834,6 @@ bool launch_tree_attention_tc(Launcher& L, TcGemmPlanCache* cache, const AttnArg
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
     }
-  }
-  // the shared-memory opt-in is a per-device property of the kernel
-  static PerDeviceFlags attr_done;
-  bool* attr = attr_done.current();
-  if (!attr || !*attr) {
-    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return false;
-    if (attr) *attr = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
