@@ -90,6 +90,15 @@ struct TcArgs {
 // barrier among the four epilogue warps only
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// e^x for the running sums of the LM-head lists (x <= 0): one multiply and the hardware's 2^x, whose relative error of
+// about 2^-22 is far below what the log-sum-exp of a vocabulary row needs; the library's expf costs several times the
+// instructions, and the scan of a CTA's last tile is not hidden behind any copy.
+__device__ __forceinline__ float exp_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x * 1.4426950408889634f));
+  return y;
+}
+
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
 struct Segment {
@@ -296,12 +305,12 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         cm = fmaxf(cm, v[j]);
       }
       if (cm > r_max) {                                          // (never -inf here: a real logit is finite)
-        r_sum *= expf(r_max - cm);                               // exp(-inf) = 0 at the first chunk
+        r_sum *= exp_fast(r_max - cm);                               // exp(-inf) = 0 at the first chunk
         r_max = cm;
       }
       float add = 0.f;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) add += expf(v[j] - r_max);   // exp(-inf) = 0 for the columns past the end
+      for (int j = 0; j < 16; ++j) add += exp_fast(v[j] - r_max);   // exp(-inf) = 0 for the columns past the end
       r_sum += add;
       if (cm > worst_v) {
 #pragma unroll
