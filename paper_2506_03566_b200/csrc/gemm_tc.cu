@@ -329,6 +329,123 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         }
       }
     };
+    // Variant 3 has 128 threads for at most 16 rows, and the one-thread scan above is a long chain of dependent
+    // instructions: the first tile of a CTA, whose list is still empty, took it 28 us (device timestamps, ten rows),
+    // later tiles 7 .. 3 us.  Here eight threads share a row: thread (row, s) holds chunk s (16 logits) of the tile
+    // and two entries of the row's list (entry k, best first, sits in thread k & 7, slot k >> 3).  Maximum and sum
+    // stay the one-thread recurrence bit for bit: chunk s needs the maximum after chunks 0..s (a prefix maximum over
+    // the eight threads), its sum of exponentials is then the same expression, and the eight steps of the recurrence
+    // are replayed in order by every thread of the row from the shuffled (maximum, sum) pairs.  The list is kept in
+    // order and takes a tile's entrants one per round (at most K rounds, a fraction of a microsecond each, none for
+    // a tile without entrants).  The K best by (value down, id up) are a set that does not depend on how it is
+    // found, so the lists equal the one-thread scan's.
+    const int row3 = t >> 3, sub3 = t & 7;
+    float ov[2] = {-INFINITY, -INFINITY};
+    int oi[2] = {0x7fffffff, 0x7fffffff};
+    auto scan_tile3 = [&](int n0, int n_cols) {
+      float c_v[16];
+      int c_i[16];
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        const float4 x4 = *reinterpret_cast<const float4*>(xt + row3 * XT_LD + sub3 * 16 + j);
+        c_v[j] = x4.x; c_v[j + 1] = x4.y; c_v[j + 2] = x4.z; c_v[j + 3] = x4.w;
+      }
+      const int nv = n_cols - sub3 * 16, id0 = n0 + sub3 * 16;
+      float cm = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (j >= nv) c_v[j] = -INFINITY;
+        c_i[j] = j < nv ? id0 + j : 0x7fffffff;
+        cm = fmaxf(cm, c_v[j]);
+      }
+      float pm = cm;                                             // the row's maximum after this chunk
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, pm, o, 8);
+        if (sub3 >= o) pm = fmaxf(pm, y);
+      }
+      pm = fmaxf(pm, r_max);
+      float add = 0.f;
+      if (nv > 0) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) add += exp_fast(c_v[j] - pm);
+      }
+#pragma unroll
+      for (int s8 = 0; s8 < 8; ++s8) {
+        const float cs = __shfl_sync(0xffffffffu, cm, s8, 8), as = __shfl_sync(0xffffffffu, add, s8, 8);
+        if (n_cols > 16 * s8) {
+          if (cs > r_max) {
+            r_sum *= exp_fast(r_max - cs);
+            r_max = cs;
+          }
+          r_sum += as;
+        }
+      }
+      // The row's K-th entry so far: a logit enters only if it beats it (an equal one carries a higher id and
+      // loses).  Entrants are taken best first; entrant number r lands at position (old entries better than it) + r,
+      // and a row is done once a position reaches K or nothing is left.  Then every thread rebuilds its two entries:
+      // an entrant that landed there, or the old entry that moved up by the entrants before it.
+      const float kth = __shfl_sync(0xffffffffu, ((K - 1) >> 3) ? ov[1] : ov[0], (K - 1) & 7, 8);
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (!(c_v[j] > kth) || row3 >= a.M) { c_v[j] = -INFINITY; c_i[j] = 0x7fffffff; }
+      if (!__any_sync(0xffffffffu, cm > kth && row3 < a.M)) return;
+      const unsigned row_lanes = 0xffu << (lane & 24);
+      unsigned taken = 0;                                        // positions entrants took (the same in a row's threads)
+      int placed = 0;
+      float ev[2] = {0.f, 0.f};
+      int ei[2] = {0, 0};
+      bool mine0 = false, mine1 = false;
+#pragma unroll 1
+      for (int r = 0; r < K; ++r) {
+        float wv = c_v[0];
+        int wi = c_i[0];
+#pragma unroll
+        for (int i = 1; i < 16; ++i)
+          if (better(c_v[i], c_i[i], wv, wi)) { wv = c_v[i]; wi = c_i[i]; }
+#pragma unroll
+        for (int x = 4; x > 0; x >>= 1) {
+          const float yv = __shfl_xor_sync(0xffffffffu, wv, x, 8);
+          const int yi = __shfl_xor_sync(0xffffffffu, wi, x, 8);
+          if (better(yv, yi, wv, wi)) { wv = yv; wi = yi; }
+        }
+        const bool real = wi != 0x7fffffff;
+        if (!__any_sync(0xffffffffu, real)) break;
+        const unsigned b0 = __ballot_sync(0xffffffffu, better(ov[0], oi[0], wv, wi));
+        const unsigned b1 = __ballot_sync(0xffffffffu, better(ov[1], oi[1], wv, wi));
+        const int pos = __popc(b0 & row_lanes) + __popc(b1 & row_lanes) + placed;
+        if (real && pos < K) {
+          taken |= 1u << pos;
+          ++placed;
+          if (sub3 == (pos & 7)) {
+            if (pos >> 3) { ev[1] = wv; ei[1] = wi; mine1 = true; }
+            else { ev[0] = wv; ei[0] = wi; mine0 = true; }
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (c_i[i] == wi) { c_v[i] = -INFINITY; c_i[i] = 0x7fffffff; }   // (ids are distinct)
+        } else {
+          // nothing further of this row enters
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { c_v[i] = -INFINITY; c_i[i] = 0x7fffffff; }
+        }
+      }
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int k = sub3 + 8 * sl;
+        const int src = k - __popc(taken & ((1u << k) - 1u));    // the old entry that ends at k if no entrant did
+        const float f0 = __shfl_sync(0xffffffffu, ov[0], src & 7, 8), f1 = __shfl_sync(0xffffffffu, ov[1], src & 7, 8);
+        const int g0 = __shfl_sync(0xffffffffu, oi[0], src & 7, 8), g1 = __shfl_sync(0xffffffffu, oi[1], src & 7, 8);
+        const bool mine = sl ? mine1 : mine0;
+        if (!mine) {
+          ev[sl] = (src >> 3) ? f1 : f0;
+          ei[sl] = (src >> 3) ? g1 : g0;
+        }
+        if (k >= K) { ev[sl] = -INFINITY; ei[sl] = 0x7fffffff; }   // entries past K stay fillers
+      }
+      ov[0] = ev[0]; ov[1] = ev[1];
+      oi[0] = ei[0]; oi[1] = ei[1];
+    };
     // argmax mode: every lane keeps, in registers, the best (value, id) of its own rows for each of up to
     // 64 activation rows; the lanes are merged once, after the CTA's last tile
     float abv[ARGMAX ? 4 : 1][16];
@@ -458,17 +575,7 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
           for (int j = 0; j < 16; ++j) xt[j * XT_LD + t] = v[j];
         }
         epi_sync();
-        if (t < a.M) {
-          for (int c0 = 0; c0 < n_cols; c0 += 16) {
-            float v[16];
-#pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-              const float4 x4 = *reinterpret_cast<const float4*>(xt + t * XT_LD + c0 + j);
-              v[j] = x4.x; v[j + 1] = x4.y; v[j + 2] = x4.z; v[j + 3] = x4.w;
-            }
-            scan16(v, min(16, n_cols - c0), n0 + c0);
-          }
-        }
+        scan_tile3(n0, n_cols);
         epi_sync();                                              // the next tile overwrites the turned tile
       } else if (whole && a.mode != 3) {
         for (int c0 = 0; c0 < a.Npad && c0 < a.M; c0 += 16) {
@@ -577,7 +684,23 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
         a.pmax[o] = bv; a.psum[o] = 1.f; a.pval[o] = bv; a.pidx[o] = bi;
       }
     }
-    if (row_lists) {
+    if (VARIANT == 3) {
+      // ---- the row's list is already in order: entry k sits in thread k & 7, slot k >> 3
+      if (row3 < a.M) {
+        const size_t o = (size_t)row3 * gridDim.x + blockIdx.x;
+#pragma unroll
+        for (int k = 0; k < POSS_MAX_TOPK; ++k) {
+          if (k < K && sub3 == (k & 7)) {
+            a.pval[o * K + k] = ov[k >> 3];
+            a.pidx[o * K + k] = oi[k >> 3];
+          }
+        }
+        if (sub3 == 0) {
+          a.pmax[o] = r_max;
+          a.psum[o] = r_sum;
+        }
+      }
+    } else if (row_lists) {
       // ---- this thread's list, best first (value down, id up), is the CTA's list of its row
       if (t < a.M) {
         const size_t o = (size_t)t * gridDim.x + blockIdx.x;
