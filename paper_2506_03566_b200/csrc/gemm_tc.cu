@@ -107,11 +107,11 @@ struct Segment {
 
 // ------------------------------------------------------------------ the kernel
 // VARIANT 0: every epilogue but those below; 1: LM-head argmax only (lane-local state in registers); 2: LM-head
-// lists with the activation rows on the TMEM lanes (more than 16 rows); 3: LM-head lists for up to 16 rows, product
-// swapped like everywhere else and the accumulator tile turned through shared memory.  In 2 and 3 one thread owns
-// one activation row and scans its logits in the same order with the same operations, so a row's lists do not
-// depend on how many rows share the launch.  Separate instantiations, so that the registers of one epilogue never
-// cost another.
+// lists with the activation rows on the TMEM lanes (more than 16 rows), one thread per row; 3: LM-head lists for up
+// to 16 rows, product swapped like everywhere else, the accumulator tile turned through shared memory and eight
+// threads per row.  2 and 3 compute a row's maximum and sum with the same operations in the same order, and the K
+// best by (value down, id up) do not depend on how they are found, so a row's lists do not depend on how many rows
+// share the launch.  Separate instantiations, so that the registers of one epilogue never cost another.
 template <int VARIANT>
 __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ CUtensorMap map_x,
                                                        const __grid_constant__ CUtensorMap map_w0,
@@ -284,16 +284,16 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int t = q * 32 + lane;                  // row inside the tile
     const int K = a.topk;
-    // LM-head lists: this thread owns activation row t; running maximum and sum in registers, an unordered list
-    // of the K best (value, id) in shared memory, and in registers the list's worst entry: a candidate enters
-    // only if it beats that one (a later equal value carries a higher id and loses)
+    // LM-head lists, rows on lanes (variant 2): this thread owns activation row t; running maximum and sum in
+    // registers, an unordered list of the K best (value, id) in shared memory, and in registers the list's worst
+    // entry: a candidate enters only if it beats that one (a later equal value carries a higher id and loses)
     float* xt = extra;                                           // variant 3: the turned tile [16][XT_LD]
-    float* lists = extra + (VARIANT == 3 ? 16 * XT_LD : 0);
+    float* lists = extra;                                        // variant 2: one list per thread
     float* my_val = lists + (size_t)t * K;
     int* my_idx = reinterpret_cast<int*>(lists + (size_t)TILE_N * K) + (size_t)t * K;
     float r_max = -INFINITY, r_sum = 0.f, worst_v = -INFINITY;
     int worst_pos = 0, worst_i = 0x7fffffff;
-    if (row_lists) {
+    if (VARIANT == 2) {
       for (int i = 0; i < K; ++i) { my_val[i] = -INFINITY; my_idx[i] = 0x7fffffff; }
     }
     // sixteen consecutive logits of this thread's row (the first nv of them exist), vocabulary ids from id0 on
@@ -912,7 +912,8 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   if (ep.mode == TC_EPI_SWIGLU) extra = 64 * XCH_STRIDE * sizeof(float);
   // argmax only (no log-probabilities wanted, at most 64 rows): the lane-local epilogue, no running lists
   if (ep.mode == TC_EPI_TOPK && !argmax)
-    extra = (size_t)TILE_N * ep.topk * 8 + (a.rows_on_lanes ? 0 : (size_t)16 * (TILE_N + 4) * sizeof(float));
+    extra = a.rows_on_lanes ? (size_t)TILE_N * ep.topk * 8                    // one list per thread
+                            : (size_t)16 * (TILE_N + 4) * sizeof(float);       // the turned tile
   // rows on lanes: the activation operand is read as 128 rows from a tile that holds Npad of them; the last
   // stage's read runs up to 16 KB past the ring, into this slack (never written, never used)
   const size_t slack = a.rows_on_lanes ? (size_t)W_TILE_BYTES : 0;
@@ -920,7 +921,7 @@ void launch_gemm_tc(Launcher& L, TcGemmPlanCache* cache, const bf16* X, int ldx,
   // round, 190: +2, 210: +24), 200 KB = eight 24 KB stages at 64 rows (the target pass; 176 and 220 KB: +18 us
   // per pass)
   const int smem_kb = a.Npad <= 16 ? 170 : 200;
-  // (the slack and the per-thread lists of the LM-head epilogue come on top: the ring keeps its stages)
+  // (the slack and the lists or the turned tile of the LM-head epilogue come on top: the ring keeps its stages)
   const size_t on_top = lists ? slack + extra : 0;
   int stages = (int)(((size_t)smem_kb * 1024u + on_top - extra - slack - 1024u) / stage_bytes);
   while (stages > 2 && (size_t)stages * stage_bytes + slack + extra + 1024 > 225u * 1024u) --stages;
