@@ -645,6 +645,8 @@ void launch_rerank(Launcher& L, const TreeState& ts, int n_cand, int K, int tota
                    const int32_t* new_tokens, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
                    int32_t* out_depth, uint64_t* out_mask, int32_t* out_n_nodes) {
   size_t smem = (size_t)(n_cand + 4) * 16;
+  // (a round's tree slots fit two mask words, so at most 2064 candidates: 33 KB)
+  if (smem > 48 * 1024) { L.err = POSS_E_CAPACITY; return; }
   launch_pdl(L, k_rerank, dim3(rb.batch), dim3(1024), smem, ts, n_cand, K, total, rb, new_tokens, out_tokens,
              out_parents, out_scores, out_depth, out_mask, out_n_nodes);
 }
