@@ -55,6 +55,53 @@ def test_full_size_draft_round_matches_oracle(name, n_new, seed):
     assert int(g["n_nodes"][0]) == cfg.total + 1
 
 
+def test_full_size_batched_draft_round_equals_single_rounds_and_the_oracle():
+    """The batched workload bench.py times (--batch 12: Llama-3-8B shape, one specialist, width 10, depth 6, 60
+    tokens, twelve sequences = 120 stacked rows, the LM head with the rows on the TMEM lanes): sequences with their
+    own prefix lengths, caches and verified pairs.  Three of them are compared bit for bit with the single-sequence
+    call, and the first one with the oracle under the full-size rules."""
+    B = 12
+    cfg = ps.CONFIGS["c2"].replace(S=1, n=6)
+    w = ps.make_weights(cfg, 104)
+    n_news = [1 + (b % 3) for b in range(B)]
+    prefixes = [cfg.prefix - 7 * b for b in range(B)]
+    cap = cfg.prefix + 3 + cfg.tree_slots
+    from paper_2506_03566_b200 import Poss, make_config
+    P = Poss(make_config(cfg, cap, 0, max_batch=B), w)
+    kvs_np = [ps.make_draft_kv(cfg, 104 + 100 * b, cap, prefixes[b]) for b in range(B)]
+    ins = [ps.make_round_inputs(cfg, 104 + 100 * b, n_news[b]) for b in range(B)]
+    tok_all = torch.from_numpy(np.concatenate([t for t, _ in ins])).cuda()
+    feat_all = _dev(np.concatenate([f for _, f in ins], axis=0))
+    kvs = [_dev(k) for k in kvs_np]
+    out = P.poss_draft_round_batched(kvs, prefixes, tok_all, feat_all, n_news, cfg.depth, cfg.topk, cfg.total)
+    torch.cuda.synchronize()
+    assert P.poss_last_status() == 0
+    host = {k: pu.np_of(v) for k, v in out.items()}
+    keep = {}
+    for b in (0, 5, B - 1):
+        tr = {k: pu.np_of(v) for k, v in P.poss_draft_trace(cfg.depth, cfg.topk, int(host["n_nodes"][b]), seq=b).items()}
+        gb = {k: (host[k][b] if k != "n_nodes" else host[k][b:b + 1]) for k in host}
+        gb["anc_mask"] = gb["anc_mask"].view(np.uint64)
+        keep[b] = (gb, tr)
+    for b in (0, 5, B - 1):
+        gb, tr = keep[b]
+        g1, tr1, dkv1 = pu.run_gpu_round(P, cfg, kvs_np[b], prefixes[b], ins[b][0], ins[b][1], cfg.depth, cfg.topk, cfg.total)
+        for k in ("tokens", "parents", "scores", "depth", "anc_mask", "n_nodes"):
+            assert np.array_equal(gb[k], g1[k]), (b, k)
+        for k in tr1:
+            assert np.array_equal(tr[k], tr1[k]), (b, k)
+        assert torch.equal(kvs[b], dkv1), f"sequence {b}: cache entries differ from the single round's"
+        assert int(gb["n_nodes"][0]) == cfg.total + 1
+    P.close()
+    del P
+    torch.cuda.empty_cache()
+    gb, tr = keep[0]
+    rep = pu.compare_round(cfg, w, kvs_np[0], prefixes[0], ins[0][0], ins[0][1], cfg.depth, cfg.topk, cfg.total, gb, tr,
+                           pu.oracle_num(cfg, big=True), False, noise_num=po.Num(np.float64, "bf16"))
+    pu.compare_kv(cfg, kvs[0], rep["kv_oracle"], prefixes[0], prefixes[0] + n_news[0], pu.TOL[cfg.dtype])
+    print("batched c2 x 12", {k: v for k, v in rep.items() if k != "kv_oracle"})
+
+
 @pytest.mark.parametrize("rows,P_len", [(61, 1024), (81, 8192)])
 def test_full_size_verification_attention_matches_oracle(rows, P_len):
     """Target geometry of the Llama-3-8B shape: 32 query heads, 8 KV heads, head_dim 128."""
