@@ -542,6 +542,11 @@ __global__ void __launch_bounds__(N_THREADS) k_gemm_tc(const __grid_constant__ C
 #pragma unroll
               for (int j = 0; j < 16; ++j)
                 if (v[j] > abv[cc][j]) { abv[cc][j] = v[j]; abi[cc][j] = n_local; }   // rows only grow: ties keep the lower id
+              if (a.out) {                                       // the caller also wants the logits: same read
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  if (c0 + j < a.M) a.out[(size_t)(c0 + j) * a.ldo + col] = v[j];
+              }
             }
           }
         }

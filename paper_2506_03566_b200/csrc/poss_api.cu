@@ -213,7 +213,9 @@ struct Impl {
   void attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc, T* out);
   void attention_batch(const AttnArgs& aa, const AttnBatch& ab, const T* q, T* out);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
-  bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists, bool argmax_only = false);
+  // logits_out (argmax only, at most 64 rows): the fp32 logits are stored from the same accumulator read
+  bool gemm_topk_partials(const T* x, int M, int K, int topk, int* n_lists, bool argmax_only = false,
+                          float* logits_out = nullptr);
 
   // need_logp = false (with K = 1): the caller wants the argmax only; logp is then meaningless
   void lm_head_topk(const T* feats, int rows, int K, int32_t* ids, float* logp, float* logits_out,
@@ -223,7 +225,11 @@ struct Impl {
     float* lg = logits_out ? logits_out : c->b.logits;
     int pr = expand != nullptr ? prof_begin(POSS_PROF_LM_HEAD) : -1;   // the draft steps' launches only
     int n_lists = 0;
-    bool fused = !logits_out && gemm_topk_partials(feats, rows, g.hidden, K, &n_lists, !need_logp && K == 1);
+    // wanted logits leave the fused path, except where the argmax epilogue can store them on its way
+    const bool argmax_only = !need_logp && K == 1;
+    const bool store_too = logits_out && argmax_only && rows <= 64;
+    bool fused = (!logits_out || store_too) &&
+                 gemm_topk_partials(feats, rows, g.hidden, K, &n_lists, argmax_only, store_too ? logits_out : nullptr);
     if (!fused) gemm(feats, g.hidden, rows, sg, g.hidden, nullptr, nullptr, 0, lg, g.vocab, 0, nullptr, POSS_K_GEMM_LM_HEAD);
     prof_end(pr);
     if (!fused) {
@@ -569,13 +575,15 @@ void Impl<bf16>::attention_batch(const AttnArgs& aa, const AttnBatch& ab, const 
 }
 
 template <typename T>
-bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*, bool) { return false; }
+bool Impl<T>::gemm_topk_partials(const T*, int, int, int, int*, bool, float*) { return false; }
 template <>
-bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists, bool argmax_only) {
+bool Impl<bf16>::gemm_topk_partials(const bf16* x, int M, int K, int topk, int* n_lists, bool argmax_only,
+                                    float* logits_out) {
   GemmSegs sg; sg.n = 1; sg.w[0] = c->lm_head; sg.rows[0] = c->cfg.vocab;
   if (!tc_gemm_supported(sg, K, K, M)) return false;
   TcEpilogue ep;
   ep.mode = TC_EPI_TOPK; ep.topk = topk; ep.argmax_only = argmax_only; ep.trace_tag = POSS_K_GEMM_LM_HEAD;
+  ep.out = logits_out; ep.ldo = c->cfg.vocab;
   ep.pmax = c->b.pmax; ep.psum = c->b.psum; ep.pval = c->b.pval; ep.pidx = c->b.pidx; ep.n_lists = n_lists;
   launch_gemm_tc(L, c->tc, x, K, M, sg, K, ep, c->b.tc_scratch, c->b.status);
   return true;
