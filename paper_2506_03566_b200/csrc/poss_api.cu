@@ -209,7 +209,7 @@ struct Impl {
   // act[M][F] = T(silu(x . gate^T) * (x . up^T))
   void gemm_swiglu(const T* x, int M, const void* w_gate, const void* w_up, int F, int K, T* act);
   // tree-masked attention: the tcgen05 kernel where it covers the call (bf16, head dimension 128, at most
-  // 2048 keys), else the split-KV kernels with their partial buffer
+  // 10240 keys), else the split-KV kernels with their partial buffer
   void attention(const AttnArgs& aa, const T* q, const T* kc, const T* vc, T* out);
   void attention_batch(const AttnArgs& aa, const AttnBatch& ab, const T* q, T* out);
   // per-row max / sum-exp / top-k partial lists of x . lm_head^T without storing the logits; false = not covered
