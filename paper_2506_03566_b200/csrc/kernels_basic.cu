@@ -139,22 +139,6 @@ template void launch_gather_x<float>(Launcher&, const BatchRows&, const int32_t*
 template void launch_gather_x<bf16>(Launcher&, const BatchRows&, const int32_t*, const bf16*, const TreeState&, int,
                                     const bf16*, int, const bf16*, int, bf16*);
 
-template <typename T>
-__global__ void k_embed_rows(const int32_t* tokens, const T* embed, int H,
-                             float* out) {
-  pdl_enter(POSS_K_EMBED_ROWS);
-  int m = blockIdx.x;
-  const T* e = embed + (size_t)tokens[m] * H;
-  for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)m * H + i] = to_f(e[i]);
-}
-template <typename T>
-void launch_embed_rows(Launcher& L, const int32_t* tokens, int rows, const T* embed, int H, float* out) {
-  if (rows <= 0) return;
-  launch_pdl(L, k_embed_rows<T>, dim3(rows), dim3(256), 0, tokens, embed, H, out);
-}
-template void launch_embed_rows<float>(Launcher&, const int32_t*, int, const float*, int, float*);
-template void launch_embed_rows<bf16>(Launcher&, const int32_t*, int, const bf16*, int, float*);
-
 // ------------------------------------------------------------------ RMSNorm: out = T(gain * x / sqrt(mean x^2 + eps))
 template <typename T>
 __global__ void __launch_bounds__(256) k_rmsnorm(const float* x, int H, const T* gain,
@@ -292,6 +276,34 @@ template <> __device__ __forceinline__ void store4<bf16>(bf16* p, const float* v
   *reinterpret_cast<uint2*>(p) = raw;
 }
 __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// ------------------------------------------------------------------ embedding rows as fp32 (the target pass's input)
+template <typename T>
+__global__ void k_embed_rows(const int32_t* tokens, const T* embed, int H,
+                             float* out) {
+  pdl_enter(POSS_K_EMBED_ROWS);
+  int m = blockIdx.x;
+  const T* e = embed + (size_t)tokens[m] * H;
+  float* o = out + (size_t)m * H;
+  // four elements per access where the row allows it (the rows are cold: few, wide loads in flight together)
+  if ((H & 3) == 0 && aligned16(o) && (reinterpret_cast<uintptr_t>(e) & (4 * sizeof(T) - 1)) == 0) {
+    for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+      float v[4];
+      load4<T>(e + i, v);
+      store4<float>(o + i, v);
+    }
+    return;
+  }
+  for (int i = threadIdx.x; i < H; i += blockDim.x) o[i] = to_f(e[i]);
+}
+template <typename T>
+void launch_embed_rows(Launcher& L, const int32_t* tokens, int rows, const T* embed, int H, float* out) {
+  if (rows <= 0) return;
+  launch_pdl(L, k_embed_rows<T>, dim3(rows), dim3(256), 0, tokens, embed, H, out);
+}
+template void launch_embed_rows<float>(Launcher&, const int32_t*, int, const float*, int, float*);
+template void launch_embed_rows<bf16>(Launcher&, const int32_t*, int, const bf16*, int, float*);
+
 
 // four consecutive entries of a weight vector (bias, gain) as floats; `fill` where there is none
 template <typename T>
